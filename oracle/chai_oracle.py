@@ -1,0 +1,161 @@
+"""ctypes front end of the CPU oracle (test infrastructure, never the product path).
+
+Compiles ``chai_oracle.c`` with gcc into ``libchai_oracle.so`` next to this file on
+first use and exposes numpy-in / numpy-out wrappers.  Stored values (bf16 or fp32
+bits) are widened exactly to float64 before they reach the C code.
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "chai_oracle.c")
+_LIB = os.path.join(_HERE, "libchai_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (fp contraction off, OpenMP on) and return the library path."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared",
+               "-Wall", "-Wextra", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        dp = ctypes.POINTER(ctypes.c_double)
+        ip = ctypes.POINTER(ctypes.c_int32)
+        lib.oracle_cha_attention.argtypes = [dp, dp, dp, ip, ip, dp] + [ctypes.c_int] * 6 + [
+            ctypes.c_double, ctypes.c_int]
+        lib.oracle_cha_attention.restype = ctypes.c_int
+        lib.oracle_prefix_features.argtypes = [dp, dp, dp] + [ctypes.c_int] * 5 + [ctypes.c_double]
+        lib.oracle_prefix_features.restype = ctypes.c_int
+        lib.oracle_kmeans.argtypes = [dp, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                      ctypes.c_uint64, ip, ip, ip, dp, dp, ip]
+        lib.oracle_kmeans.restype = ctypes.c_int
+        lib.oracle_compact_k_cache.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ip] + [
+            ctypes.c_int] * 6 + [ctypes.POINTER(ctypes.c_int64)]
+        lib.oracle_compact_k_cache.restype = ctypes.c_int
+        lib.oracle_num_threads.restype = ctypes.c_int
+        lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
+        _lib = lib
+    return _lib
+
+
+def _f64(x) -> np.ndarray:
+    """Exact widening to a C-contiguous float64 array (accepts numpy arrays and torch CPU tensors)."""
+    if hasattr(x, "detach"):
+        x = x.detach().cpu().double().numpy()
+    return np.ascontiguousarray(x, dtype=np.float64)
+
+
+def _i32(x) -> np.ndarray:
+    if hasattr(x, "detach"):
+        x = x.detach().cpu().numpy()
+    return np.ascontiguousarray(x, dtype=np.int32)
+
+
+def _dp(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _ip(a):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    _load().oracle_set_num_threads(int(n))
+
+
+def cha_attention(q, k_rep, v, membership, reps, scale: float, causal: bool) -> np.ndarray:
+    """Clustered-head attention.  q [B,H,Tq,D] (or [B,H,D] for decode), k_rep [B,k,T,D],
+    v [B,H,T,D], membership [B,H], reps [B,k]  ->  float64 output shaped like q."""
+    q = _f64(q)
+    decode = q.ndim == 3
+    if decode:
+        q = q[:, :, None, :]
+    k_rep, v = _f64(k_rep), _f64(v)
+    membership, reps = _i32(membership), _i32(reps)
+    B, H, Tq, D = q.shape
+    k, T = k_rep.shape[1], k_rep.shape[2]
+    assert k_rep.shape == (B, k, T, D) and v.shape == (B, H, T, D)
+    assert membership.shape == (B, H) and reps.shape == (B, k)
+    out = np.empty((B, H, Tq, D), dtype=np.float64)
+    rc = _load().oracle_cha_attention(_dp(q), _dp(k_rep), _dp(v), _ip(membership), _ip(reps),
+                                      _dp(out), B, H, k, Tq, T, D, float(scale), int(bool(causal)))
+    if rc != 0:
+        raise ValueError("oracle_cha_attention rejected its arguments")
+    return out[:, :, 0, :] if decode else out
+
+
+def prefix_features(q_full, k_full, P: int, scale: float) -> np.ndarray:
+    """q_full, k_full [B,H,T,D] -> features [B,H,P*P] float64."""
+    q_full, k_full = _f64(q_full), _f64(k_full)
+    B, H, T, D = q_full.shape
+    out = np.empty((B, H, P * P), dtype=np.float64)
+    rc = _load().oracle_prefix_features(_dp(q_full), _dp(k_full), _dp(out), B, H, T, D, int(P),
+                                        float(scale))
+    if rc != 0:
+        raise ValueError("oracle_prefix_features rejected its arguments")
+    return out
+
+
+def kmeans(features, k: int, max_iter: int = 20, seed: int = 0):
+    """features [B,H,F] (or [H,F]) -> dict(membership [B,H], reps [B,k], k_eff [B], inertia [B],
+    trace [B,max_iter], init_idx [B,k]); every request is clustered independently."""
+    x = _f64(features)
+    single = x.ndim == 2
+    if single:
+        x = x[None]
+    B, H, F = x.shape
+    membership = np.empty((B, H), dtype=np.int32)
+    reps = np.empty((B, k), dtype=np.int32)
+    k_eff = np.empty((B,), dtype=np.int32)
+    inertia = np.empty((B,), dtype=np.float64)
+    trace = np.empty((B, max_iter), dtype=np.float64)
+    init_idx = np.empty((B, k), dtype=np.int32)
+    lib = _load()
+    for b in range(B):
+        xb = np.ascontiguousarray(x[b])
+        rc = lib.oracle_kmeans(_dp(xb), H, F, int(k), int(max_iter), ctypes.c_uint64(int(seed)),
+                               _ip(membership[b]), _ip(reps[b]), _ip(k_eff[b:b + 1]),
+                               _dp(inertia[b:b + 1]), _dp(trace[b]), _ip(init_idx[b]))
+        if rc != 0:
+            raise ValueError("oracle_kmeans rejected its arguments")
+    res = dict(membership=membership, reps=reps, k_eff=k_eff, inertia=inertia, trace=trace,
+               init_idx=init_idx)
+    if single:
+        res = {n: a[0] for n, a in res.items()}
+    return res
+
+
+def compact_k_cache(k_full: np.ndarray, reps) -> tuple[np.ndarray, tuple[int, int]]:
+    """k_full [B,H,T,D] of any fixed-size dtype (pass bf16 as its uint16 bit pattern) ->
+    (k_rep [B,k,T,D] same dtype, (kv_bytes_before, kv_bytes_after))."""
+    k_full = np.ascontiguousarray(k_full)
+    reps = _i32(reps)
+    B, H, T, D = k_full.shape
+    k = reps.shape[1]
+    out = np.empty((B, k, T, D), dtype=k_full.dtype)
+    nbytes = np.zeros(2, dtype=np.int64)
+    rc = _load().oracle_compact_k_cache(k_full.ctypes.data_as(ctypes.c_void_p),
+                                        out.ctypes.data_as(ctypes.c_void_p), _ip(reps), B, H, k, T,
+                                        D, k_full.dtype.itemsize,
+                                        nbytes.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)))
+    if rc != 0:
+        raise ValueError("oracle_compact_k_cache rejected its arguments")
+    return out, (int(nbytes[0]), int(nbytes[1]))
