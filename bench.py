@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the clustered-head-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 2|3|4]
+
+One *step* is one decode step of the whole model-shaped workload: the L per-layer
+chai_decode_attention calls for one new token per request, enqueued back to back on one stream.
+All layers' caches are resident in HBM, each layer has its own buffers, and one layer's working set
+(>= 168 MiB) already exceeds L2, so every step streams from DRAM.  The headline value is algorithmic
+bytes per step / step time (GB/s); microseconds per step ride along.  The same run also times
+clustered prefill (workload 5) and K-cache compaction (workload 4's shape) and reports them as
+extra objects of the one JSON line.
+
+With N > 1 (torchrun) every rank runs an independent replica of the workload on its own GPU: the
+path has no exchange step, so there is no collective on the data path; the barrier and the
+max-over-ranks reduction are the only communication.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2403_08058_b200 import chai, synth  # noqa: E402
+
+METRIC = "clustered decode attention: algorithmic HBM GB/s over one decode step (us/step alongside)"
+UNIT = "GB/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=float(p["hbm_gbs"]), tf_burst=float(p["bf16_tflops"]),
+                    tf_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:  # NVML missing: clocks are reported as unknown
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        return dict(sm_mhz=(statistics.median(self.samples) if self.samples else None), sm_max_mhz=self.max_mhz,
+                    reasons=sorted(self.reasons), samples=len(self.samples))
+
+
+def decode_bytes(B, H, k, T, D, es):
+    """Algorithmic bytes of one layer's decode call: (k+H) cache planes, the representatives' query rows,
+    the outputs and the two maps."""
+    return (k + H) * B * T * D * es + k * B * D * es + H * B * D * es + 4 * B * (H + k)
+
+
+def prefill_flops(B, H, k, T, D):
+    """Causal pairs only: one QK^T per cluster and one PV per head, 2*D flops per (row, key) pair each."""
+    return 2 * D * (T * (T + 1) // 2) * (k + H) * B
+
+
+class DecodeWorkload:
+    def __init__(self, cfg_id: int, device, seed: int = 0):
+        w = synth.WORKLOADS[cfg_id]
+        self.w, self.cfg_id, self.device = w, cfg_id, device
+        self.layers = []
+        self.es = 2 if w.dtype == "bf16" else 4
+        self.dt = chai.CHAI_BF16 if w.dtype == "bf16" else chai.CHAI_F32
+        ws_bytes = 0
+        for layer in range(w.layers):
+            c = synth.decode_layer(cfg_id, layer, seed, device=device, with_k_full=False)
+            c["out"] = torch.empty_like(c["q"])
+            ws_bytes = max(ws_bytes, chai.chai_decode_workspace_bytes(w.B, w.H, c["k"], w.T, w.D, self.dt))
+            self.layers.append(c)
+        self.ws = chai.new_workspace(ws_bytes, device)
+        self.bytes_per_layer = [decode_bytes(w.B, w.H, c["k"], w.T, w.D, self.es) for c in self.layers]
+        self.bytes_per_step = sum(self.bytes_per_layer)
+        self.launches_per_step = 2 * w.layers
+
+    def step(self):
+        for c in self.layers:
+            chai.chai_decode_attention(c["q"], c["k_rep"], c["v"], c["membership"], c["reps"], c["scale"], out=c["out"],
+                                       workspace=self.ws)
+
+    def step_with_events(self, events):
+        events[0].record()
+        for i, c in enumerate(self.layers):
+            chai.chai_decode_attention(c["q"], c["k_rep"], c["v"], c["membership"], c["reps"], c["scale"], out=c["out"],
+                                       workspace=self.ws)
+            events[i + 1].record()
+
+    def make_host_buffers(self):
+        self.q_host = [c["q"].cpu().pin_memory() for c in self.layers]
+        self.o_host = [torch.empty_like(q).pin_memory() for q in self.q_host]
+        self.q_stage = torch.empty_like(self.layers[0]["q"])
+        self.o_stage = torch.empty_like(self.layers[0]["q"])
+
+    def step_host(self):
+        for c, qh, oh in zip(self.layers, self.q_host, self.o_host):
+            chai.chai_decode_attention_host(qh, oh, self.q_stage, self.o_stage, c["k_rep"], c["v"], c["membership"],
+                                            c["reps"], c["scale"], self.ws)
+
+
+def time_region(fn, steps, sync_all):
+    """Times `steps` calls of fn with CUDA events on the current stream; barrier + synchronize on both sides."""
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    sync_all()
+    return ms
+
+
+def cpu_baseline_decode(cfg_id: int, seed: int, budget_s: float = 15.0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the same workload: whole layers of
+    the decode step, request by request, until about `budget_s` seconds of oracle time are spent."""
+    from oracle import chai_oracle as orc
+    w = synth.WORKLOADS[cfg_id]
+    es = 2 if w.dtype == "bf16" else 4
+    spent, nbytes, n_req, layer = 0.0, 0, 0, 0
+    while spent < budget_s and layer < w.layers:
+        c = synth.decode_layer(cfg_id, layer, seed, device="cpu", B=2, with_k_full=False)
+        args = [orc._f64(c[n]) for n in ("q", "k_rep", "v")]
+        t0 = time.perf_counter()
+        orc.cha_attention(args[0], args[1], args[2], c["membership"], c["reps"], c["scale"], causal=False)
+        spent += time.perf_counter() - t0
+        nbytes += decode_bytes(2, w.H, c["k"], w.T, w.D, es)
+        n_req += 2
+        layer += 1
+    return dict(value=nbytes / spent / 1e9, unit=UNIT, cores=orc.num_threads(), kind="oracle",
+                sample=f"{layer} layers x 2 requests of workload {cfg_id} ({n_req} request-layers, "
+                       f"{spent:.1f} s of oracle time, inputs already widened to fp64)", seconds=spent)
+
+
+def run_reference(args, rank):
+    """The reference arm of this tier is the CPU oracle timed on the host cores."""
+    if rank != 0:
+        return
+    from oracle import chai_oracle as orc
+    cfg_id = args.workload
+    w = synth.WORKLOADS[cfg_id]
+    es = 2 if w.dtype == "bf16" else 4
+    c = synth.decode_layer(cfg_id, 0, 0, device="cpu", B=2, with_k_full=False)
+    a = [orc._f64(c[n]) for n in ("q", "k_rep", "v")]
+    nbytes = decode_bytes(2, w.H, c["k"], w.T, w.D, es)
+
+    def step():
+        orc.cha_attention(a[0], a[1], a[2], c["membership"], c["reps"], c["scale"], causal=False)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = nbytes * args.steps / dt / 1e9
+    sample = f"each step = layer 0, 2 of {w.B} requests of workload {cfg_id} (fp64 oracle, inputs pre-widened)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def bench_prefill(device, peaks, iters=20, warmup=3):
+    case = synth.prefill_case(seed=0, device=device)
+    B, H, T, D, k = case["B"], case["H"], case["T"], case["D"], case["k"]
+    k_rep = chai.chai_compact_k_cache(case["k_full"], case["reps"])
+    ws = chai.new_workspace(chai.chai_prefill_workspace_bytes(B, H, k, T, D, chai.CHAI_BF16), device)
+    out = torch.empty_like(case["q_full"])
+    feats = torch.empty((B, H, 25), device=device, dtype=torch.float32)
+
+    def attn():
+        chai.chai_prefill_attention(case["q_full"], k_rep, case["v"], case["membership"], case["reps"], case["scale"],
+                                    True, out=out, workspace=ws)
+
+    def flow():
+        chai.chai_prefix_features(case["q_full"], case["k_full"], 5, case["scale"], features=feats)
+        mem, reps, _, _ = chai.chai_cluster_heads(feats, k, 20, 0, want_inertia=False)
+        chai.chai_compact_k_cache(case["k_full"], reps, k_rep=k_rep)
+        chai.chai_prefill_attention(case["q_full"], k_rep, case["v"], mem, reps, case["scale"], True, out=out,
+                                    workspace=ws)
+
+    res = {}
+    for name, fn in (("attention", attn), ("flow", flow)):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        res[name] = statistics.median(ts)
+    fl = prefill_flops(B, H, k, T, D)
+    tf = fl / (res["attention"] * 1e-3) / 1e12
+    return {
+        "workload": synth.WORKLOADS[5].name, "ms_attention": res["attention"], "ms_flow_features_kmeans_compact_attention": res["flow"],
+        "algorithmic_gflop": fl / 1e9, "tflops": tf,
+        "roofline": {"bound": "tensor", "achieved": tf, "peak": peaks["tf_burst"], "unit": "TFLOP/s",
+                     "frac": tf / peaks["tf_burst"], "peak_source": peaks["source"] + " (burst: kernel timed alone)",
+                     "traffic": None},
+        "l2": "working set 168 MB per call exceeds L2",
+    }
+
+
+def bench_compaction(device, peaks, iters=20, warmup=3):
+    w = synth.WORKLOADS[4]
+    k = 24
+    g = torch.Generator(device=device).manual_seed(4)
+    k_full = torch.randn((w.B, w.H, w.T, w.D), device=device, generator=g).to(torch.bfloat16)
+    _, reps = synth.batch_partitions(w.B, w.H, k, "uneven", 0, 4, 0)
+    reps = torch.as_tensor(reps, device=device)
+    k_rep = torch.empty((w.B, k, w.T, w.D), device=device, dtype=torch.bfloat16)
+    flush = torch.empty(256 << 20, device=device, dtype=torch.uint8)
+    ts = []
+    for i in range(warmup + iters):
+        flush.fill_(i & 1)  # 256 MB write: evicts L2 between iterations
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        chai.chai_compact_k_cache(k_full, reps, k_rep=k_rep)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= warmup:
+            ts.append(e0.elapsed_time(e1))
+    ms = statistics.median(ts)
+    nbytes = 2 * k * w.B * w.T * w.D * 2
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"workload": "config4 one layer, k=24", "us": ms * 1e3, "algorithmic_mb": nbytes / 1e6, "gbs": gbs,
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"],
+                         "peak_source": peaks["source"], "traffic": None}, "l2": "flushed by a 256 MB write"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4])
+    ap.add_argument("--skip-extras", action="store_true", help="only the decode step (no prefill/compaction/CPU legs)")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    chai.load()
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist_mod.init_process_group("nccl", device_id=device)
+        dist = dist_mod
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    peaks = load_peaks()
+    wl = DecodeWorkload(args.workload, device)
+    w = wl.w
+    for _ in range(args.warmup):
+        wl.step()
+    # 1) device-resident timing: exactly K steps, two events
+    with ClockSampler(local_rank) as clk:
+        ms_total = time_region(wl.step, args.steps, sync_all)
+        # 2) same K steps again with an event after every layer call: per-launch durations for the roofline
+        events = [[torch.cuda.Event(enable_timing=True) for _ in range(w.layers + 1)] for _ in range(args.steps)]
+        sync_all()
+        for s in range(args.steps):
+            wl.step_with_events(events[s])
+        torch.cuda.synchronize()
+    layer_ms = np.array([[ev[i].elapsed_time(ev[i + 1]) for i in range(w.layers)] for ev in events])
+    # 3) end to end through the host-buffer entry point: H2D of every layer's queries, D2H of every output
+    wl.make_host_buffers()
+    for _ in range(3):
+        wl.step_host()
+    ms_e2e = time_region(wl.step_host, args.steps, sync_all)
+
+    if dist is not None:
+        t = torch.tensor([ms_total, ms_e2e], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_step = ms_total / args.steps
+    value = world * wl.bytes_per_step / (ms_step * 1e-3) / 1e9
+    e2e_value = world * wl.bytes_per_step / (ms_e2e / args.steps * 1e-3) / 1e9
+
+    if rank == 0:
+        per_launch_ms = float(layer_ms.mean())
+        achieved = float(np.mean(wl.bytes_per_layer)) / (per_launch_ms * 1e-3) / 1e9
+        by_k = {}
+        for c, col in zip(wl.layers, layer_ms.T):
+            by_k.setdefault(c["k"], []).append(float(np.median(col)) * 1e3)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 storage, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": w.name, "layers": w.layers, "B": w.B, "H": w.H, "D": w.D, "T": w.T,
+                       "k_per_layer": [c["k"] for c in wl.layers], "partition": w.partition,
+                       "algorithmic_gb_per_step": wl.bytes_per_step / 1e9,
+                       "l2": "inputs larger than L2: every layer has its own >=168 MiB caches, 12+ GB per step",
+                       "multi_gpu": "independent replicas, no data-path collective"},
+            "gpu_launches": wl.launches_per_step * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "decode_scores_kernel + decode_pv_kernel (one layer call)",
+                         "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
+                         "peak_source": peaks["source"], "traffic": None,
+                         "us_per_layer_by_k": {str(k): statistics.median(v) for k, v in sorted(by_k.items())},
+                         "frac_of_nominal_8TBs": achieved / 8000.0},
+            "e2e": {"value": e2e_value, "unit": UNIT, "us_per_step": ms_e2e / args.steps * 1e3,
+                    "h2d_bytes_per_step": w.layers * w.B * w.H * w.D * wl.es,
+                    "d2h_bytes_per_step": w.layers * w.B * w.H * w.D * wl.es,
+                    "note": "queries from pinned host memory and outputs back to it every layer; caches stay resident"},
+            "clocks": clk.summary(),
+        }
+        if not args.skip_extras and world == 1:
+            del wl
+            torch.cuda.empty_cache()
+            line["prefill"] = bench_prefill(device, peaks)
+            line["compaction"] = bench_compaction(device, peaks)
+            line["cpu_baseline"] = cpu_baseline_decode(args.workload, 0)
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

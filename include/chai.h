@@ -1,0 +1,155 @@
+/*
+ * chai.h -- C ABI of the B200 clustered-head-attention library (libchai.so).
+ *
+ * The library implements the inference hot path of CHAI (Clustered Head
+ * Attention, arXiv 2403.08058): per request, the heads of a layer are grouped by
+ * k-means over attention-score features of a five-token prompt prefix; afterwards
+ * only each cluster's representative head computes Q K^T and the softmax, against
+ * a key cache that stores representative heads only, and every member head
+ * applies those shared probabilities to its own value cache.
+ *
+ * Conventions common to every entry point
+ *   - All tensor arguments are DEVICE pointers to contiguous row-major arrays
+ *     unless the name ends in _host.  Pointers must be 16-byte aligned.
+ *   - Ownership: the caller allocates and frees every buffer, including the
+ *     workspace.  The library allocates no device memory and keeps no state
+ *     between calls other than the text of the last error.
+ *   - Asynchrony: a call validates its scalar arguments on the host, enqueues its
+ *     kernels on `stream` (a cudaStream_t passed as void*) and returns; it never
+ *     synchronises, except chai_device_status and the *_host entry points.
+ *   - Errors: the return value is a chai_status_t.  Anything checkable on the host
+ *     (null or misaligned pointer, non-positive size, k > H, unsupported head
+ *     dimension, workspace too small) is refused before any launch.  Errors in
+ *     device-resident data (membership[b][h] outside [0,k), reps[b][c] outside
+ *     {-1} U [0,H), membership[b][reps[b][c]] != c) cannot be seen by the host:
+ *     the kernels record CHAI_ERR_BAD_MEMBERSHIP in the status word at the head of
+ *     the workspace, give the affected heads an all-zero output and never form an
+ *     out-of-range address.  Read the word with chai_device_status.
+ *   - dtype: CHAI_F32 or CHAI_BF16 for Q, K, V and the output; accumulation is
+ *     always fp32.  Head dimension D must be 64 or 128.
+ *   - T counts cached positions INCLUDING the current token; T_cap (>= T) is the
+ *     row capacity of the caches, i.e. the stride between heads is T_cap*D.
+ *   - membership [B,H] int32: cluster id of each head.  reps [B,k] int32: head
+ *     index of each cluster's representative, or -1 for an unused cluster slot.
+ *     Both are per request (Section 3.5: membership is decided for each request).
+ */
+#ifndef CHAI_H_
+#define CHAI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CHAI_OK = 0,
+    CHAI_ERR_INVALID_ARG = 1,    /* null/misaligned pointer, non-positive size, k > H, T > T_cap ... */
+    CHAI_ERR_UNSUPPORTED = 2,    /* head_dim not 64/128, unknown dtype, problem too large for a kernel */
+    CHAI_ERR_WORKSPACE = 3,      /* workspace_bytes smaller than the matching *_workspace_bytes() */
+    CHAI_ERR_BAD_MEMBERSHIP = 4, /* device status word only: inconsistent membership / reps */
+    CHAI_ERR_TIMEOUT = 5,        /* device status word only: a bounded device-side wait expired */
+    CHAI_ERR_CUDA = 6            /* a CUDA call failed; text in chai_last_error() */
+} chai_status_t;
+
+typedef enum { CHAI_F32 = 0, CHAI_BF16 = 1 } chai_dtype_t;
+
+/*
+ * Prefix score features (Section 3.3 and Fig. 6(b): the first five tokens of a
+ * request run with plain multi-head attention and their attention scores are what
+ * is clustered; Section 3.1 defines head similarity on softmax(Q K^T)).
+ *   q_full, k_full  [B,H,T_cap,D]  every head's own queries / keys; rows 0..P-1 are read
+ *   features        [B,H,P*P] fp32 out: entry i*P+j = causal softmax probability of
+ *                   query i on key j (j <= i) of that head, 0 for j > i
+ * 1 <= P <= 32, P <= T_cap.
+ */
+int chai_prefix_features(const void* q_full, const void* k_full, int B, int H, int T_cap, int D, int P,
+                         float scale, int dtype, float* features, void* stream);
+
+/*
+ * Cluster membership by k-means (Section 3.5: K-Means once five tokens have been
+ * processed; Section 3.2: error = sum of squared distances to the closest centre).
+ * Deterministic: seeded farthest-first initial centres (first = seed mod H; ties
+ * to the lowest index), Lloyd iterations in fp64 until the assignment repeats or
+ * max_iter assignments were made, empty clusters keep their centre, clusters are
+ * renumbered by their lowest member and the lowest member is the representative.
+ *   features   [B,H,F] fp32         one request = one independent problem
+ *   membership [B,H] int32 out      cluster id in [0,k_eff)
+ *   reps       [B,k] int32 out      representative head; -1 for slots >= k_eff
+ *   k_eff      [B] int32 out        number of non-empty clusters (< k only when fewer
+ *                                   than k distinct feature vectors exist)
+ *   inertia    [B] fp64 out or NULL sum of squared distances to the members' means
+ * 1 <= k <= H <= 1024; (H+k)*F + H*k doubles must fit in 200 KB of shared memory.
+ */
+int chai_cluster_heads(const float* features, int B, int H, int F, int k, int max_iter, uint64_t seed,
+                       int32_t* membership, int32_t* reps, int32_t* k_eff, double* inertia, void* stream);
+
+/*
+ * K-cache compaction (Section 3.5: once membership is fixed the keys of pruned
+ * heads are removed; Section 4.3: all values are kept).
+ *   k_full [B,H,T_cap,D] -> k_rep [B,k,T_cap,D]:  k_rep[b][c][0..T) = k_full[b][reps[b][c]][0..T)
+ * Bit copy, out of place; the buffers must not overlap.  A slot with reps = -1 (or
+ * an out-of-range head) is zero-filled.
+ */
+int chai_compact_k_cache(const void* k_full, void* k_rep, const int32_t* reps, int B, int H, int k, int T,
+                         int T_cap, int D, int dtype, void* stream);
+
+/*
+ * Clustered decode attention, one new token per request (Fig. 3(b), Section 3.4,
+ * Section 4.3; A = softmax(Q K^T / sqrt(d)) of Section 2 with `scale` given explicitly).
+ *   q    [B,H,D]         all heads' queries; only q[b][reps[b][c]] is read
+ *   k_rep[B,k,T_cap,D]   representative-only key cache
+ *   v    [B,H,T_cap,D]   full value cache
+ *   out  [B,H,D]         out[b][h] = sum_t softmax_t(scale * q[b][r] . k_rep[b][c][t]) * v[b][h][t],
+ *                        c = membership[b][h], r = reps[b][c], over t in [0,T)
+ * The workspace holds the scores, split-KV partials and the status word; calls
+ * that share a workspace must be ordered on one stream.
+ */
+int chai_decode_attention(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                          const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D,
+                          float scale, int dtype, void* workspace, size_t workspace_bytes, void* stream);
+size_t chai_decode_workspace_bytes(int B, int H, int k, int T, int D, int dtype);
+
+/*
+ * The same decode step with the per-step tensors in HOST memory: q_host [B,H,D] is
+ * copied to q_stage, the kernels run, out_stage is copied to out_host [B,H,D] and
+ * the call returns after the stream has drained.  q_stage / out_stage are device
+ * buffers of B*H*D elements owned by the caller; the caches stay device resident
+ * (they are state, not per-step input).  Pinned host memory makes the copies
+ * asynchronous; pageable memory works too.
+ */
+int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage, void* out_stage,
+                               const void* k_rep, const void* v, const int32_t* membership,
+                               const int32_t* reps, int B, int H, int k, int T, int T_cap, int D, float scale,
+                               int dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Clustered prefill attention over a whole prompt (same operator as decode with T
+ * query rows; decoder-only models attend causally, Section 2).
+ *   q [B,H,T,D] (only representative heads' rows are read), k_rep [B,k,T,D],
+ *   v [B,H,T,D], out [B,H,T,D];  causal != 0: row i sees keys j <= i.
+ * bf16 with D = 128 runs on the tcgen05 tensor-core kernel; fp32 (and D = 64) on
+ * the CUDA-core kernel, which chai_prefill_attention_simt selects for any dtype.
+ */
+int chai_prefill_attention(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                           const int32_t* reps, void* out, int B, int H, int k, int T, int D, float scale,
+                           int causal, int dtype, void* workspace, size_t workspace_bytes, void* stream);
+int chai_prefill_attention_simt(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                const int32_t* reps, void* out, int B, int H, int k, int T, int D,
+                                float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
+                                void* stream);
+size_t chai_prefill_workspace_bytes(int B, int H, int k, int T, int D, int dtype);
+
+/* Blocking read of the status word a decode/prefill call left in `workspace`
+ * (synchronises `stream`).  *status_out receives a chai_status_t. */
+int chai_device_status(const void* workspace, int* status_out, void* stream);
+
+const char* chai_status_string(int status);
+const char* chai_last_error(void); /* text of the last CHAI_ERR_CUDA / refusal on this thread */
+int chai_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CHAI_H_ */

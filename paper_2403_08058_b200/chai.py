@@ -1,0 +1,220 @@
+"""Thin ctypes binding of libchai.so: same names as include/chai.h, argument marshalling only.
+
+Torch supplies device memory and the current stream; every step of the path runs in the
+library's kernels.  There is no fallback: if the library has not been built (or cannot be
+loaded) the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libchai.so")
+
+CHAI_OK = 0
+CHAI_ERR_INVALID_ARG, CHAI_ERR_UNSUPPORTED, CHAI_ERR_WORKSPACE = 1, 2, 3
+CHAI_ERR_BAD_MEMBERSHIP, CHAI_ERR_TIMEOUT, CHAI_ERR_CUDA = 4, 5, 6
+CHAI_F32, CHAI_BF16 = 0, 1
+
+# every symbol include/chai.h declares
+EXPORTS = [
+    "chai_prefix_features", "chai_cluster_heads", "chai_compact_k_cache", "chai_decode_attention",
+    "chai_decode_workspace_bytes", "chai_decode_attention_host", "chai_prefill_attention",
+    "chai_prefill_attention_simt", "chai_prefill_workspace_bytes", "chai_device_status",
+    "chai_status_string", "chai_last_error", "chai_version",
+]
+
+_lib = None
+
+
+class ChaiError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__(f"libchai status {status}: {text}")
+        self.status = status
+
+
+def load() -> ctypes.CDLL:
+    """Load libchai.so from the package directory (raises if it has not been built)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2403_08058_b200.build` "
+                           "(there is no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, cf, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+    lib.chai_prefix_features.argtypes = [vp, vp, ci, ci, ci, ci, ci, cf, ci, vp, vp]
+    lib.chai_cluster_heads.argtypes = [vp, ci, ci, ci, ci, ci, ctypes.c_uint64, vp, vp, vp, vp, vp]
+    lib.chai_compact_k_cache.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp]
+    lib.chai_decode_attention.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp, sz, vp]
+    lib.chai_decode_attention_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci,
+                                               vp, sz, vp]
+    for name in ("chai_prefill_attention", "chai_prefill_attention_simt"):
+        getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
+    for name in ("chai_decode_workspace_bytes", "chai_prefill_workspace_bytes"):
+        getattr(lib, name).argtypes = [ci, ci, ci, ci, ci, ci]
+        getattr(lib, name).restype = sz
+    lib.chai_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
+    lib.chai_status_string.argtypes = [ci]
+    lib.chai_status_string.restype = ctypes.c_char_p
+    lib.chai_last_error.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _check(rc: int) -> None:
+    if rc != CHAI_OK:
+        lib = load()
+        text = lib.chai_last_error().decode() or lib.chai_status_string(rc).decode()
+        raise ChaiError(rc, text)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return CHAI_F32
+    if t.dtype == torch.bfloat16:
+        return CHAI_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _dev(*tensors) -> None:
+    for t in tensors:
+        if t is None:
+            continue
+        if not t.is_cuda or not t.is_contiguous():
+            raise ValueError("tensors must be contiguous CUDA tensors")
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def chai_version() -> int:
+    return int(load().chai_version())
+
+
+def chai_status_string(status: int) -> str:
+    return load().chai_status_string(int(status)).decode()
+
+
+def chai_decode_workspace_bytes(B, H, k, T, D, dtype) -> int:
+    return int(load().chai_decode_workspace_bytes(B, H, k, T, D, dtype))
+
+
+def chai_prefill_workspace_bytes(B, H, k, T, D, dtype) -> int:
+    return int(load().chai_prefill_workspace_bytes(B, H, k, T, D, dtype))
+
+
+def chai_prefix_features(q_full, k_full, P: int, scale: float, features=None):
+    """q_full, k_full [B,H,T_cap,D] -> features [B,H,P*P] fp32."""
+    _dev(q_full, k_full, features)
+    B, H, T_cap, D = q_full.shape
+    if features is None:
+        features = torch.empty((B, H, P * P), device=q_full.device, dtype=torch.float32)
+    _check(load().chai_prefix_features(_ptr(q_full), _ptr(k_full), B, H, T_cap, D, P, scale, _dt(q_full),
+                                       _ptr(features), _stream()))
+    return features
+
+
+def chai_cluster_heads(features, k: int, max_iter: int = 20, seed: int = 0, want_inertia: bool = True):
+    """features [B,H,F] fp32 -> (membership [B,H] i32, reps [B,k] i32, k_eff [B] i32, inertia [B] f64|None)."""
+    _dev(features)
+    if features.dtype != torch.float32:
+        raise TypeError("features must be float32")
+    B, H, F = features.shape
+    dev = features.device
+    membership = torch.empty((B, H), device=dev, dtype=torch.int32)
+    reps = torch.empty((B, k), device=dev, dtype=torch.int32)
+    k_eff = torch.empty((B,), device=dev, dtype=torch.int32)
+    inertia = torch.empty((B,), device=dev, dtype=torch.float64) if want_inertia else None
+    _check(load().chai_cluster_heads(_ptr(features), B, H, F, k, max_iter, seed, _ptr(membership), _ptr(reps),
+                                     _ptr(k_eff), _ptr(inertia), _stream()))
+    return membership, reps, k_eff, inertia
+
+
+def chai_compact_k_cache(k_full, reps, T: int | None = None, k_rep=None):
+    """k_full [B,H,T_cap,D], reps [B,k] -> k_rep [B,k,T_cap,D] (rows [0,T) of each slot are written)."""
+    _dev(k_full, reps, k_rep)
+    B, H, T_cap, D = k_full.shape
+    k = reps.shape[1]
+    T = T_cap if T is None else T
+    if k_rep is None:
+        k_rep = torch.empty((B, k, T_cap, D), device=k_full.device, dtype=k_full.dtype)
+    _check(load().chai_compact_k_cache(_ptr(k_full), _ptr(k_rep), _ptr(reps), B, H, k, T, T_cap, D, _dt(k_full),
+                                       _stream()))
+    return k_rep
+
+
+def new_workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty((max(int(nbytes), 256),), device=device, dtype=torch.uint8)
+
+
+def chai_decode_attention(q, k_rep, v, membership, reps, scale: float, T: int | None = None, out=None,
+                          workspace=None):
+    """q [B,H,D], k_rep [B,k,T_cap,D], v [B,H,T_cap,D], membership [B,H], reps [B,k] -> out [B,H,D]."""
+    _dev(q, k_rep, v, membership, reps, out, workspace)
+    B, H, D = q.shape
+    k, T_cap = k_rep.shape[1], k_rep.shape[2]
+    T = T_cap if T is None else T
+    dt = _dt(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(chai_decode_workspace_bytes(B, H, k, T, D, dt), q.device)
+    _check(load().chai_decode_attention(_ptr(q), _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps), _ptr(out), B,
+                                        H, k, T, T_cap, D, scale, dt, _ptr(workspace), workspace.numel(),
+                                        _stream()))
+    return out
+
+
+def chai_decode_attention_host(q_host, out_host, q_stage, out_stage, k_rep, v, membership, reps, scale: float,
+                               workspace, T: int | None = None):
+    """Decode step with q / out in (pinned) host memory; returns after the stream has drained."""
+    _dev(q_stage, out_stage, k_rep, v, membership, reps, workspace)
+    B, H, D = q_host.shape
+    k, T_cap = k_rep.shape[1], k_rep.shape[2]
+    T = T_cap if T is None else T
+    _check(load().chai_decode_attention_host(q_host.data_ptr(), out_host.data_ptr(), _ptr(q_stage),
+                                             _ptr(out_stage), _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps),
+                                             B, H, k, T, T_cap, D, scale, _dt(q_host), _ptr(workspace),
+                                             workspace.numel(), _stream()))
+    return out_host
+
+
+def _prefill(fn_name, q, k_rep, v, membership, reps, scale, causal, out, workspace):
+    _dev(q, k_rep, v, membership, reps, out, workspace)
+    B, H, T, D = q.shape
+    k = k_rep.shape[1]
+    dt = _dt(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(chai_prefill_workspace_bytes(B, H, k, T, D, dt), q.device)
+    _check(getattr(load(), fn_name)(_ptr(q), _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps), _ptr(out), B, H, k,
+                                    T, D, scale, int(bool(causal)), dt, _ptr(workspace), workspace.numel(),
+                                    _stream()))
+    return out
+
+
+def chai_prefill_attention(q, k_rep, v, membership, reps, scale: float, causal: bool = True, out=None,
+                           workspace=None):
+    """q [B,H,T,D], k_rep [B,k,T,D], v [B,H,T,D] -> out [B,H,T,D]."""
+    return _prefill("chai_prefill_attention", q, k_rep, v, membership, reps, scale, causal, out, workspace)
+
+
+def chai_prefill_attention_simt(q, k_rep, v, membership, reps, scale: float, causal: bool = True, out=None,
+                                workspace=None):
+    return _prefill("chai_prefill_attention_simt", q, k_rep, v, membership, reps, scale, causal, out, workspace)
+
+
+def chai_device_status(workspace) -> int:
+    st = ctypes.c_int(0)
+    _check(load().chai_device_status(_ptr(workspace), ctypes.byref(st), _stream()))
+    return int(st.value)

@@ -1,0 +1,116 @@
+// Shared host/device helpers of libchai: status plumbing, argument checks, dtype loads.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "chai.h"
+
+namespace chai {
+
+// The first 256 bytes of every workspace.  `status` is a chai_status_t; the other words say where
+// the first inconsistency was seen (debugging aid only).
+struct WsHeader {
+    int status;
+    int bad_b;
+    int bad_h;
+    int pad[61];
+};
+static_assert(sizeof(WsHeader) == 256, "workspace header is 256 bytes");
+
+void set_last_error(const char* fmt, ...);
+int cuda_fail(cudaError_t e, const char* what);  // records the text, returns CHAI_ERR_CUDA
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline size_t elem_size(int dtype) { return dtype == CHAI_BF16 ? 2 : 4; }
+
+#define CHAI_REQUIRE(cond, code, ...)            \
+    do {                                         \
+        if (!(cond)) {                           \
+            ::chai::set_last_error(__VA_ARGS__); \
+            return (code);                       \
+        }                                        \
+    } while (0)
+
+#define CHAI_LAUNCH_CHECK(what)                                   \
+    do {                                                          \
+        cudaError_t e__ = cudaGetLastError();                     \
+        if (e__ != cudaSuccess) return ::chai::cuda_fail(e__, what); \
+    } while (0)
+
+// ---- device helpers ---------------------------------------------------------------------------
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T>
+__device__ __forceinline__ T from_float(float x);
+template <>
+__device__ __forceinline__ float from_float<float>(float x) { return x; }
+template <>
+__device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// 16-byte vector of T unpacked to floats: 8 bf16 or 4 fp32.
+template <typename T>
+struct Vec16;
+template <>
+struct Vec16<float> {
+    static constexpr int N = 4;
+    __device__ __forceinline__ static void unpack(const uint4& r, float* f) {
+        f[0] = __uint_as_float(r.x);
+        f[1] = __uint_as_float(r.y);
+        f[2] = __uint_as_float(r.z);
+        f[3] = __uint_as_float(r.w);
+    }
+};
+template <>
+struct Vec16<__nv_bfloat16> {
+    static constexpr int N = 8;
+    // bf16 -> fp32 is a 16-bit shift
+    __device__ __forceinline__ static void unpack(const uint4& r, float* f) {
+        f[0] = __uint_as_float(r.x << 16);
+        f[1] = __uint_as_float(r.x & 0xffff0000u);
+        f[2] = __uint_as_float(r.y << 16);
+        f[3] = __uint_as_float(r.y & 0xffff0000u);
+        f[4] = __uint_as_float(r.z << 16);
+        f[5] = __uint_as_float(r.z & 0xffff0000u);
+        f[6] = __uint_as_float(r.w << 16);
+        f[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+};
+
+// Streaming 16-byte load that does not pollute L1 (cache data are read exactly once).
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+                 : "l"(p));
+    return r;
+}
+
+// Records the first data inconsistency a kernel meets; never traps.
+__device__ __forceinline__ void flag_bad_membership(WsHeader* hdr, int b, int h) {
+    if (atomicCAS(&hdr->status, CHAI_OK, CHAI_ERR_BAD_MEMBERSHIP) == CHAI_OK) {
+        hdr->bad_b = b;
+        hdr->bad_h = h;
+    }
+}
+
+// Resolves head h of request b to (cluster, representative); returns false (and flags) when the
+// membership data are inconsistent.  No address outside the arrays is formed.
+__device__ __forceinline__ bool resolve_head(const int32_t* membership, const int32_t* reps, int b, int h,
+                                             int H, int k, int* c_out, int* r_out) {
+    int c = membership[(size_t)b * H + h];
+    if (c < 0 || c >= k) return false;
+    int r = reps[(size_t)b * k + c];
+    if (r < 0 || r >= H) return false;
+    if (membership[(size_t)b * H + r] != c) return false;
+    *c_out = c;
+    *r_out = r;
+    return true;
+}
+
+}  // namespace chai

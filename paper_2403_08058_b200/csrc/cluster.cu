@@ -1,0 +1,252 @@
+// Membership identification: prefix score features and k-means over heads.
+//
+// Both kernels are tiny and latency-bound (one CTA per (request, head) resp. per request); there is
+// no roofline to chase.  The k-means kernel runs in fp64 with explicitly rounded operations in a
+// fixed order, so its trajectory does not depend on the launch shape or on compiler contraction.
+#include "chai_common.cuh"
+
+namespace chai {
+
+// ---- prefix score features (Section 3.3; similarity is defined on softmax(Q K^T), Section 3.1) ----
+// grid (H, B), block P*P threads: thread (i,j) computes the scaled dot product of query i and key j
+// of its own head, then thread (i,0) normalises row i causally.
+template <typename T>
+__global__ void prefix_features_kernel(const T* __restrict__ q_full, const T* __restrict__ k_full,
+                                       float* __restrict__ features, int H, int T_cap, int D, int P,
+                                       float scale) {
+    extern __shared__ float s_scores[];  // [P*P]
+    const int h = blockIdx.x, b = blockIdx.y;
+    const int i = threadIdx.x / P, j = threadIdx.x % P;
+    const size_t head = ((size_t)b * H + h) * (size_t)T_cap * D;
+    if (j <= i) {
+        const T* q = q_full + head + (size_t)i * D;
+        const T* kk = k_full + head + (size_t)j * D;
+        float s = 0.f;
+        for (int d = 0; d < D; ++d) s = fmaf(to_float(q[d]), to_float(kk[d]), s);
+        s_scores[i * P + j] = s * scale;
+    }
+    __syncthreads();
+    if (j == 0) {
+        float m = -INFINITY;
+        for (int jj = 0; jj <= i; ++jj) m = fmaxf(m, s_scores[i * P + jj]);
+        float z = 0.f;
+        for (int jj = 0; jj <= i; ++jj) {
+            float p = expf(s_scores[i * P + jj] - m);
+            s_scores[i * P + jj] = p;
+            z += p;
+        }
+        float* f = features + ((size_t)b * H + h) * (size_t)P * P + (size_t)i * P;
+        for (int jj = 0; jj < P; ++jj) f[jj] = jj <= i ? s_scores[i * P + jj] / z : 0.f;
+    }
+}
+
+// ---- k-means (Section 3.5; objective of Section 3.2) ------------------------------------------------
+__device__ __forceinline__ double sqdist(const double* x, const double* y, int F) {
+    double s = 0.0;
+    for (int f = 0; f < F; ++f) {
+        double d = __dsub_rn(x[f], y[f]);
+        s = __dadd_rn(s, __dmul_rn(d, d));
+    }
+    return s;
+}
+
+// One CTA per request.  Shared memory: X [H,F], C [k,F], dist [H,k] doubles; a, prev, count ints.
+__global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ features, int H, int F, int k,
+                                                     int max_iter, unsigned long long seed,
+                                                     int32_t* __restrict__ membership, int32_t* __restrict__ reps,
+                                                     int32_t* __restrict__ k_eff, double* __restrict__ inertia) {
+    extern __shared__ double smem_d[];
+    double* X = smem_d;
+    double* C = X + (size_t)H * F;
+    double* dist = C + (size_t)k * F;  // [H,k]; its first H entries double as dmin during initialisation
+    int* a = reinterpret_cast<int*>(dist + (size_t)H * k);
+    int* prev = a + H;
+    int* count = prev + H;
+    int* newid = count + k;
+    __shared__ int s_far, s_ncentres, s_same;
+
+    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+    const float* xin = features + (size_t)b * H * F;
+    for (int i = tid; i < H * F; i += nt) X[i] = (double)xin[i];
+    __syncthreads();
+
+    // farthest-first traversal: first centre = head (seed mod H)
+    const int first = (int)(seed % (unsigned long long)H);
+    for (int f = tid; f < F; f += nt) C[f] = X[(size_t)first * F + f];
+    if (tid == 0) s_ncentres = 1;
+    __syncthreads();
+    double* dmin = dist;
+    for (int h = tid; h < H; h += nt) dmin[h] = sqdist(X + (size_t)h * F, C, F);
+    __syncthreads();
+    for (int n = 1; n < k; ++n) {
+        if (tid == 0) {
+            int far = 0;
+            for (int h = 1; h < H; ++h)
+                if (dmin[h] > dmin[far]) far = h;
+            s_far = dmin[far] == 0.0 ? -1 : far;
+        }
+        __syncthreads();
+        const int far = s_far;
+        if (far < 0) break;  // uniform: every thread reads the same shared value
+        double* cn = C + (size_t)n * F;
+        for (int f = tid; f < F; f += nt) cn[f] = X[(size_t)far * F + f];
+        if (tid == 0) s_ncentres = n + 1;
+        __syncthreads();
+        for (int h = tid; h < H; h += nt) {
+            double d = sqdist(X + (size_t)h * F, cn, F);
+            if (d < dmin[h]) dmin[h] = d;
+        }
+        __syncthreads();
+    }
+    __syncthreads();
+    const int nc = s_ncentres;
+
+    // Lloyd iterations
+    for (int it = 0; it < max_iter; ++it) {
+        for (int p = tid; p < H * nc; p += nt) {
+            int h = p / nc, c = p % nc;
+            dist[(size_t)h * k + c] = sqdist(X + (size_t)h * F, C + (size_t)c * F, F);
+        }
+        if (tid == 0) s_same = 1;
+        __syncthreads();
+        for (int h = tid; h < H; h += nt) {
+            int best = 0;
+            double bd = dist[(size_t)h * k];
+            for (int c = 1; c < nc; ++c) {
+                double d = dist[(size_t)h * k + c];
+                if (d < bd) {
+                    bd = d;
+                    best = c;
+                }
+            }
+            a[h] = best;
+            if (it == 0 || best != prev[h]) s_same = 0;  // benign race: every writer stores 0
+        }
+        __syncthreads();
+        if (s_same) break;
+        for (int h = tid; h < H; h += nt) prev[h] = a[h];
+        for (int c = tid; c < nc; c += nt) {
+            int n = 0;
+            for (int h = 0; h < H; ++h) n += (a[h] == c);
+            count[c] = n;
+        }
+        __syncthreads();
+        for (int p = tid; p < nc * F; p += nt) {
+            int c = p / F, f = p % F;
+            if (count[c] == 0) continue;  // an empty cluster keeps its centre
+            double s = 0.0;
+            for (int h = 0; h < H; ++h)
+                if (a[h] == c) s = __dadd_rn(s, X[(size_t)h * F + f]);
+            C[(size_t)c * F + f] = __ddiv_rn(s, (double)count[c]);
+        }
+        __syncthreads();
+    }
+    __syncthreads();
+
+    // canonical labels: clusters ordered by their lowest member; representative = lowest member
+    if (tid == 0) {
+        for (int c = 0; c < k; ++c) {
+            newid[c] = -1;
+            reps[(size_t)b * k + c] = -1;
+        }
+        int next = 0;
+        for (int h = 0; h < H; ++h) {
+            if (newid[a[h]] < 0) {
+                newid[a[h]] = next;
+                reps[(size_t)b * k + next] = h;
+                ++next;
+            }
+        }
+        k_eff[b] = next;
+        s_ncentres = next;
+    }
+    __syncthreads();
+    for (int h = tid; h < H; h += nt) {
+        a[h] = newid[a[h]];
+        membership[(size_t)b * H + h] = a[h];
+    }
+    if (inertia == nullptr) return;
+    __syncthreads();
+
+    // inertia against the final members' means, summed in (cluster, head) order
+    const int ke = s_ncentres;
+    for (int c = tid; c < ke; c += nt) {
+        int n = 0;
+        for (int h = 0; h < H; ++h) n += (a[h] == c);
+        count[c] = n;
+    }
+    __syncthreads();
+    for (int p = tid; p < ke * F; p += nt) {
+        int c = p / F, f = p % F;
+        double s = 0.0;
+        for (int h = 0; h < H; ++h)
+            if (a[h] == c) s = __dadd_rn(s, X[(size_t)h * F + f]);
+        C[(size_t)c * F + f] = __ddiv_rn(s, (double)count[c]);
+    }
+    __syncthreads();
+    for (int h = tid; h < H; h += nt) dist[h] = sqdist(X + (size_t)h * F, C + (size_t)a[h] * F, F);
+    __syncthreads();
+    if (tid == 0) {
+        double total = 0.0;
+        for (int c = 0; c < ke; ++c)
+            for (int h = 0; h < H; ++h)
+                if (a[h] == c) total = __dadd_rn(total, dist[h]);
+        inertia[b] = total;
+    }
+}
+
+static size_t kmeans_smem_bytes(int H, int F, int k) {
+    return sizeof(double) * ((size_t)H * F + (size_t)k * F + (size_t)H * k) + sizeof(int) * (2 * (size_t)H + 2 * (size_t)k);
+}
+
+}  // namespace chai
+
+extern "C" {
+
+int chai_prefix_features(const void* q_full, const void* k_full, int B, int H, int T_cap, int D, int P,
+                         float scale, int dtype, float* features, void* stream) {
+    using namespace chai;
+    CHAI_REQUIRE(q_full && k_full && features, CHAI_ERR_INVALID_ARG, "chai_prefix_features: null pointer");
+    CHAI_REQUIRE(aligned16(q_full) && aligned16(k_full), CHAI_ERR_INVALID_ARG,
+                 "chai_prefix_features: pointers must be 16-byte aligned");
+    CHAI_REQUIRE(B > 0 && H > 0 && T_cap > 0 && D > 0 && P > 0, CHAI_ERR_INVALID_ARG,
+                 "chai_prefix_features: sizes must be positive");
+    CHAI_REQUIRE(P <= T_cap, CHAI_ERR_INVALID_ARG, "chai_prefix_features: P=%d exceeds T_cap=%d", P, T_cap);
+    CHAI_REQUIRE(P <= 32 && B <= 65535, CHAI_ERR_UNSUPPORTED, "chai_prefix_features: P <= 32 and B <= 65535");
+    CHAI_REQUIRE(dtype == CHAI_F32 || dtype == CHAI_BF16, CHAI_ERR_UNSUPPORTED, "chai_prefix_features: dtype");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    dim3 grid(H, B), block(P * P);
+    size_t smem = sizeof(float) * P * P;
+    if (dtype == CHAI_BF16)
+        prefix_features_kernel<__nv_bfloat16><<<grid, block, smem, s>>>(
+            static_cast<const __nv_bfloat16*>(q_full), static_cast<const __nv_bfloat16*>(k_full), features, H,
+            T_cap, D, P, scale);
+    else
+        prefix_features_kernel<float><<<grid, block, smem, s>>>(static_cast<const float*>(q_full),
+                                                               static_cast<const float*>(k_full), features, H,
+                                                               T_cap, D, P, scale);
+    CHAI_LAUNCH_CHECK("prefix_features_kernel launch");
+    return CHAI_OK;
+}
+
+int chai_cluster_heads(const float* features, int B, int H, int F, int k, int max_iter, uint64_t seed,
+                       int32_t* membership, int32_t* reps, int32_t* k_eff, double* inertia, void* stream) {
+    using namespace chai;
+    CHAI_REQUIRE(features && membership && reps && k_eff, CHAI_ERR_INVALID_ARG,
+                 "chai_cluster_heads: null pointer");
+    CHAI_REQUIRE(B > 0 && H > 0 && F > 0 && max_iter > 0, CHAI_ERR_INVALID_ARG,
+                 "chai_cluster_heads: sizes must be positive");
+    CHAI_REQUIRE(k >= 1 && k <= H, CHAI_ERR_INVALID_ARG, "chai_cluster_heads: need 1 <= k <= H (k=%d, H=%d)", k, H);
+    size_t smem = kmeans_smem_bytes(H, F, k);
+    CHAI_REQUIRE(H <= 1024 && smem <= 200 * 1024, CHAI_ERR_UNSUPPORTED,
+                 "chai_cluster_heads: problem needs %zu bytes of shared memory (limit 204800)", smem);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaFuncSetAttribute(kmeans_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e, "kmeans_kernel shared-memory opt-in");
+    kmeans_kernel<<<B, 256, smem, s>>>(features, H, F, k, max_iter, (unsigned long long)seed, membership, reps,
+                                       k_eff, inertia);
+    CHAI_LAUNCH_CHECK("kmeans_kernel launch");
+    return CHAI_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,347 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same bits."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import chai_oracle as orc
+from paper_2403_08058_b200 import chai, synth
+from parity import assert_parity, errors, gate_ok
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def to_dev(case, names=("q", "k_rep", "v", "membership", "reps", "k_full", "q_full")):
+    return {n: (case[n].to(DEV) if n in case and torch.is_tensor(case[n]) else case.get(n)) for n in names}
+
+
+def oracle_decode(case, T=None):
+    T = T or case["T"]
+    return orc.cha_attention(case["q"], case["k_rep"][:, :, :T], case["v"][:, :, :T], case["membership"],
+                             case["reps"], case["scale"], causal=False)
+
+
+def run_decode(case, T=None, **kw):
+    d = to_dev(case)
+    out = chai.chai_decode_attention(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"],
+                                     T=T or case["T"], **kw)
+    torch.cuda.synchronize()
+    return out.float().cpu().numpy()
+
+
+# ---- decode ---------------------------------------------------------------------------------------
+
+def test_decode_config1_fp32():
+    case = synth.decode_layer(1)
+    got = run_decode(case)
+    e = assert_parity(got, oracle_decode(case), "f32", "config 1 decode")
+    assert e["max_rel"] <= 1e-5
+
+
+@pytest.mark.parametrize("T", [1, 2, 5, 127, 128, 129, 255, 256, 257, 700])
+@pytest.mark.parametrize("cfg", [1, 2, 3])
+def test_decode_ragged_lengths(cfg, T):
+    """Lengths around the 64/128/256-row chunk edges, capacity larger than the length."""
+    case = synth.decode_layer(cfg, layer=T % 7, seed=T, B=2, H=12 if cfg != 1 else 8, T=T, T_cap=T + 3, k=3)
+    got = run_decode(case)
+    assert_parity(got, oracle_decode(case), case["dtype"], f"cfg {cfg} T {T}")
+
+
+@pytest.mark.parametrize("cfg,D,H,k", [(2, 64, 8, 2), (1, 64, 6, 6), (2, 128, 52, 13), (3, 128, 72, 36),
+                                       (3, 128, 9, 1)])
+def test_decode_shapes(cfg, D, H, k):
+    case = synth.decode_layer(cfg, seed=5, B=3, H=H, T=300, k=k)
+    if D == 64:
+        for n in ("q", "k_rep", "v"):
+            case[n] = case[n][..., :64].contiguous()
+        case["scale"] = 0.125
+    got = run_decode(case)
+    assert_parity(got, oracle_decode(case), case["dtype"], f"cfg {cfg} D {D} H {H} k {k}")
+
+
+@pytest.mark.parametrize("cfg", [2, 3])
+def test_decode_peaked_and_negative_controls(cfg):
+    """A peaked softmax gives the gate power; wrong membership / reps / K slots must fail it."""
+    case = synth.decode_layer(cfg, seed=3, B=2, H=16, T=1024, k=4, peaked=8.0)
+    ref = oracle_decode(case)
+    got = run_decode(case)
+    assert_parity(got, ref, "bf16", "peaked decode")
+    # shuffled membership (still a consistent partition, but the wrong one)
+    wrong = dict(case)
+    perm = torch.roll(torch.arange(16), 5)
+    mem = case["membership"][:, perm].contiguous()
+    labels = [synth.canonical_labels(m.numpy()) for m in mem]
+    wrong["membership"] = torch.as_tensor(np.stack([l[0] for l in labels]))
+    wrong["reps"] = torch.as_tensor(np.stack([l[1] for l in labels]))
+    assert not gate_ok(run_decode(wrong), ref, "bf16")
+    # K slots swapped
+    wrong = dict(case)
+    wrong["k_rep"] = case["k_rep"][:, [1, 0, 2, 3]].contiguous()
+    assert not gate_ok(run_decode(wrong), ref, "bf16")
+    # the oracle itself distinguishes them too
+    assert not gate_ok(oracle_decode(wrong), ref, "bf16")
+
+
+def test_decode_full_size_layers():
+    """One layer of each decode workload at full size, every output element against the oracle
+    (the oracle is cheap for a single query row), in the launch configuration the bench uses."""
+    for cfg, layer in ((2, 0), (2, 3), (3, 1), (4, 2)):
+        case = synth.decode_layer(cfg, layer=layer, seed=0, device=DEV, with_k_full=False)
+        ws = chai.new_workspace(chai.chai_decode_workspace_bytes(case["B"], case["H"], case["k"], case["T"], 128,
+                                                                 chai.CHAI_BF16), DEV)
+        out = chai.chai_decode_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"],
+                                         case["scale"], workspace=ws)
+        out2 = chai.chai_decode_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"],
+                                          case["scale"], workspace=ws)
+        torch.cuda.synchronize()
+        assert chai.chai_device_status(ws) == chai.CHAI_OK
+        assert torch.equal(out, out2)                      # run-to-run bitwise identical
+        got = out.float().cpu().numpy()
+        for b in range(case["B"]):
+            sl = {n: case[n][b:b + 1].cpu() for n in ("q", "k_rep", "v", "membership", "reps")}
+            ref = orc.cha_attention(sl["q"], sl["k_rep"], sl["v"], sl["membership"], sl["reps"], case["scale"],
+                                    causal=False)
+            assert_parity(got[b:b + 1], ref, "bf16", f"cfg {cfg} layer {layer} b {b}")
+        del case, out, out2, ws
+        torch.cuda.empty_cache()
+
+
+def test_decode_bad_membership_is_reported_not_faulted():
+    case = synth.decode_layer(2, seed=1, B=2, H=8, T=200, k=4)
+    ref = oracle_decode(case)
+    d = to_dev(case)
+    ws = chai.new_workspace(chai.chai_decode_workspace_bytes(2, 8, 4, 200, 128, chai.CHAI_BF16), DEV)
+    canary = torch.full((2, 8, 128), 7.0, device=DEV, dtype=torch.bfloat16)
+
+    def run(mem, reps):
+        out = canary.clone()
+        chai.chai_decode_attention(d["q"], d["k_rep"], d["v"], mem, reps, case["scale"], out=out, workspace=ws)
+        return out.float().cpu().numpy(), chai.chai_device_status(ws)
+
+    got, st = run(d["membership"], d["reps"])
+    assert st == chai.CHAI_OK and gate_ok(got, ref, "bf16")
+    # cluster id out of range for one head
+    mem = d["membership"].clone()
+    mem[1, 5] = 99
+    got, st = run(mem, d["reps"])
+    assert st == chai.CHAI_ERR_BAD_MEMBERSHIP
+    # head 5 of request 1 is zero; heads that did not depend on it are untouched
+    assert not got[1, 5].any()
+    assert gate_ok(got[0], ref[0], "bf16")
+    # a cluster without representative: its members get zeros
+    reps = d["reps"].clone()
+    reps[0, 2] = -1
+    got, st = run(d["membership"], reps)
+    assert st == chai.CHAI_ERR_BAD_MEMBERSHIP
+    dead = (case["membership"][0] == 2).numpy()
+    assert not got[0, dead].any() and gate_ok(got[0, ~dead], ref[0, ~dead], "bf16")
+    # representative outside its own cluster
+    reps = d["reps"].clone()
+    reps[0, 1] = int(case["reps"][0, 0])
+    got, st = run(d["membership"], reps)
+    assert st == chai.CHAI_ERR_BAD_MEMBERSHIP
+    # and a good call afterwards clears the word
+    got, st = run(d["membership"], d["reps"])
+    assert st == chai.CHAI_OK and gate_ok(got, ref, "bf16")
+
+
+def test_decode_host_entry_point():
+    case = synth.decode_layer(2, seed=2, B=2, H=8, T=300, k=4)
+    d = to_dev(case)
+    ws = chai.new_workspace(chai.chai_decode_workspace_bytes(2, 8, 4, 300, 128, chai.CHAI_BF16), DEV)
+    qh = case["q"].pin_memory()
+    oh = torch.empty_like(case["q"]).pin_memory()
+    chai.chai_decode_attention_host(qh, oh, torch.empty_like(d["q"]), torch.empty_like(d["q"]), d["k_rep"], d["v"],
+                                    d["membership"], d["reps"], case["scale"], ws)
+    assert_parity(oh.float().numpy(), oracle_decode(case), "bf16", "host entry")
+
+
+# ---- k-means, features, compaction ---------------------------------------------------------------------
+
+def gpu_kmeans(x, k, max_iter=20, seed=0):
+    mem, reps, ke, inertia = chai.chai_cluster_heads(torch.as_tensor(x, device=DEV), k, max_iter, seed)
+    torch.cuda.synchronize()
+    return mem.cpu().numpy(), reps.cpu().numpy(), ke.cpu().numpy(), inertia.cpu().numpy()
+
+
+def test_kmeans_config1_blobs_every_seed():
+    x, planted, planted_reps = synth.blob_features(1, 32, 64, 8, seed=0)
+    for seed in range(32):
+        mem, reps, ke, inertia = gpu_kmeans(x, 8, 20, seed)
+        ref = orc.kmeans(x, 8, 20, seed)
+        assert np.array_equal(mem, planted) and np.array_equal(mem, ref["membership"])
+        assert np.array_equal(reps, planted_reps) and ke[0] == 8
+        assert inertia[0] == ref["inertia"][0]
+
+
+def test_kmeans_identical_trajectories_on_unstructured_inputs():
+    """Same arithmetic in the same order: labels agree bit for bit even where nothing is separated."""
+    r = np.random.default_rng(0)
+    for trial in range(25):
+        B, H, F = 3, int(r.integers(2, 80)), int(r.integers(1, 70))
+        k = int(r.integers(1, H + 1))
+        x = r.standard_normal((B, H, F)).astype(np.float32)
+        it = int(r.integers(1, 30))
+        mem, reps, ke, inertia = gpu_kmeans(x, k, it, trial)
+        ref = orc.kmeans(x, k, it, trial)
+        assert np.array_equal(mem, ref["membership"]), trial
+        assert np.array_equal(reps, ref["reps"]) and np.array_equal(ke, ref["k_eff"])
+        np.testing.assert_array_equal(inertia, ref["inertia"])
+
+
+def test_kmeans_degenerate_inputs():
+    r = np.random.default_rng(4)
+    y = np.repeat(r.standard_normal((1, 3, 5)), 3, axis=1).astype(np.float32)     # 3 distinct points x3
+    mem, reps, ke, _ = gpu_kmeans(y, 5, 20, 1)
+    ref = orc.kmeans(y, 5, 20, 1)
+    assert ke[0] == 3 and np.array_equal(mem, ref["membership"]) and np.array_equal(reps, ref["reps"])
+    mem, reps, ke, inertia = gpu_kmeans(np.ones((2, 6, 2), np.float32), 4, 20, 3)
+    assert (ke == 1).all() and not mem.any() and (reps[:, 1:] == -1).all() and np.isfinite(inertia).all()
+    x = r.standard_normal((1, 72, 25)).astype(np.float32)
+    mem, reps, ke, _ = gpu_kmeans(x, 72, 20, 0)                                  # k = H
+    assert mem[0].tolist() == list(range(72))
+    mem, _, _, _ = gpu_kmeans(x, 1, 20, 0)
+    assert not mem.any()
+
+
+def test_prefix_features():
+    for dtype, tol in ((torch.float32, 2e-6), (torch.bfloat16, 2e-6)):
+        g = torch.Generator().manual_seed(3)
+        q = torch.randn(2, 5, 9, 128, generator=g).to(dtype)
+        k = torch.randn(2, 5, 9, 128, generator=g).to(dtype)
+        for P in (1, 5, 8):
+            f = chai.chai_prefix_features(q.to(DEV), k.to(DEV), P, 0.09).cpu().numpy()
+            ref = orc.prefix_features(q, k, P, 0.09)
+            assert np.abs(f - ref).max() <= tol
+            assert not np.triu(f.reshape(2, 5, P, P), 1).any()
+
+
+def test_compaction_bit_exact():
+    for dtype in (torch.bfloat16, torch.float32):
+        B, H, k, T, T_cap, D = 3, 10, 4, 333, 340, 128
+        g = torch.Generator().manual_seed(1)
+        kf = torch.randn(B, H, T_cap, D, generator=g).to(dtype)
+        _, reps = synth.batch_partitions(B, H, k, "uneven", 4, 4)
+        reps[2, 3] = -1
+        out = torch.full((B, k, T_cap, D), 3.0, dtype=dtype, device=DEV)
+        chai.chai_compact_k_cache(kf.to(DEV), torch.as_tensor(reps, device=DEV), T=T, k_rep=out)
+        out = out.cpu()
+        bits = kf.view(torch.int16 if dtype == torch.bfloat16 else torch.int32).numpy()
+        want, _ = orc.compact_k_cache(np.ascontiguousarray(bits[:, :, :T]), reps)
+        got = out.view(torch.int16 if dtype == torch.bfloat16 else torch.int32).numpy()
+        assert np.array_equal(got[:, :, :T], want)
+        assert (out[:, :, T:] == 3.0).all()              # rows beyond T are not written
+        assert not got[2, 3, :T].any()
+
+
+# ---- prefill --------------------------------------------------------------------------------------------
+
+def prefill_inputs(seed, B, H, T, k, dtype="bf16", kind="uneven", peaked=1.0, D=128):
+    r = synth.batch_partitions(B, H, k, kind, seed, 77, T)
+    g = torch.Generator().manual_seed(seed)
+    td = synth.TORCH_DTYPE[dtype]
+    sigma = 0.5 if dtype == "bf16" else 1.0
+    q = (torch.randn(B, H, T, D, generator=g) * sigma * peaked).to(td)
+    kr = (torch.randn(B, k, T, D, generator=g) * sigma).to(td)
+    v = (torch.randn(B, H, T, D, generator=g) * sigma).to(td)
+    return dict(q=q, k_rep=kr, v=v, membership=torch.as_tensor(r[0]), reps=torch.as_tensor(r[1]),
+                scale=1.0 / np.sqrt(D), dtype=dtype)
+
+
+def run_prefill(case, causal=True, fn=None):
+    fn = fn or chai.chai_prefill_attention
+    d = to_dev(case)
+    out = fn(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"], causal)
+    torch.cuda.synchronize()
+    return out.float().cpu().numpy()
+
+
+@pytest.mark.parametrize("fn_name", ["chai_prefill_attention", "chai_prefill_attention_simt"])
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("T", [1, 5, 31, 33, 64, 100, 128, 129, 200, 257, 300])
+def test_prefill_ragged_lengths(fn_name, dtype, T):
+    case = prefill_inputs(T, 2, 7, T, 3, dtype, peaked=4.0)
+    for causal in (True, False):
+        got = run_prefill(case, causal, getattr(chai, fn_name))
+        ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"],
+                                case["scale"], causal)
+        assert_parity(got, ref, dtype, f"{fn_name} {dtype} T {T} causal {causal}")
+
+
+@pytest.mark.parametrize("H,k,kind", [(8, 8, "even"), (8, 1, "even"), (12, 3, "even"), (16, 2, "uneven"),
+                                      (52, 13, "uneven"), (9, 4, "uneven")])
+def test_prefill_cluster_shapes(H, k, kind):
+    """Singletons (plain MHA), one cluster of everything, groups of 1..many members."""
+    case = prefill_inputs(H * k, 1, H, 160, k, "bf16", kind, peaked=4.0)
+    got = run_prefill(case)
+    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], True)
+    assert_parity(got, ref, "bf16", f"H {H} k {k}")
+
+
+def test_prefill_head_dim_64():
+    case = prefill_inputs(9, 2, 6, 150, 2, "bf16", D=64, peaked=4.0)
+    got = run_prefill(case)
+    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], True)
+    assert_parity(got, ref, "bf16", "D 64")
+
+
+def test_prefill_negative_controls_and_bad_membership():
+    case = prefill_inputs(2, 1, 8, 256, 4, "bf16", "even", peaked=8.0)
+    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], True)
+    assert gate_ok(run_prefill(case), ref, "bf16")
+    wrong = dict(case)
+    wrong["k_rep"] = case["k_rep"][:, [1, 0, 2, 3]].contiguous()
+    assert not gate_ok(run_prefill(wrong), ref, "bf16")
+    # invalid cluster id on a non-representative head: reported, zero rows, other heads intact
+    d = to_dev(case)
+    hbad = [h for h in range(8) if h not in case["reps"][0].tolist()][0]
+    mem = d["membership"].clone()
+    mem[0, hbad] = -5
+    ws = chai.new_workspace(chai.chai_prefill_workspace_bytes(1, 8, 4, 256, 128, chai.CHAI_BF16), DEV)
+    out = torch.full_like(d["q"], 7.0)
+    chai.chai_prefill_attention(d["q"], d["k_rep"], d["v"], mem, d["reps"], case["scale"], True, out=out, workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_ERR_BAD_MEMBERSHIP
+    got = out.float().cpu().numpy()
+    assert not got[0, hbad].any()
+    keep = np.arange(8) != hbad
+    assert gate_ok(got[0, keep], ref[0, keep], "bf16")
+
+
+def test_prefill_full_size_sampled_rows():
+    """Workload 5 at full size: the first 192 rows and the last 64 rows of every request and head
+    (causal attention of the first rows depends only on the first keys; the last rows see everything)."""
+    case = synth.prefill_case(seed=0, device=DEV)
+    k_rep = chai.chai_compact_k_cache(case["k_full"], case["reps"])
+    out = chai.chai_prefill_attention(case["q_full"], k_rep, case["v"], case["membership"], case["reps"], case["scale"])
+    out2 = chai.chai_prefill_attention(case["q_full"], k_rep, case["v"], case["membership"], case["reps"], case["scale"])
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    T = case["T"]
+    q, kr, v = case["q_full"].cpu(), k_rep.cpu(), case["v"].cpu()
+    mem, reps = case["membership"].cpu(), case["reps"].cpu()
+    head = orc.cha_attention(q[:, :, :192], kr[:, :, :192], v[:, :, :192], mem, reps, case["scale"], True)
+    assert_parity(out[:, :, :192].float().cpu().numpy(), head, "bf16", "first rows")
+    tail = orc.cha_attention(q[:, :, T - 64:], kr, v, mem, reps, case["scale"], True)
+    assert_parity(out[:, :, T - 64:].float().cpu().numpy(), tail, "bf16", "last rows")
+
+
+def test_prefill_flow_features_kmeans_compaction_attention():
+    """Workload 5's whole flow at reduced length: both sides derive the membership themselves."""
+    case = synth.prefill_case(seed=1, B=2, T=192, peaked=4.0)
+    d = to_dev(case, ("q_full", "k_full", "v"))
+    feats = chai.chai_prefix_features(d["q_full"], d["k_full"], 5, case["scale"])
+    mem, reps, ke, _ = chai.chai_cluster_heads(feats, case["k"], 20, 0)
+    k_rep = chai.chai_compact_k_cache(d["k_full"], reps)
+    out = chai.chai_prefill_attention(d["q_full"], k_rep, d["v"], mem, reps, case["scale"])
+    torch.cuda.synchronize()
+    o_feats = orc.prefix_features(case["q_full"], case["k_full"], 5, case["scale"])
+    o_km = orc.kmeans(o_feats.astype(np.float32), case["k"], 20, 0)
+    assert np.array_equal(mem.cpu().numpy(), o_km["membership"])          # bit-exact as a partition
+    assert np.array_equal(mem.cpu().numpy(), case["planted"])
+    assert np.array_equal(reps.cpu().numpy(), o_km["reps"])
+    bits = case["k_full"].view(torch.int16).numpy()
+    o_krep, _ = orc.compact_k_cache(bits, o_km["reps"])
+    assert np.array_equal(k_rep.cpu().view(torch.int16).numpy(), o_krep)
+    ref = orc.cha_attention(case["q_full"], torch.from_numpy(o_krep).view(torch.bfloat16), case["v"],
+                            o_km["membership"], o_km["reps"], case["scale"], True)
+    assert_parity(out.float().cpu().numpy(), ref, "bf16", "flow")
