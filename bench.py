@@ -183,7 +183,7 @@ def cpu_baseline_decode(cfg_id: int, seed: int, budget_s: float = 12.0):
         c = synth.decode_layer(cfg_id, layer, seed, device="cpu", B=2, with_k_full=False)
         args = [orc._f64(c[n]) for n in ("q", "k_rep", "v")]
         reps_run = 0
-        while reps_run < 8 and spent < budget_s:
+        while reps_run < 40 and spent < budget_s:
             t0 = time.perf_counter()
             orc.cha_attention(args[0], args[1], args[2], c["membership"], c["reps"], c["scale"], causal=False)
             spent += time.perf_counter() - t0
@@ -192,7 +192,7 @@ def cpu_baseline_decode(cfg_id: int, seed: int, budget_s: float = 12.0):
             reps_run += 1
         layer += 1
     return dict(value=nbytes / spent / 1e9, unit=UNIT, cores=orc.num_threads(), kind="oracle",
-                sample=f"first {layer} layers x 2 requests of workload {cfg_id}, each up to 8 times ({n_req} request-layers, "
+                sample=f"first {layer} layers x 2 requests of workload {cfg_id}, each up to 40 times ({n_req} request-layers, "
                        f"{spent:.1f} s of oracle time, inputs already widened to fp64)", seconds=spent)
 
 
