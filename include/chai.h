@@ -55,6 +55,9 @@ typedef enum {
 
 typedef enum { CHAI_F32 = 0, CHAI_BF16 = 1 } chai_dtype_t;
 
+/* size of the built-in scratch array used by chai_decode_attention_static */
+#define CHAI_DECODE_STATIC_SCRATCH_BYTES (8u << 20)
+
 /*
  * Prefix score features (Section 3.3 and Fig. 6(b): the first five tokens of a
  * request run with plain multi-head attention and their attention scores are what
@@ -123,6 +126,30 @@ int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage
                                const void* k_rep, const void* v, const int32_t* membership,
                                const int32_t* reps, int B, int H, int k, int T, int T_cap, int D, float scale,
                                int dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Decode step for callers that can neither pass a workspace nor let the library allocate one
+ * (no counterpart in the paper: this is a deployment convenience).  Typical cases: a serving
+ * engine that has already handed every free byte of HBM to its KV-cache pool, so a later
+ * allocation would fail, and a latency-critical loop where the implicit device synchronisation
+ * of an allocation is not acceptable.  Same arguments and result as chai_decode_attention, minus
+ * the workspace: the scratch lives in an array of CHAI_DECODE_STATIC_SCRATCH_BYTES (8 MiB) that
+ * is part of the library image, resident on every GPU that loads the library until the
+ * process exits.  The call allocates nothing (no cudaMalloc / cudaFree, no allocating library
+ * routine).
+ *   - A problem whose scratch (chai_decode_workspace_bytes) exceeds the array is refused with
+ *     CHAI_ERR_WORKSPACE and a message that states both sizes.
+ *   - The first call on each device looks up the array's device address (the device that is
+ *     current at the time of the call); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which still holds whatever the previous call left;
+ *     the kernels clear the parts that must start at zero.  Two calls that can overlap on the GPU
+ *     (different streams without ordering) race on it: order them, or use chai_decode_attention
+ *     with separate workspaces.  The status word of the last call is not readable through this
+ *     entry point; inconsistent membership still yields zero rows and never faults.
+ */
+int chai_decode_attention_static(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                 const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D,
+                                 float scale, int dtype, void* stream);
 
 /*
  * Clustered prefill attention over a whole prompt (same operator as decode with T

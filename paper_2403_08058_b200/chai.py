@@ -24,8 +24,9 @@ EXPORTS = [
     "chai_prefix_features", "chai_cluster_heads", "chai_compact_k_cache", "chai_decode_attention",
     "chai_decode_workspace_bytes", "chai_decode_attention_host", "chai_prefill_attention",
     "chai_prefill_attention_simt", "chai_prefill_workspace_bytes", "chai_device_status",
-    "chai_status_string", "chai_last_error", "chai_version",
+    "chai_status_string", "chai_last_error", "chai_version", "chai_decode_attention_static",
 ]
+DECODE_STATIC_SCRATCH_BYTES = 8 << 20   # CHAI_DECODE_STATIC_SCRATCH_BYTES
 
 _lib = None
 
@@ -57,6 +58,7 @@ def load() -> ctypes.CDLL:
     for name in ("chai_decode_workspace_bytes", "chai_prefill_workspace_bytes"):
         getattr(lib, name).argtypes = [ci, ci, ci, ci, ci, ci]
         getattr(lib, name).restype = sz
+    lib.chai_decode_attention_static.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
     lib.chai_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
     lib.chai_status_string.argtypes = [ci]
     lib.chai_status_string.restype = ctypes.c_char_p
@@ -171,6 +173,22 @@ def chai_decode_attention(q, k_rep, v, membership, reps, scale: float, T: int | 
     _check(load().chai_decode_attention(_ptr(q), _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps), _ptr(out), B,
                                         H, k, T, T_cap, D, scale, dt, _ptr(workspace), workspace.numel(),
                                         _stream()))
+    return out
+
+
+def chai_decode_attention_static(q, k_rep, v, membership, reps, scale: float, T: int | None = None, out=None):
+    """Decode step that uses the library's built-in 8 MiB scratch array: for callers that cannot pass
+    a workspace and must not allocate (all HBM already committed to a cache pool, or no allocation
+    allowed on the hot loop).  Problems needing more scratch raise ChaiError(CHAI_ERR_WORKSPACE).
+    `out` must be supplied by such callers; it is created here only for convenience in tests."""
+    _dev(q, k_rep, v, membership, reps, out)
+    B, H, D = q.shape
+    k, T_cap = k_rep.shape[1], k_rep.shape[2]
+    T = T_cap if T is None else T
+    if out is None:
+        out = torch.empty_like(q)
+    _check(load().chai_decode_attention_static(_ptr(q), _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps),
+                                               _ptr(out), B, H, k, T, T_cap, D, scale, _dt(q), _stream()))
     return out
 
 

@@ -328,4 +328,56 @@ int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage
     return CHAI_OK;
 }
 
+
+// ---- decode without any caller-provided or allocated scratch -------------------------------------------
+//
+// Some callers cannot hand the library a workspace and cannot let it allocate one either: a serving
+// engine that reserved all of HBM for its KV-cache pool at start-up has nothing left for cudaMalloc
+// to return, and a caller that is inside a latency-critical loop (or between two captured regions)
+// must not trigger the device-wide synchronisation an allocation implies.  For them the scratch of the
+// decode kernels lives in this fixed array, which is part of the loaded library image: every GPU
+// that loads libchai.so carries these 8 MiB until the process exits.
+constexpr size_t kStaticScratchBytes = CHAI_DECODE_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_ptr[kMaxDevices] = {};  // device address of g_static_scratch, per device
+}  // namespace
+
+int chai_decode_attention_static(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                 const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D,
+                                 float scale, int dtype, void* stream) {
+    using namespace chai;
+    CHAI_REQUIRE(B > 0 && H > 0 && k > 0 && T > 0, CHAI_ERR_INVALID_ARG,
+                 "chai_decode_attention_static: sizes must be positive");
+    CHAI_REQUIRE(dtype == CHAI_F32 || dtype == CHAI_BF16, CHAI_ERR_UNSUPPORTED,
+                 "chai_decode_attention_static: unknown dtype %d", dtype);
+    CHAI_REQUIRE(D == 64 || D == 128, CHAI_ERR_UNSUPPORTED,
+                 "chai_decode_attention_static: head_dim %d (64 or 128 supported)", D);
+    DecodeLayout L;
+    decode_layout(B, H, k, T, D, dtype, &L);
+    CHAI_REQUIRE(L.total <= kStaticScratchBytes, CHAI_ERR_WORKSPACE,
+                 "chai_decode_attention_static: this problem needs %zu bytes of scratch but the built-in array holds "
+                 "%zu; use chai_decode_attention with a caller-owned workspace",
+                 L.total, kStaticScratchBytes);
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_static: cudaGetDevice");
+    CHAI_REQUIRE(dev >= 0 && dev < kMaxDevices, CHAI_ERR_UNSUPPORTED,
+                 "chai_decode_attention_static: device index %d out of range", dev);
+    // The array's name is only a host-side handle here; kernels need the address it has on the
+    // current device, looked up once per device (benign if two threads race: same value).
+    void* ptr = g_static_scratch_ptr[dev];
+    if (ptr == nullptr) {
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_static: cudaGetSymbolAddress");
+        g_static_scratch_ptr[dev] = ptr;
+    }
+    // The decode kernels reset the tickets and the status word themselves at the start of every
+    // call, so whatever the previous call left in the array does not matter.
+    return chai_decode_attention(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, D, scale, dtype, ptr,
+                                 kStaticScratchBytes, stream);
+}
+
 }  // extern "C"
