@@ -12,14 +12,12 @@
 //                          and writes out = sum / l.  The result does not depend on scheduling.
 //
 // Because the softmax reference maximum is global (two-pass), partials need no rescaling.
-#include "chai_common.cuh"
+#include <stdlib.h>
+#include <string.h>
+
+#include "decode_layout.cuh"
 
 namespace chai {
-
-constexpr int kDecThreads = 256;
-constexpr int kDecWarps = kDecThreads / 32;
-constexpr int kStepsK = 8;   // independent 16-byte loads per thread in flight, score kernel
-constexpr int kStepsV = 16;  // rows per thread in a value chunk (two batches of 8 loads)
 
 template <typename T, int D>
 struct DecodeGeom {
@@ -31,34 +29,6 @@ struct DecodeGeom {
     static constexpr int CV = RPS * kStepsV;         // rows per value chunk
     static_assert(LPR >= 1 && LPR <= 32 && (32 % LPR) == 0, "row must split evenly over a warp");
 };
-
-struct DecodeLayout {
-    int CK, CV, nK, nV;
-    size_t off_counters, off_scores, off_cmax, off_lpart, off_opart, total;
-};
-
-static bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLayout* L) {
-    const int epv = 16 / (int)elem_size(dtype);
-    if (D != 64 && D != 128) return false;
-    const int lpr = D / epv, rpw = 32 / lpr, rps = kDecWarps * rpw;
-    L->CK = rps * kStepsK;
-    L->CV = rps * kStepsV;
-    L->nK = (T + L->CK - 1) / L->CK;
-    L->nV = (T + L->CV - 1) / L->CV;
-    size_t off = sizeof(WsHeader);
-    L->off_counters = off;
-    off = round_up(off + sizeof(int) * (size_t)B * H, 256);
-    L->off_scores = off;
-    off = round_up(off + sizeof(float) * (size_t)B * k * T, 256);
-    L->off_cmax = off;
-    off = round_up(off + sizeof(float) * (size_t)B * k * L->nK, 256);
-    L->off_lpart = off;
-    off = round_up(off + sizeof(float) * (size_t)B * H * L->nV, 256);
-    L->off_opart = off;
-    off = round_up(off + sizeof(float) * (size_t)B * H * L->nV * D, 256);
-    L->total = off;
-    return true;
-}
 
 __device__ __forceinline__ float block_max(float v, float* s_w) {
 #pragma unroll
@@ -297,6 +267,17 @@ int chai_decode_attention(const void* q, const void* k_rep, const void* v, const
                  "chai_decode_attention: workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
+    // The persistent streaming kernel is the product path; the split kernels remain for devices
+    // without cooperative launch and for A/B measurements (CHAI_DECODE_IMPL=split).
+    static const bool force_split = [] {
+        const char* e = getenv("CHAI_DECODE_IMPL");
+        return e != nullptr && strcmp(e, "split") == 0;
+    }();
+    if (!force_split) {
+        const int rc = launch_decode_persistent(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, D, scale, dtype,
+                                                ws, L, s);
+        if (rc != kDecodeNotLaunched) return rc;
+    }
     if (dtype == CHAI_BF16) {
         if (D == 128) return launch_decode<__nv_bfloat16, 128>(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, scale, ws, L, s);
         return launch_decode<__nv_bfloat16, 64>(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, scale, ws, L, s);

@@ -1,0 +1,57 @@
+// Workspace layout shared by the two decode implementations (split kernels and persistent kernel).
+#pragma once
+
+#include "chai_common.cuh"
+
+namespace chai {
+
+constexpr int kDecThreads = 256;
+constexpr int kDecWarps = kDecThreads / 32;
+constexpr int kStepsK = 8;   // independent 16-byte loads per thread in flight, score kernel
+constexpr int kStepsV = 16;  // rows per thread in a value chunk (two batches of 8 loads)
+constexpr int kTileBytes = 32768;  // persistent kernel: one ring slot = TR cache rows
+
+struct DecodeLayout {
+    int CK, CV, nK, nV;  // split kernels: rows per key / value chunk and chunks per plane
+    int TR;              // persistent kernel: rows per 16 KB tile
+    int capK, capV;      // entries per plane reserved for chunk maxima / partials (either implementation)
+    size_t off_counters, off_scores, off_cmax, off_lpart, off_opart, total;
+};
+
+inline bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLayout* L) {
+    const int es = (int)elem_size(dtype);
+    const int epv = 16 / es;
+    if (D != 64 && D != 128) return false;
+    const int lpr = D / epv, rpw = 32 / lpr, rps = kDecWarps * rpw;
+    L->CK = rps * kStepsK;
+    L->CV = rps * kStepsV;
+    L->nK = (T + L->CK - 1) / L->CK;
+    L->nV = (T + L->CV - 1) / L->CV;
+    L->TR = kTileBytes / (D * es);
+    // the persistent kernel uses key items of >= 1 tile and value items of >= 4 tiles
+    const int pk = (T + L->TR - 1) / L->TR, pv = (T + 4 * L->TR - 1) / (4 * L->TR);
+    L->capK = pk > L->nK ? pk : L->nK;
+    L->capV = pv > L->nV ? pv : L->nV;
+    size_t off = sizeof(WsHeader);
+    L->off_counters = off;
+    off = round_up(off + sizeof(int) * (size_t)B * H, 256);
+    L->off_scores = off;
+    off = round_up(off + sizeof(float) * (size_t)B * k * T, 256);
+    L->off_cmax = off;
+    off = round_up(off + sizeof(float) * (size_t)B * k * L->capK, 256);
+    L->off_lpart = off;
+    off = round_up(off + sizeof(float) * (size_t)B * H * L->capV, 256);
+    L->off_opart = off;
+    off = round_up(off + sizeof(float) * (size_t)B * H * L->capV * D, 256);
+    L->total = off;
+    return true;
+}
+
+// Persistent decode kernel (decode_persist.cu).  Returns CHAI_OK, an error, or kDecodeNotLaunched
+// when the device cannot run it (no cooperative launch), in which case the caller uses the split kernels.
+constexpr int kDecodeNotLaunched = -1;
+int launch_decode_persistent(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                             const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D, float scale,
+                             int dtype, char* ws, const DecodeLayout& L, cudaStream_t s);
+
+}  // namespace chai
