@@ -28,22 +28,17 @@ int prefill_run_plan(const int32_t* membership, const int32_t* reps, int B, int 
 
 namespace tc {
 
-// stage timestamps (SM clock) of CTA (0,0,0), per key tile: debugging aid read by chai_debug_prefill_stats
-__device__ long long g_pf_stats[64][8];
-// (smid, start ns, end ns, key tiles) of every working CTA of the last launch
-__device__ long long g_pf_cta[4096][4];
-__device__ int g_pf_cta_n;
-
 constexpr int BM = 128;            // query rows per CTA
 constexpr int BN = 128;            // keys per tile
 constexpr int HD = 128;            // head dimension
 constexpr int G = 2;               // member heads per CTA
-constexpr int KST = 2;             // K tile stages
-constexpr int VST = 4;             // V tile slots: two key tiles' worth of member tiles in flight
+constexpr int KST = 2;             // K tile stages (tile kt uses stage kt & 1)
+constexpr int VST = 2 * G;         // V tile slots: tile kt uses slots (kt & 1) * G + g
 constexpr int TILE_BYTES = BN * HD * 2;        // 32 KB: one 128 x 128 bf16 tile = two 64-column boxes
 constexpr int HALF_BYTES = TILE_BYTES / 2;     // 16 KB: one 128-row x 64-column swizzled box
 constexpr int SOFTMAX_WARPS = 8;    // two per TMEM lane quadrant: each thread owns half a row (64 columns)
-constexpr int THREADS = 64 + SOFTMAX_WARPS * 32;
+constexpr int EPILOGUE_WARPS = 4;   // one thread per query row: O / l -> bf16 -> global while the next item computes
+constexpr int THREADS = 64 + (SOFTMAX_WARPS + EPILOGUE_WARPS) * 32;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t S_COL0 = 0, O_COL0 = 256;   // S buffers at columns 0 and 128, O_g at 256 + 128 g
 constexpr long long TIMEOUT_CYCLES = 2000000000ll;  // about a second
@@ -53,10 +48,18 @@ constexpr int OFF_Q = 0;
 constexpr int OFF_K = OFF_Q + TILE_BYTES;
 constexpr int OFF_V = OFF_K + KST * TILE_BYTES;
 constexpr int OFF_BAR = OFF_V + VST * TILE_BYTES;
-constexpr int NUM_BARS = 1 + 2 * KST + 2 * VST + 2 + 2;
+constexpr int NUM_BARS = 18;
 constexpr int OFF_XCH = OFF_BAR + 8 * NUM_BARS + 16;               // after the barriers and the tmem slot / abort word
-constexpr int XCH_BYTES = 2 * BM * 4;                              // row maxima / sums exchanged between the two halves
-constexpr int SMEM_BYTES = OFF_XCH + XCH_BYTES + 1024;             // + alignment slack
+constexpr int XCH_BYTES = 2 * BM * 4;                              // row maxima exchanged between the two halves
+constexpr int OFF_LSUM = OFF_XCH + XCH_BYTES;                      // row sums handed to the epilogue warps
+constexpr int OFF_ITEM = OFF_LSUM + 2 * BM * 4;                    // two work-item descriptors + one for the epilogue
+constexpr int ITEM_BYTES = 3 * 32;
+constexpr int OFF_PREFIX = OFF_ITEM + ITEM_BYTES;                  // running sum of groups per request
+constexpr int MAX_B = 64;                                          // requests per launch on this path
+// No alignment slack: the dynamic shared memory of a kernel without static shared memory starts right
+// after the 1 KB the system reserves per CTA, i.e. 1024-byte aligned; the kernel checks and refuses otherwise.
+constexpr int SMEM_BYTES = OFF_PREFIX + 4 * (MAX_B + 1) + 12;
+static_assert(SMEM_BYTES <= 232448, "shared memory budget");
 
 // ---- PTX wrappers ---------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -94,10 +97,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+// one 128-row x 128-column bf16 tile = box (64 columns, 128 rows, 2 column halves, 1 plane): lands as two
+// consecutive 16 KB blocks of 128-byte swizzled rows, which is the layout the MMA descriptors describe
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int row, int plane, uint32_t bar) {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(0), "r"(plane), "r"(bar)
         : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -182,61 +187,80 @@ __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 }
 
-// mbarrier addresses, computed rather than stored so that stage indices stay in registers
+// mbarrier addresses, computed rather than stored so that stage indices stay in registers.
+// Tile-indexed barriers come in pairs: key tile number kt (counted over the CTA's whole life) uses
+// entry kt & 1 in phase (kt >> 1) & 1.  qk_done[i] tells the softmax warps that S is ready AND the
+// producer that the K stage is free; pv_done[i] tells the softmax warps that O may be touched AND
+// the producer that the tile's V slots are free: one tcgen05.commit serves both waiters.
 struct Bars {
     uint32_t base;
     __device__ __forceinline__ uint32_t q_full() const { return base; }
-    __device__ __forceinline__ uint32_t k_full(int i) const { return base + 8 * (1 + i); }
-    __device__ __forceinline__ uint32_t k_empty(int i) const { return base + 8 * (1 + KST + i); }
-    __device__ __forceinline__ uint32_t v_full(int i) const { return base + 8 * (1 + 2 * KST + i); }
-    __device__ __forceinline__ uint32_t v_empty(int i) const { return base + 8 * (1 + 2 * KST + VST + i); }
-    __device__ __forceinline__ uint32_t s_full(int i) const { return base + 8 * (1 + 2 * KST + 2 * VST + i); }
-    __device__ __forceinline__ uint32_t p_full() const { return base + 8 * (3 + 2 * KST + 2 * VST); }
-    __device__ __forceinline__ uint32_t pv_done() const { return base + 8 * (4 + 2 * KST + 2 * VST); }
+    __device__ __forceinline__ uint32_t q_empty() const { return base + 8; }
+    __device__ __forceinline__ uint32_t o_free() const { return base + 16; }
+    __device__ __forceinline__ uint32_t p_full() const { return base + 24; }
+    __device__ __forceinline__ uint32_t item_full(int i) const { return base + 8 * (4 + i); }
+    __device__ __forceinline__ uint32_t item_empty(int i) const { return base + 8 * (6 + i); }
+    __device__ __forceinline__ uint32_t k_full(int i) const { return base + 8 * (8 + i); }
+    __device__ __forceinline__ uint32_t v_full(int i) const { return base + 8 * (10 + i); }
+    __device__ __forceinline__ uint32_t qk_done(int i) const { return base + 8 * (12 + i); }
+    __device__ __forceinline__ uint32_t pv_done(int i) const { return base + 8 * (14 + i); }
+    __device__ __forceinline__ uint32_t epi_full() const { return base + 8 * 16; }
+    __device__ __forceinline__ uint32_t epi_empty() const { return base + 8 * 17; }
+};
+static_assert(NUM_BARS == 18, "barrier count");
+
+// One unit of work, published by the producer to the other roles through shared memory.
+struct Item {
+    int n_kv;        // key tiles to walk; 0 = zero-fill item (unresolved heads); -1 = no more work
+    int n_members;   // heads in this group (1..G)
+    int q0;          // first query row of the tile
+    int q_plane;     // b * H + representative head
+    int k_plane;     // b * k + cluster
+    int o_plane[G];  // b * H + member head
+    int pad;
 };
 
+// Persistent kernel: one CTA per SM walks work items (request, member group, query tile) handed out
+// by an atomic counter in descending order of cost.  While the softmax warps finish one item, the
+// producer is already fetching the next item's Q, K and V tiles and the tensor core computes its
+// first scores, so the pipeline fill of an item hides behind the drain of the previous one.
 __global__ void __launch_bounds__(THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int* __restrict__ n_groups,
                   const GroupEntry* __restrict__ groups, __nv_bfloat16* __restrict__ out, WsHeader* __restrict__ hdr,
-                  int H, int k, int T_len, float scale_log2, int causal, int n_qtiles) {
-    const int b = blockIdx.z, slot = blockIdx.y;
-    if (slot >= n_groups[b]) return;
-    const GroupEntry e = groups[(size_t)b * H + slot];
-    const int qt = n_qtiles - 1 - (int)blockIdx.x;  // heaviest query tiles first
-    const int q0 = qt * BM;
+                  int b_begin, int B, int H, int k, int T_len, float scale_log2, int causal, int n_qtiles, int counter_slot) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const bool dbg = blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0;
-
-    if (e.cluster < 0) {  // unresolved heads: zero rows
-        for (int g = 0; g < e.n; ++g) {
-            uint4* o = reinterpret_cast<uint4*>(out + (((size_t)b * H + e.heads[g]) * T_len + q0) * HD);
-            const int rows = min(BM, T_len - q0);
-            for (int idx = tid; idx < rows * (HD / 8); idx += THREADS) o[idx] = make_uint4(0, 0, 0, 0);
-        }
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = smem_raw;
+    const uint32_t sbase = smem_u32(smem);
+    if ((sbase & 1023u) != 0) {  // swizzled tiles need 1024-byte alignment; never observed, but refuse rather than corrupt
+        if (tid == 0) atomicExch(&hdr->status, CHAI_ERR_TIMEOUT);
         return;
     }
-    const int n_members = min(e.n, G);
-    long long cta_t0 = 0;
-    if (tid == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(cta_t0));
-    const int n_kv = causal ? min(qt + 1, (T_len + BN - 1) / BN) : (T_len + BN - 1) / BN;
-
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t sbase = smem_u32(smem);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + OFF_BAR + 8 * NUM_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
+    Item* items = reinterpret_cast<Item*>(smem + OFF_ITEM);          // [2] producer -> MMA / softmax; [2] = softmax -> epilogue
+    int* prefix = reinterpret_cast<int*>(smem + OFF_PREFIX);         // [B + 1] running sum of n_groups
     const Bars bar{sbase + OFF_BAR};
 
     if (tid == 0) {
         mbar_init(bar.q_full(), 1);
-        for (int i = 0; i < KST; ++i) { mbar_init(bar.k_full(i), 1); mbar_init(bar.k_empty(i), 1); }
-        for (int i = 0; i < VST; ++i) { mbar_init(bar.v_full(i), 1); mbar_init(bar.v_empty(i), 1); }
-        for (int i = 0; i < 2; ++i) mbar_init(bar.s_full(i), 1);
+        mbar_init(bar.q_empty(), 1);
+        mbar_init(bar.o_free(), EPILOGUE_WARPS * 32);
+        mbar_init(bar.epi_full(), SOFTMAX_WARPS * 32);
+        mbar_init(bar.epi_empty(), EPILOGUE_WARPS * 32);
         mbar_init(bar.p_full(), SOFTMAX_WARPS * 32);
-        mbar_init(bar.pv_done(), 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(bar.item_full(i), 1);
+            mbar_init(bar.item_empty(i), 1 + SOFTMAX_WARPS * 32);
+            mbar_init(bar.k_full(i), 1);
+            mbar_init(bar.v_full(i), 1);
+            mbar_init(bar.qk_done(i), 1);
+            mbar_init(bar.pv_done(i), 1);
+        }
         *abort_flag = 0;
+        prefix[0] = 0;
+        for (int bb = 0; bb < B; ++bb) prefix[bb + 1] = prefix[bb] + n_groups[b_begin + bb];
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_proxy();
     }
@@ -250,37 +274,78 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- producer: work distribution and TMA loads ----------------
         if (lane == 0) {
-            const int q_plane = b * H + e.rep, k_plane = b * k + e.cluster;
-            mbar_expect_tx(bar.q_full(), TILE_BYTES);
-            tma_load_3d(sbase + OFF_Q, &map_q, 0, q0, q_plane, bar.q_full());
-            tma_load_3d(sbase + OFF_Q + HALF_BYTES, &map_q, 64, q0, q_plane, bar.q_full());
+            const int n_pairs = prefix[B];                 // (request, group) pairs that exist
+            const int n_items = n_pairs * n_qtiles;        // heaviest query tiles first
             bool ok = true;
-            auto load_k = [&](int j) -> bool {
-                const int ks = j % KST;
-                if (!mbar_wait(bar.k_empty(ks), ((j / KST) & 1) ^ 1, abort_flag)) return false;
-                mbar_expect_tx(bar.k_full(ks), TILE_BYTES);
-                tma_load_3d(sbase + OFF_K + ks * TILE_BYTES, &map_k, 0, j * BN, k_plane, bar.k_full(ks));
-                tma_load_3d(sbase + OFF_K + ks * TILE_BYTES + HALF_BYTES, &map_k, 64, j * BN, k_plane, bar.k_full(ks));
-                return true;
-            };
-            // order of need: K(0), K(1), V(0,*), K(2), V(1,*), ...  (S of tile j+1 is computed before P V of tile j)
-            ok = load_k(0);
-            for (int j = 0; j < n_kv && ok; ++j) {
-                if (dbg && j < 16) g_pf_stats[48 + j][0] = clock64();
-                if (j + 1 < n_kv) ok = load_k(j + 1);
-                if (dbg && j < 16) g_pf_stats[48 + j][1] = clock64();
-                for (int g = 0; g < n_members && ok; ++g) {
-                    const int t = j * n_members + g, vs = t % VST;
-                    ok = mbar_wait(bar.v_empty(vs), ((t / VST) & 1) ^ 1, abort_flag);
-                    if (!ok) break;
-                    if (dbg && j < 16 && g < 2) g_pf_stats[48 + j][2 + g] = clock64();
-                    const int v_plane = b * H + e.heads[g];
-                    mbar_expect_tx(bar.v_full(vs), TILE_BYTES);
-                    tma_load_3d(sbase + OFF_V + vs * TILE_BYTES, &map_v, 0, j * BN, v_plane, bar.v_full(vs));
-                    tma_load_3d(sbase + OFF_V + vs * TILE_BYTES + HALF_BYTES, &map_v, 64, j * BN, v_plane, bar.v_full(vs));
+            int it = 0, qi = 0, kt = 0;                    // items published, items with loads, key tiles issued
+            while (ok) {
+                const int id = atomicAdd(&hdr->pad[counter_slot], 1);  // next unit of work (the header was cleared by the host)
+                const int is = it & 1;
+                ok = mbar_wait(bar.item_empty(is), ((it >> 1) & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                Item& item = items[is];
+                if (id >= n_items) {
+                    item.n_kv = -1;
+                    mbar_arrive(bar.item_full(is));
+                    break;
                 }
+                const int qt = n_qtiles - 1 - id / n_pairs, pair = id % n_pairs;
+                int lo = 0, hi = B;                        // largest b with prefix[b] <= pair
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (prefix[mid] <= pair) lo = mid; else hi = mid;
+                }
+                const int b = b_begin + lo, slot = pair - prefix[lo];
+                const GroupEntry e = groups[(size_t)b * H + slot];
+                const int n_members = min(e.n, G);
+                item.q0 = qt * BM;
+                item.n_members = n_members;
+                for (int g = 0; g < G; ++g) item.o_plane[g] = b * H + e.heads[g < n_members ? g : 0];
+                if (e.cluster < 0) {                       // unresolved heads: zero rows, nothing to load
+                    item.n_kv = 0;
+                    item.q_plane = item.k_plane = 0;
+                    mbar_arrive(bar.item_full(is));
+                    ++it;
+                    continue;
+                }
+                const int n_kv = causal ? min(qt + 1, (T_len + BN - 1) / BN) : (T_len + BN - 1) / BN;
+                item.n_kv = n_kv;
+                item.q_plane = b * H + e.rep;
+                item.k_plane = b * k + e.cluster;
+                mbar_arrive(bar.item_full(is));
+                const int q_plane = item.q_plane, k_plane = item.k_plane, q0 = item.q0;
+                int v_plane[G];
+                for (int g = 0; g < G; ++g) v_plane[g] = item.o_plane[g];
+                // Q: wait until the previous item's last S = Q K^T has been computed
+                ok = mbar_wait(bar.q_empty(), (qi & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                mbar_expect_tx(bar.q_full(), TILE_BYTES);
+                tma_load_4d(sbase + OFF_Q, &map_q, q0, q_plane, bar.q_full());
+                // key tile number kt + j of this CTA's life: K stage and V slots (kt + j) & 1
+                auto load_k = [&](int j) -> bool {
+                    const int n = kt + j, ts = n & 1;
+                    if (!mbar_wait(bar.qk_done(ts), ((n >> 1) & 1) ^ 1, abort_flag)) return false;  // stage free
+                    mbar_expect_tx(bar.k_full(ts), TILE_BYTES);
+                    tma_load_4d(sbase + OFF_K + ts * TILE_BYTES, &map_k, j * BN, k_plane, bar.k_full(ts));
+                    return true;
+                };
+                // order of need: K(0), K(1), V(0,*), K(2), V(1,*), ...  (S of tile j+1 is computed before P V of tile j)
+                ok = load_k(0);
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    if (j + 1 < n_kv) ok = load_k(j + 1);
+                    if (!ok) break;
+                    const int n = kt + j, ts = n & 1;
+                    ok = mbar_wait(bar.pv_done(ts), ((n >> 1) & 1) ^ 1, abort_flag);  // the tile's V slots are free
+                    if (!ok) break;
+                    mbar_expect_tx(bar.v_full(ts), n_members * TILE_BYTES);
+                    for (int g = 0; g < n_members; ++g)
+                        tma_load_4d(sbase + OFF_V + (ts * G + g) * TILE_BYTES, &map_v, j * BN, v_plane[g], bar.v_full(ts));
+                }
+                kt += n_kv;
+                ++it;
+                ++qi;
             }
         }
     } else if (warp == 1) {
@@ -295,53 +360,63 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const uint32_t hi_k = (uint32_t)(dq >> 32), hi_v = (uint32_t)(dv >> 32);
             const uint32_t q_lo = (uint32_t)dq, k_lo = (uint32_t)dk, v_lo = (uint32_t)dv;
             auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
-            bool ok = mbar_wait(bar.q_full(), 0, abort_flag);
-            auto issue_qk = [&](int j) -> bool {
-                const int ks = j % KST, sb = j & 1;
-                if (!mbar_wait(bar.k_full(ks), (j / KST) & 1, abort_flag)) return false;
-                tc_fence_after();
-                const uint32_t d = tmem_base + S_COL0 + sb * BN;
-                const uint32_t kb = k_lo + ks * (TILE_BYTES >> 4);
+            bool ok = true;
+            int it = 0, qi = 0, kt = 0;  // items seen, items computed, key tiles whose S has been issued
+            while (ok) {
+                const int is = it & 1;
+                ok = mbar_wait(bar.item_full(is), (it >> 1) & 1, abort_flag);
+                if (!ok) break;
+                const int n_kv = items[is].n_kv, n_members = items[is].n_members;
+                mbar_arrive(bar.item_empty(is));  // the two fields are in registers
+                if (n_kv < 0) break;
+                if (n_kv == 0) {
+                    ++it;
+                    continue;
+                }
+                ok = mbar_wait(bar.q_full(), qi & 1, abort_flag);
+                // S(tile kt) = Q K^T into S buffer kt & 1
+                auto issue_qk = [&](bool last) -> bool {
+                    const int ts = kt & 1;
+                    if (!mbar_wait(bar.k_full(ts), (kt >> 1) & 1, abort_flag)) return false;
+                    tc_fence_after();
+                    const uint32_t d = tmem_base + S_COL0 + ts * BN;
+                    const uint32_t kb = k_lo + ts * (TILE_BYTES >> 4);
 #pragma unroll
-                for (int s = 0; s < HD / 16; ++s) {
-                    const uint32_t off = ((s >> 2) * HALF_BYTES + (s & 3) * 32) >> 4;
-                    tc_mma(d, desc(hi_k, q_lo + off), desc(hi_k, kb + off), IDESC_QK, s > 0);
-                }
-                tc_commit(bar.k_empty(ks));
-                tc_commit(bar.s_full(sb));
-                return true;
-            };
-            if (ok) ok = issue_qk(0);
-            for (int j = 0; j < n_kv && ok; ++j) {
-                if (j + 1 < n_kv) ok = issue_qk(j + 1);
-                if (!ok) break;
-                if (dbg && j < 64) g_pf_stats[j][5] = clock64();
-                ok = mbar_wait(bar.p_full(), j & 1, abort_flag);
-                if (dbg && j < 16) g_pf_stats[32 + j][0] = clock64();
-                for (int g = 0; g < n_members && ok; ++g) {
-                    const int t = j * n_members + g;
-                    ok = mbar_wait(bar.v_full(t % VST), (t / VST) & 1, abort_flag);
-                }
-                if (!ok) break;
-                tc_fence_after();
-                if (dbg && j < 64) g_pf_stats[j][6] = clock64();
-                const uint32_t p_addr = tmem_base + S_COL0 + (j & 1) * BN;  // P(j): first 64 columns of S(j)
-                for (int g = 0; g < n_members; ++g) {
-                    const int vs = (j * n_members + g) % VST;
-                    const uint32_t d = tmem_base + O_COL0 + g * HD;
-                    const uint32_t vb = v_lo + vs * (TILE_BYTES >> 4);
+                    for (int s = 0; s < HD / 16; ++s) {
+                        const uint32_t off = ((s >> 2) * HALF_BYTES + (s & 3) * 32) >> 4;
+                        tc_mma(d, desc(hi_k, q_lo + off), desc(hi_k, kb + off), IDESC_QK, s > 0);
+                    }
+                    tc_commit(bar.qk_done(ts));
+                    if (last) tc_commit(bar.q_empty());  // Q may be overwritten by the next item's tile
+                    ++kt;
+                    return true;
+                };
+                if (ok) ok = issue_qk(n_kv == 1);
+                for (int j = 0; j < n_kv && ok; ++j) {
+                    if (j + 1 < n_kv) ok = issue_qk(j + 2 == n_kv);
+                    if (!ok) break;
+                    const int pt = kt - (j + 1 < n_kv ? 2 : 1), ts = pt & 1;  // global index of tile j
+                    ok = mbar_wait(bar.p_full(), pt & 1, abort_flag) && mbar_wait(bar.v_full(ts), (pt >> 1) & 1, abort_flag);
+                    // the previous item's output must have left tensor memory before its accumulators are reused
+                    if (ok && j == 0 && qi > 0) ok = mbar_wait(bar.o_free(), (qi - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t p_addr = tmem_base + S_COL0 + ts * BN;  // P: first 64 columns of its S buffer
+                    for (int g = 0; g < n_members; ++g) {
+                        const uint32_t d = tmem_base + O_COL0 + g * HD;
+                        const uint32_t vb = v_lo + (ts * G + g) * (TILE_BYTES >> 4);
 #pragma unroll
-                    for (int s = 0; s < BN / 16; ++s)  // 16 keys per step: 8 TMEM columns of P, 2048 bytes of V
-                        tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV, (j > 0 || s > 0) ? 1u : 0u);
-                    tc_commit(bar.v_empty(vs));
+                        for (int s = 0; s < BN / 16; ++s)  // 16 keys per step: 8 TMEM columns of P, 2048 bytes of V
+                            tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV, (j > 0 || s > 0) ? 1u : 0u);
+                    }
+                    tc_commit(bar.pv_done(ts));
                 }
-                if (!ok) break;
-                tc_commit(bar.pv_done());
-                if (dbg && j < 64) g_pf_stats[j][7] = clock64();
+                ++it;
+                ++qi;
             }
         }
-    } else {
-        // ---------------- softmax / correction / epilogue: two threads per query row ----------------
+    } else if (warp < 2 + SOFTMAX_WARPS) {
+        // ---------------- softmax / correction: two threads per query row ----------------
         // Warps 2..5 own columns 0..63 of their rows, warps 6..9 columns 64..127; the two threads of a row
         // sit in different warps of the same TMEM lane quadrant and meet once per tile at a 64-thread
         // named barrier, where they exchange their half-row maxima.  By then both have their 64 scores in
@@ -349,146 +424,195 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int quad = warp & 3;               // TMEM lanes this warp may touch
         const int half = (warp - 2) >> 2;        // which 64 columns of the tile
         const int row = quad * 32 + lane;        // row of the tile
-        const int row_abs = q0 + row;
         const int cbase = half * 64;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-        float* xch = reinterpret_cast<float*>(smem + OFF_XCH);  // [half][row]
+        float* xch = reinterpret_cast<float*>(smem + OFF_XCH);    // [half][row]
+        float* lsum = reinterpret_cast<float*>(smem + OFF_LSUM);  // [half][row]
         auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quad) : "memory"); };
-        float m_used = -INFINITY, l_run = 0.f;
         bool ok = true;
+        int it = 0, ei = 0, kt = 0;  // items seen, items handed to the epilogue, key tiles processed so far
         uint32_t r[64];
-        for (int j = 0; j < n_kv && ok; ++j) {
-            const int sb = j & 1;
-            const bool rec = dbg && tid == 64 && j < 64;
-            if (rec) g_pf_stats[j][0] = clock64();
-            ok = __all_sync(0xffffffffu, mbar_wait(bar.s_full(sb), (j >> 1) & 1, abort_flag));
-            if (!ok) break;  // warp-uniform: the tcgen05 loads below are warp-collective
-            if (rec) g_pf_stats[j][1] = clock64();
-            tc_fence_after();
-            const uint32_t s_addr = lane_addr + S_COL0 + sb * BN;
-            const int col0 = j * BN;
-            // columns of this thread's half that the row may see: col_abs < T and (causal: col_abs <= row_abs)
-            int vis = T_len - col0;
-            if (causal) vis = min(vis, row_abs - col0 + 1);
-            vis = max(0, min(vis - cbase, 64));
-            // the whole tile is visible to every row unless it is the diagonal tile or runs past T
-            const bool full_tile = col0 + BN <= T_len && (!causal || col0 + BN - 1 <= q0);
-            tc_ld32(s_addr + cbase, r);
-            tc_ld32(s_addr + cbase + 32, r + 32);
-            tc_wait_ld();
-            float mx0 = -INFINITY, mx1 = -INFINITY;
-            if (full_tile) {
-#pragma unroll
-                for (int i = 0; i < 64; i += 2) {
-                    mx0 = fmaxf(mx0, __uint_as_float(r[i]));
-                    mx1 = fmaxf(mx1, __uint_as_float(r[i + 1]));
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 64; ++i)
-                    if (i < vis) mx0 = fmaxf(mx0, __uint_as_float(r[i]));
-            }
-            float mx = fmaxf(mx0, mx1);
-            xch[half * BM + row] = mx;
-            pair_sync();
-            mx = fmaxf(mx, xch[(half ^ 1) * BM + row]);
-            pair_sync();  // both values read before either slot is written again
-            if (rec) g_pf_stats[j][2] = clock64();
-            const float m_tile = mx * scale_log2;
-            float m_new = m_used, corr = 1.f;
-            if (m_tile > m_used + 8.f) {  // lazy rescale: only when the reference would be off by > 2^8
-                m_new = m_tile;
-                corr = fast_exp2(m_used - m_new);  // 0 on the first tile (m_used = -inf)
-            }
-            const float m_ref = m_new == -INFINITY ? 0.f : m_new;
-            // probabilities, rounded to bf16, two per 32-bit column, written over the first half of the S
-            // buffer: the layout of an A operand in tensor memory.  S columns 64 h + c map to P column 32 h + c / 2.
-            float ls0 = 0.f, ls1 = 0.f, ls2 = 0.f, ls3 = 0.f;
-            uint32_t packed[32];
-            if (full_tile) {
-#pragma unroll
-                for (int i = 0; i < 64; i += 4) {
-                    const float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
-                    const float p2 = fast_exp2(fmaf(__uint_as_float(r[i + 2]), scale_log2, -m_ref));
-                    const float p3 = fast_exp2(fmaf(__uint_as_float(r[i + 3]), scale_log2, -m_ref));
-                    ls0 += p0;
-                    ls1 += p1;
-                    ls2 += p2;
-                    ls3 += p3;
-                    __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
-                    packed[i >> 1] = *reinterpret_cast<uint32_t*>(&pa);
-                    packed[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 64; i += 2) {
-                    float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
-                    float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
-                    if (i >= vis) p0 = 0.f;
-                    if (i + 1 >= vis) p1 = 0.f;
-                    ls0 += p0;
-                    ls1 += p1;
-                    __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                    packed[i >> 1] = *reinterpret_cast<uint32_t*>(&pk);
-                }
-            }
-            tc_st16(s_addr + half * 32, packed);
-            tc_st16(s_addr + half * 32 + 16, packed + 16);
-            l_run = l_run * corr + ((ls0 + ls1) + (ls2 + ls3));
-            m_used = m_new;
-            if (rec) g_pf_stats[j][3] = clock64();
-            // the previous tile's PV must be complete before the O accumulators are rescaled
-            if (j > 0) {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done(), (j - 1) & 1, abort_flag));
-                if (!ok) break;
-                tc_fence_after();
-                if (__any_sync(0xffffffffu, corr != 1.f)) {  // this thread rescales its 64 columns of each O
+        while (true) {
+            const int is = it & 1;
+            ok = ok && mbar_wait(bar.item_full(is), (it >> 1) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const Item item = items[is];
+            __syncwarp();
+            mbar_arrive(bar.item_empty(is));  // the item is in registers
+            if (item.n_kv < 0) break;
+            const int n_kv = item.n_kv, n_members = item.n_members, q0 = item.q0;
+            const int row_abs = q0 + row;
+            if (n_kv == 0) {  // unresolved heads: zero rows
+                if (row_abs < T_len)
                     for (int g = 0; g < n_members; ++g) {
-                        const uint32_t o_addr = lane_addr + O_COL0 + g * HD + cbase;
-                        tc_ld32(o_addr, r);
-                        tc_ld32(o_addr + 32, r + 32);
-                        tc_wait_ld();
+                        uint4* o = reinterpret_cast<uint4*>(out + ((size_t)item.o_plane[g] * T_len + row_abs) * HD + cbase);
 #pragma unroll
-                        for (int i = 0; i < 64; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
-                        tc_st32(o_addr, r);
-                        tc_st32(o_addr + 32, r + 32);
+                        for (int u = 0; u < 8; ++u) o[u] = make_uint4(0, 0, 0, 0);
+                    }
+                ++it;
+                continue;
+            }
+            float m_used = -INFINITY, l_run = 0.f;
+            for (int j = 0; j < n_kv && ok; ++j, ++kt) {
+                const int sb = kt & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar.qk_done(sb), (kt >> 1) & 1, abort_flag));
+                if (!ok) break;  // warp-uniform: the tcgen05 loads below are warp-collective
+                tc_fence_after();
+                const uint32_t s_addr = lane_addr + S_COL0 + sb * BN;
+                const int col0 = j * BN;
+                // columns of this thread's half that the row may see: col_abs < T and (causal: col_abs <= row_abs)
+                int vis = T_len - col0;
+                if (causal) vis = min(vis, row_abs - col0 + 1);
+                vis = max(0, min(vis - cbase, 64));
+                // the whole tile is visible to every row unless it is the diagonal tile or runs past T
+                const bool full_tile = col0 + BN <= T_len && (!causal || col0 + BN - 1 <= q0);
+                tc_ld32(s_addr + cbase, r);
+                tc_ld32(s_addr + cbase + 32, r + 32);
+                tc_wait_ld();
+                float mx0 = -INFINITY, mx1 = -INFINITY;
+                if (full_tile) {
+#pragma unroll
+                    for (int i = 0; i < 64; i += 2) {
+                        mx0 = fmaxf(mx0, __uint_as_float(r[i]));
+                        mx1 = fmaxf(mx1, __uint_as_float(r[i + 1]));
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 64; ++i)
+                        if (i < vis) mx0 = fmaxf(mx0, __uint_as_float(r[i]));
+                }
+                float mx = fmaxf(mx0, mx1);
+                xch[half * BM + row] = mx;
+                pair_sync();
+                mx = fmaxf(mx, xch[(half ^ 1) * BM + row]);
+                pair_sync();  // both values read before either slot is written again
+                const float m_tile = mx * scale_log2;
+                float m_new = m_used, corr = 1.f;
+                if (m_tile > m_used + 8.f) {  // lazy rescale: only when the reference would be off by > 2^8
+                    m_new = m_tile;
+                    corr = fast_exp2(m_used - m_new);  // 0 on the first tile (m_used = -inf)
+                }
+                const float m_ref = m_new == -INFINITY ? 0.f : m_new;
+                // probabilities, rounded to bf16, two per 32-bit column, written over the first half of the S
+                // buffer: the layout of an A operand in tensor memory.  S columns 64 h + c map to P column 32 h + c / 2.
+                float ls0 = 0.f, ls1 = 0.f, ls2 = 0.f, ls3 = 0.f;
+                uint32_t packed[32];
+                if (full_tile) {
+#pragma unroll
+                    for (int i = 0; i < 64; i += 4) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
+                        const float p2 = fast_exp2(fmaf(__uint_as_float(r[i + 2]), scale_log2, -m_ref));
+                        const float p3 = fast_exp2(fmaf(__uint_as_float(r[i + 3]), scale_log2, -m_ref));
+                        ls0 += p0;
+                        ls1 += p1;
+                        ls2 += p2;
+                        ls3 += p3;
+                        __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
+                        packed[i >> 1] = *reinterpret_cast<uint32_t*>(&pa);
+                        packed[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 64; i += 2) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
+                        if (i >= vis) p0 = 0.f;
+                        if (i + 1 >= vis) p1 = 0.f;
+                        ls0 += p0;
+                        ls1 += p1;
+                        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                        packed[i >> 1] = *reinterpret_cast<uint32_t*>(&pk);
                     }
                 }
-            }
-            tc_wait_st();          // P (and any rescaled O) is in tensor memory
-            tc_fence_before();
-            mbar_arrive(bar.p_full());
-            if (rec) g_pf_stats[j][4] = clock64();
-            if (dbg && j < 16) atomicMax(reinterpret_cast<unsigned long long*>(&g_pf_stats[32 + j][2]), (unsigned long long)clock64());
-        }
-        // epilogue: O_g / l -> bf16 -> global; the row sum is the sum of the two halves' sums
-        if (ok) ok = mbar_wait(bar.pv_done(), (n_kv - 1) & 1, abort_flag);
-        ok = __all_sync(0xffffffffu, ok);
-        {
-            xch[half * BM + row] = l_run;
-            pair_sync();
-            l_run += xch[(half ^ 1) * BM + row];
-        }
-        if (ok) {
-            tc_fence_after();
-            const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-            for (int g = 0; g < n_members; ++g) {
-                __nv_bfloat16* orow = out + (((size_t)b * H + e.heads[g]) * T_len + row_abs) * HD + cbase;
-                tc_ld32(lane_addr + O_COL0 + g * HD + cbase, r);
-                tc_ld32(lane_addr + O_COL0 + g * HD + cbase + 32, r + 32);
-                tc_wait_ld();
-                if (row_abs < T_len) {
+                tc_st16(s_addr + half * 32, packed);
+                tc_st16(s_addr + half * 32 + 16, packed + 16);
+                l_run = l_run * corr + ((ls0 + ls1) + (ls2 + ls3));
+                m_used = m_new;
+                // the previous tile's PV must be complete before the O accumulators are rescaled
+                if (j > 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done((kt - 1) & 1), ((kt - 1) >> 1) & 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (__any_sync(0xffffffffu, corr != 1.f)) {  // this thread rescales its 64 columns of each O
+                        for (int g = 0; g < n_members; ++g) {
+                            const uint32_t o_addr = lane_addr + O_COL0 + g * HD + cbase;
+                            tc_ld32(o_addr, r);
+                            tc_ld32(o_addr + 32, r + 32);
+                            tc_wait_ld();
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        uint32_t w[4];
-#pragma unroll
-                        for (int x = 0; x < 4; ++x) {
-                            __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(r[8 * u + 2 * x]) * inv,
-                                                                      __uint_as_float(r[8 * u + 2 * x + 1]) * inv);
-                            w[x] = *reinterpret_cast<uint32_t*>(&pk);
+                            for (int i = 0; i < 64; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+                            tc_st32(o_addr, r);
+                            tc_st32(o_addr + 32, r + 32);
                         }
-                        *reinterpret_cast<uint4*>(orow + u * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+                tc_wait_st();          // P (and any rescaled O) is in tensor memory
+                tc_fence_before();
+                mbar_arrive(bar.p_full());
+            }
+            // hand the item to the epilogue warps: row sums of both halves and where the output goes
+            ok = __all_sync(0xffffffffu, ok && mbar_wait(bar.epi_empty(), (ei & 1) ^ 1, abort_flag));
+            if (!ok) break;
+            lsum[half * BM + row] = l_run;
+            if (tid == 64) {
+                Item& ep = items[2];
+                ep = item;
+                ep.n_kv = kt - 1;  // global index of the item's last key tile (its P V completion is awaited)
+            }
+            mbar_arrive(bar.epi_full());
+            ++ei;
+            ++it;
+        }
+        // tell the epilogue warps that nothing more will come
+        if (__all_sync(0xffffffffu, mbar_wait(bar.epi_empty(), (ei & 1) ^ 1, abort_flag))) {
+            if (tid == 64) items[2].n_members = -1;
+            mbar_arrive(bar.epi_full());
+        }
+    } else {
+        // ---------------- epilogue: O_g / l -> bf16 -> global, one thread per query row ----------------
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const float* lsum = reinterpret_cast<const float*>(smem + OFF_LSUM);
+        uint32_t r[32];
+        for (int ei = 0;; ++ei) {
+            bool ok = __all_sync(0xffffffffu, mbar_wait(bar.epi_full(), ei & 1, abort_flag));
+            if (!ok) break;
+            const Item ep = items[2];
+            const float l = lsum[row] + lsum[BM + row];
+            if (ep.n_members < 0) break;
+            const int last = ep.n_kv;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done(last & 1), (last >> 1) & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
+            __syncwarp();
+            mbar_arrive(bar.epi_empty());  // the hand-over area is in registers
+            const int row_abs = ep.q0 + row;
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            for (int g = 0; g < ep.n_members; ++g) {
+                __nv_bfloat16* orow = out + ((size_t)ep.o_plane[g] * T_len + row_abs) * HD;
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    tc_ld32(lane_addr + O_COL0 + g * HD + ch * 32, r);
+                    tc_wait_ld();
+                    if (g == ep.n_members - 1 && ch == 3) {  // this row's accumulators are in registers
+                        tc_fence_before();
+                        mbar_arrive(bar.o_free());
+                    }
+                    if (row_abs < T_len) {
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int x = 0; x < 4; ++x) {
+                                __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(r[8 * u + 2 * x]) * inv,
+                                                                          __uint_as_float(r[8 * u + 2 * x + 1]) * inv);
+                                w[x] = *reinterpret_cast<uint32_t*>(&pk);
+                            }
+                            *reinterpret_cast<uint4*>(orow + ch * 32 + u * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
                     }
                 }
             }
@@ -503,19 +627,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
     if (tid == 0 && *abort_flag) atomicExch(&hdr->status, CHAI_ERR_TIMEOUT);
-    if (tid == 0) {
-        long long t1;
-        unsigned smid;
-        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
-        asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-        const int idx = atomicAdd(&g_pf_cta_n, 1);
-        if (idx < 4096) {
-            g_pf_cta[idx][0] = smid;
-            g_pf_cta[idx][1] = cta_t0;
-            g_pf_cta[idx][2] = t1;
-            g_pf_cta[idx][3] = n_kv;
-        }
-    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -534,15 +645,16 @@ static EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// [planes, T, 128] bf16 viewed as a 3-D tensor (innermost first); box = 64 columns x 128 rows x 1 plane.
+// [planes, T, 128] bf16 viewed as a 4-D tensor (innermost first): 64 columns, T rows, 2 column halves, planes;
+// box = 64 x 128 x 2 x 1, i.e. a whole 128 x 128 tile per copy, stored as two swizzled 64-column blocks.
 static bool make_map(CUtensorMap* map, const void* base, int planes, int T) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)HD, (cuuint64_t)T, (cuuint64_t)planes};
-    cuuint64_t strides[2] = {(cuuint64_t)HD * 2, (cuuint64_t)T * HD * 2};
-    cuuint32_t box[3] = {64, (cuuint32_t)BN, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+    cuuint64_t dims[4] = {64, (cuuint64_t)T, 2, (cuuint64_t)planes};
+    cuuint64_t strides[3] = {(cuuint64_t)HD * 2, 128, (cuuint64_t)T * HD * 2};
+    cuuint32_t box[4] = {64, (cuuint32_t)BN, 2, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -554,7 +666,7 @@ extern "C" int chai_prefill_attention(const void* q, const void* k_rep, const vo
                                       const int32_t* reps, void* out, int B, int H, int k, int T, int D, float scale,
                                       int causal, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
     using namespace chai;
-    if (dtype != CHAI_BF16 || D != tc::HD)
+    if (dtype != CHAI_BF16 || D != tc::HD || B > 60 * tc::MAX_B)
         return chai_prefill_attention_simt(q, k_rep, v, membership, reps, out, B, H, k, T, D, scale, causal, dtype,
                                            workspace, workspace_bytes, stream);
     int rc = prefill_check_args("chai_prefill_attention", q, k_rep, v, membership, reps, out, B, H, k, T, D, dtype,
@@ -568,29 +680,27 @@ extern "C" int chai_prefill_attention(const void* q, const void* k_rep, const vo
     rc = prefill_run_plan(membership, reps, B, H, k, tc::G, ws, s);
     if (rc != CHAI_OK) return rc;
     const PrefillLayout L = prefill_layout(B, H);
-    cudaError_t e = cudaFuncSetAttribute(tc::prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
-    if (e != cudaSuccess) return cuda_fail(e, "prefill_tc_kernel shared-memory opt-in");
+    static int n_sms = 0;
+    static bool configured = false;
+    if (!configured) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc::prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+        if (e != cudaSuccess) return cuda_fail(e, "prefill_tc_kernel set-up");
+        configured = true;
+    }
     const int n_qtiles = (T + tc::BM - 1) / tc::BM;
-    tc::prefill_tc_kernel<<<dim3(n_qtiles, H, B), tc::THREADS, tc::SMEM_BYTES, s>>>(
-        mq, mk, mv, reinterpret_cast<const int*>(ws + L.off_ngroups),
-        reinterpret_cast<const GroupEntry*>(ws + L.off_groups), static_cast<__nv_bfloat16*>(out),
-        reinterpret_cast<WsHeader*>(ws), H, k, T, scale * 1.4426950408889634f, causal, n_qtiles);
-    CHAI_LAUNCH_CHECK("prefill_tc_kernel launch");
+    // one persistent CTA per SM; requests are processed in chunks of MAX_B (the per-request group counts of
+    // a chunk are kept in shared memory), each chunk with its own work counter in the workspace header
+    for (int b0 = 0, chunk = 0; b0 < B; b0 += tc::MAX_B, ++chunk) {
+        const int nb = B - b0 < tc::MAX_B ? B - b0 : tc::MAX_B;
+        tc::prefill_tc_kernel<<<n_sms, tc::THREADS, tc::SMEM_BYTES, s>>>(
+            mq, mk, mv, reinterpret_cast<const int*>(ws + L.off_ngroups),
+            reinterpret_cast<const GroupEntry*>(ws + L.off_groups), static_cast<__nv_bfloat16*>(out),
+            reinterpret_cast<WsHeader*>(ws), b0, nb, H, k, T, scale * 1.4426950408889634f, causal, n_qtiles, chunk);
+        CHAI_LAUNCH_CHECK("prefill_tc_kernel launch");
+    }
     return CHAI_OK;
-}
-
-// Debugging aid (not part of the public interface): stage timestamps of one CTA of the last tensor-core prefill.
-extern "C" int chai_debug_prefill_ctas(long long* host_out, int max_ctas, int* n_out) {
-    if (host_out == nullptr || n_out == nullptr || max_ctas <= 0 || max_ctas > 4096) return CHAI_ERR_INVALID_ARG;
-    int zero = 0;
-    cudaError_t e = cudaMemcpyFromSymbol(n_out, chai::tc::g_pf_cta_n, sizeof(int));
-    if (e == cudaSuccess) e = cudaMemcpyFromSymbol(host_out, chai::tc::g_pf_cta, sizeof(long long) * 4 * max_ctas);
-    if (e == cudaSuccess) e = cudaMemcpyToSymbol(chai::tc::g_pf_cta_n, &zero, sizeof(int));
-    return e == cudaSuccess ? CHAI_OK : chai::cuda_fail(e, "chai_debug_prefill_ctas");
-}
-
-extern "C" int chai_debug_prefill_stats(long long* host_out) {
-    if (host_out == nullptr) return CHAI_ERR_INVALID_ARG;
-    cudaError_t e = cudaMemcpyFromSymbol(host_out, chai::tc::g_pf_stats, sizeof(long long) * 64 * 8);
-    return e == cudaSuccess ? CHAI_OK : chai::cuda_fail(e, "chai_debug_prefill_stats");
 }
