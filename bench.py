@@ -253,15 +253,15 @@ def bench_prefill(device, peaks, iters=20, warmup=3):
         for _ in range(warmup):
             fn()
         torch.cuda.synchronize()
-        ts = []
+        # calls enqueued back to back, one pair of events around all of them (launch latency overlaps the
+        # previous call, as in a serving loop); every call streams its 168 MB working set again
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         for _ in range(iters):
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
             fn()
-            e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1))
-        res[name] = statistics.median(ts)
+        e1.record()
+        torch.cuda.synchronize()
+        res[name] = e0.elapsed_time(e1) / iters
     fl = prefill_flops(B, H, k, T, D)
     tf = fl / (res["attention"] * 1e-3) / 1e12
     return {

@@ -14,7 +14,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const T* __restrict__ v,
                     const int* __restrict__ n_groups, const GroupEntry* __restrict__ groups, T* __restrict__ out,
-                    int H, int k, int T_len, float scale, int causal, int n_qtiles) {
+                    WsHeader* __restrict__ hdr, const int* __restrict__ bad, int H, int k, int T_len, float scale,
+                    int causal, int n_qtiles) {
     constexpr int DP = D + 1;         // padded row: conflict-free column walks
     constexpr int DPT = D / 4;        // output columns per thread
     extern __shared__ float smem_f[];
@@ -24,6 +25,7 @@ prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const 
     float* Ps = Vs + kSimtBK * D;     // [32][33]
 
     const int b = blockIdx.z, slot = blockIdx.y;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) publish_plan_status(hdr, bad, gridDim.z);
     if (slot >= n_groups[b]) return;
     const int qt = n_qtiles - 1 - (int)blockIdx.x;  // longest (latest) query tiles first
     const GroupEntry e = groups[(size_t)b * H + slot];
@@ -128,15 +130,15 @@ prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const 
 
 template <typename T, int D>
 static int launch_prefill_simt(const void* q, const void* k_rep, const void* v, const int* n_groups,
-                               const GroupEntry* groups, void* out, int B, int H, int k, int T_len, float scale,
-                               int causal, cudaStream_t s) {
+                               const GroupEntry* groups, void* out, WsHeader* hdr, const int* bad, int B, int H, int k,
+                               int T_len, float scale, int causal, cudaStream_t s) {
     const int n_qtiles = (T_len + kSimtBQ - 1) / kSimtBQ;
     const size_t smem = sizeof(float) * ((size_t)kSimtBQ * (D + 1) + (size_t)kSimtBK * (D + 1) + (size_t)kSimtBK * D + 32 * 33);
     cudaError_t e = cudaFuncSetAttribute(prefill_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e, "prefill_simt_kernel shared-memory opt-in");
     prefill_simt_kernel<T, D><<<dim3(n_qtiles, H, B), kSimtThreads, smem, s>>>(
         static_cast<const T*>(q), static_cast<const T*>(k_rep), static_cast<const T*>(v), n_groups, groups,
-        static_cast<T*>(out), H, k, T_len, scale, causal, n_qtiles);
+        static_cast<T*>(out), hdr, bad, H, k, T_len, scale, causal, n_qtiles);
     CHAI_LAUNCH_CHECK("prefill_simt_kernel launch");
     return CHAI_OK;
 }
@@ -152,7 +154,8 @@ int prefill_check_args(const char* fn, const void* q, const void* k_rep, const v
     CHAI_REQUIRE(dtype == CHAI_F32 || dtype == CHAI_BF16, CHAI_ERR_UNSUPPORTED, "%s: unknown dtype %d", fn, dtype);
     CHAI_REQUIRE(D == 64 || D == 128, CHAI_ERR_UNSUPPORTED, "%s: head_dim %d (64 or 128 supported)", fn, D);
     CHAI_REQUIRE(H <= 65535 && B <= 65535, CHAI_ERR_UNSUPPORTED, "%s: H and B must be <= 65535", fn);
-    CHAI_REQUIRE((size_t)(3 * k + H) * sizeof(int) <= 48 * 1024, CHAI_ERR_UNSUPPORTED, "%s: too many heads for the planner", fn);
+    CHAI_REQUIRE((size_t)(2 * k + 2 * H + 4) * sizeof(int) + sizeof(GroupEntry) * (size_t)H <= 48 * 1024, CHAI_ERR_UNSUPPORTED,
+                 "%s: too many heads for the planner", fn);
     const PrefillLayout L = prefill_layout(B, H);
     CHAI_REQUIRE(workspace_bytes >= L.total, CHAI_ERR_WORKSPACE, "%s: workspace has %zu bytes, %zu needed", fn,
                  workspace_bytes, L.total);
@@ -162,11 +165,11 @@ int prefill_check_args(const char* fn, const void* q, const void* k_rep, const v
 int prefill_run_plan(const int32_t* membership, const int32_t* reps, int B, int H, int k, int gmax, char* ws,
                      cudaStream_t s) {
     const PrefillLayout L = prefill_layout(B, H);
-    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(WsHeader), s);
-    if (e != cudaSuccess) return cuda_fail(e, "prefill: clearing the workspace header");
-    prefill_plan_kernel<<<B, 128, sizeof(int) * (size_t)(3 * k + H), s>>>(
-        membership, reps, reinterpret_cast<WsHeader*>(ws), reinterpret_cast<int*>(ws + L.off_ngroups),
-        reinterpret_cast<GroupEntry*>(ws + L.off_groups), H, k, gmax);
+    const size_t smem = sizeof(int) * (size_t)((2 * k + 2 * H + 3) & ~3) + sizeof(GroupEntry) * (size_t)H;
+    prefill_plan_kernel<<<B, 128, smem, s>>>(membership, reps, reinterpret_cast<WsHeader*>(ws),
+                                             reinterpret_cast<int*>(ws + L.off_ngroups),
+                                             reinterpret_cast<int*>(ws + L.off_bad),
+                                             reinterpret_cast<GroupEntry*>(ws + L.off_groups), H, k, gmax);
     CHAI_LAUNCH_CHECK("prefill_plan_kernel launch");
     return CHAI_OK;
 }
@@ -198,12 +201,14 @@ int chai_prefill_attention_simt(const void* q, const void* k_rep, const void* v,
     const PrefillLayout L = prefill_layout(B, H);
     const int* ng = reinterpret_cast<const int*>(ws + L.off_ngroups);
     const GroupEntry* gr = reinterpret_cast<const GroupEntry*>(ws + L.off_groups);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
+    const int* bad = reinterpret_cast<const int*>(ws + L.off_bad);
     if (dtype == CHAI_BF16) {
-        if (D == 128) return launch_prefill_simt<__nv_bfloat16, 128>(q, k_rep, v, ng, gr, out, B, H, k, T, scale, causal, s);
-        return launch_prefill_simt<__nv_bfloat16, 64>(q, k_rep, v, ng, gr, out, B, H, k, T, scale, causal, s);
+        if (D == 128) return launch_prefill_simt<__nv_bfloat16, 128>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, scale, causal, s);
+        return launch_prefill_simt<__nv_bfloat16, 64>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, scale, causal, s);
     }
-    if (D == 128) return launch_prefill_simt<float, 128>(q, k_rep, v, ng, gr, out, B, H, k, T, scale, causal, s);
-    return launch_prefill_simt<float, 64>(q, k_rep, v, ng, gr, out, B, H, k, T, scale, causal, s);
+    if (D == 128) return launch_prefill_simt<float, 128>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, scale, causal, s);
+    return launch_prefill_simt<float, 64>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, scale, causal, s);
 }
 
 }  // extern "C"

@@ -228,7 +228,8 @@ __global__ void __launch_bounds__(THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int* __restrict__ n_groups,
                   const GroupEntry* __restrict__ groups, __nv_bfloat16* __restrict__ out, WsHeader* __restrict__ hdr,
-                  int b_begin, int B, int H, int k, int T_len, float scale_log2, int causal, int n_qtiles, int counter_slot) {
+                  const int* __restrict__ bad, int B_total, int b_begin, int B, int H, int k, int T_len, float scale_log2,
+                  int causal, int n_qtiles, int counter_slot) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw;
@@ -259,6 +260,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             mbar_init(bar.pv_done(i), 1);
         }
         *abort_flag = 0;
+        if (blockIdx.x == 0 && counter_slot == 0) publish_plan_status(hdr, bad, B_total);
         prefix[0] = 0;
         for (int bb = 0; bb < B; ++bb) prefix[bb + 1] = prefix[bb] + n_groups[b_begin + bb];
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -530,22 +532,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_st16(s_addr + half * 32 + 16, packed + 16);
                 l_run = l_run * corr + ((ls0 + ls1) + (ls2 + ls3));
                 m_used = m_new;
-                // the previous tile's PV must be complete before the O accumulators are rescaled
-                if (j > 0) {
+                // Rescaling touches the O accumulators, so the previous tile's P V must be complete first; a warp
+                // whose rows all keep their reference (the usual case after the first tiles) has nothing to wait
+                // for.  Skipping the wait cannot confuse the barrier's phase parity: S of this tile exists, so
+                // every P V up to tile kt - 2 has completed (the tensor core executes in issue order).
+                if (j > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
                     ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done((kt - 1) & 1), ((kt - 1) >> 1) & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
-                    if (__any_sync(0xffffffffu, corr != 1.f)) {  // this thread rescales its 64 columns of each O
-                        for (int g = 0; g < n_members; ++g) {
-                            const uint32_t o_addr = lane_addr + O_COL0 + g * HD + cbase;
-                            tc_ld32(o_addr, r);
-                            tc_ld32(o_addr + 32, r + 32);
-                            tc_wait_ld();
+                    for (int g = 0; g < n_members; ++g) {  // this thread rescales its 64 columns of each O
+                        const uint32_t o_addr = lane_addr + O_COL0 + g * HD + cbase;
+                        tc_ld32(o_addr, r);
+                        tc_ld32(o_addr + 32, r + 32);
+                        tc_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 64; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
-                            tc_st32(o_addr, r);
-                            tc_st32(o_addr + 32, r + 32);
-                        }
+                        for (int i = 0; i < 64; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+                        tc_st32(o_addr, r);
+                        tc_st32(o_addr + 32, r + 32);
                     }
                 }
                 tc_wait_st();          // P (and any rescaled O) is in tensor memory
@@ -699,7 +702,8 @@ extern "C" int chai_prefill_attention(const void* q, const void* k_rep, const vo
         tc::prefill_tc_kernel<<<n_sms, tc::THREADS, tc::SMEM_BYTES, s>>>(
             mq, mk, mv, reinterpret_cast<const int*>(ws + L.off_ngroups),
             reinterpret_cast<const GroupEntry*>(ws + L.off_groups), static_cast<__nv_bfloat16*>(out),
-            reinterpret_cast<WsHeader*>(ws), b0, nb, H, k, T, scale * 1.4426950408889634f, causal, n_qtiles, chunk);
+            reinterpret_cast<WsHeader*>(ws), reinterpret_cast<const int*>(ws + L.off_bad), B, b0, nb, H, k, T,
+            scale * 1.4426950408889634f, causal, n_qtiles, chunk);
         CHAI_LAUNCH_CHECK("prefill_tc_kernel launch");
     }
     return CHAI_OK;
