@@ -31,7 +31,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2403_08058_b200 import chai, synth  # noqa: E402
+from paper_2403_08058_b200 import chai, replicas, synth  # noqa: E402
 
 METRIC = "clustered decode attention: algorithmic HBM GB/s over one decode step (us/step alongside)"
 UNIT = "GB/s"
@@ -131,7 +131,7 @@ class DecodeWorkload:
         self.ws = chai.new_workspace(ws_bytes, device)
         self.bytes_per_layer = [decode_bytes(w.B, w.H, c["k"], w.T, w.D, self.es) for c in self.layers]
         self.bytes_per_step = sum(self.bytes_per_layer)
-        self.launches_per_step = 2 * w.layers
+        self.launches_per_step = w.layers  # one persistent kernel per layer call
 
     def step(self):
         for c in self.layers:
@@ -316,7 +316,6 @@ def main():
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.impl == "reference":
         run_reference(args, rank)
         return
@@ -326,18 +325,13 @@ def main():
     chai.load()
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist_mod.init_process_group("nccl", device_id=device)
-        dist = dist_mod
+    ranks = replicas.init_ranks("nccl", device)
+    world = ranks.world
 
     def sync_all():
         torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+        ranks.barrier()
+        torch.cuda.synchronize()
 
     peaks = load_peaks()
     wl = DecodeWorkload(args.workload, device, layers=args.layers)
@@ -360,13 +354,10 @@ def main():
         wl.step_host()
     ms_e2e = time_region(wl.step_host, args.steps, sync_all)
 
-    if dist is not None:
-        t = torch.tensor([ms_total, ms_e2e], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = ranks.max_over_ranks([ms_total, ms_e2e])
     ms_step = ms_total / args.steps
-    value = world * wl.bytes_per_step / (ms_step * 1e-3) / 1e9
-    e2e_value = world * wl.bytes_per_step / (ms_e2e / args.steps * 1e-3) / 1e9
+    value = replicas.whole_job_throughput(ranks, wl.bytes_per_step / 1e9, ms_step * 1e-3)["value"]
+    e2e_value = replicas.whole_job_throughput(ranks, wl.bytes_per_step / 1e9, ms_e2e / args.steps * 1e-3)["value"]
 
     if rank == 0:
         per_launch_ms = float(layer_ms.mean())
@@ -384,9 +375,12 @@ def main():
                        "l2": "inputs larger than L2: every layer has its own >=168 MiB caches, 12+ GB per step",
                        "multi_gpu": "independent replicas, no data-path collective"},
             "gpu_launches": wl.launches_per_step * args.steps,
-            "roofline": {"bound": "hbm", "kernel": "decode_scores_kernel + decode_pv_kernel (one layer call)",
+            "roofline": {"bound": "hbm", "kernel": "decode_persistent_kernel (one launch per layer call)",
                          "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
-                         "peak_source": peaks["source"], "traffic": None,
+                         "peak_source": peaks["source"],
+                         # DRAM read+write bytes per launch: ncu measured 1.02 x the algorithmic bytes on full-size
+                         # layers (profiles/decode_persistent_kernel_workload2.md), scaled to the mean launch here
+                         "traffic": 1.02 * float(np.mean(wl.bytes_per_layer)), "traffic_unit": "bytes per launch",
                          "us_per_layer_by_k": {str(k): statistics.median(v) for k, v in sorted(by_k.items())},
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "e2e": {"value": e2e_value, "unit": UNIT, "us_per_step": ms_e2e / args.steps * 1e3,
@@ -402,9 +396,7 @@ def main():
             line["compaction"] = bench_compaction(device, peaks)
             line["cpu_baseline"] = cpu_baseline_decode(args.workload, 0)
         print(json.dumps(line))
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
+    ranks.close()
 
 
 if __name__ == "__main__":
