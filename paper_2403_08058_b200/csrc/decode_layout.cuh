@@ -15,8 +15,10 @@ struct DecodeLayout {
     int CK, CV, nK, nV;  // split kernels: rows per key / value chunk and chunks per plane
     int TR;              // persistent kernel: rows per 16 KB tile
     int capK, capV;      // entries per plane reserved for chunk maxima / partials (either implementation)
-    size_t off_counters, off_scores, off_cmax, off_lpart, off_opart, total;
+    size_t off_counters, off_flags, off_scores, off_cmax, off_lpart, off_opart, total;
 };
+
+// off_flags: one 64-bit word per key tile (B * k * capK): carries the launch token once the tile's scores exist
 
 inline bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLayout* L) {
     const int es = (int)elem_size(dtype);
@@ -28,13 +30,15 @@ inline bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLa
     L->nK = (T + L->CK - 1) / L->CK;
     L->nV = (T + L->CV - 1) / L->CV;
     L->TR = kTileBytes / (D * es);
-    // the persistent kernel uses key items of >= 1 tile and value items of >= 4 tiles
-    const int pk = (T + L->TR - 1) / L->TR, pv = (T + 4 * L->TR - 1) / (4 * L->TR);
+    // the persistent kernel deals key work tile by tile and value work in items of 2 tiles
+    const int pk = (T + L->TR - 1) / L->TR, pv = (T + 2 * L->TR - 1) / (2 * L->TR);
     L->capK = pk > L->nK ? pk : L->nK;
     L->capV = pv > L->nV ? pv : L->nV;
     size_t off = sizeof(WsHeader);
     L->off_counters = off;
     off = round_up(off + sizeof(int) * (size_t)B * H, 256);
+    L->off_flags = off;
+    off = round_up(off + sizeof(unsigned long long) * (size_t)B * k * L->capK, 256);
     L->off_scores = off;
     off = round_up(off + sizeof(float) * (size_t)B * k * T, 256);
     L->off_cmax = off;

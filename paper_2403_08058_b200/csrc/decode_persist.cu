@@ -1,50 +1,65 @@
 // Clustered decode attention, persistent streaming kernel (Fig. 3(b), Section 3.4).
 //
-// One CTA per SM, launched cooperatively.  Warp 8 is the producer: it streams the cache rows of this
-// CTA's work, 32 KB tile by tile, into a shared-memory ring with bulk async copies that complete on
+// One CTA per SM (cooperative launch, for co-residency only).  Warp 8 is the producer: it streams cache
+// rows, 32 KB tile by tile, into a shared-memory ring with bulk async copies that complete on
 // mbarriers, and runs ahead of the consumers by the depth of the ring, so HBM stays busy while a
-// consumer does an item's serial prologue and epilogue.  Warps 0..7 consume, each on its own: ring
-// position n belongs to one consumer warp, nothing is synchronised across warps.
+// consumer does the serial part of a tile.  Warps 0..7 consume, each on its own: ring position n
+// belongs to warp n mod 8, nothing is synchronised across the warps of a CTA except item completion.
 //
-//   phase K   unit = one key tile (TR rows of one cluster's K_rep): scaled scores s_t -> workspace
-//             (fp32, stays in L2) and the tile's maximum.  Every K_rep row is read exactly once.
-//   grid-wide barrier (cooperative groups).  The producer has already filled the ring with value
-//             tiles by then.
-//   phase V   unit = item (request, head, IV value tiles) owned by one warp: reference maximum of the
-//             cluster's whole score row, p_t = exp(s_t - max), partial sums (sum p_t V_t, sum p_t)
-//             -> workspace; the warp that completes a head's last item (atomic ticket, nobody waits)
-//             adds the partials in chunk order and writes out = sum / l.
+//   phase K   unit = one key tile (TR rows of one cluster's K_rep), dealt round-robin over CTAs: scaled
+//             scores s_t -> workspace (fp32, stays in L2), the tile's maximum, then the tile's flag word
+//             is set to this launch's token.  Every K_rep row is read exactly once.
+//   phase V   unit = item (request, head, run of IV value tiles), claimed by the producers from an atomic
+//             counter, so fast SMs take more.  A tile waits (almost never in practice: planes complete in
+//             request order) until all flags of its cluster's plane carry the token, takes the plane's
+//             global maximum, forms p_t = exp(s_t - max) and reduces its rows; the warp that finishes an
+//             item's last tile adds the tile partials in tile order and publishes (sum p_t V_t, sum p_t);
+//             the warp that completes a head's last item (atomic ticket, nobody waits) adds the item
+//             partials in chunk order and writes out = sum / l.
 //
-// Units have the same size whatever the cluster sizes and are dealt round-robin over CTAs and warps, so
-// the schedule is static and balanced for skewed memberships too.  The softmax is the exact two-pass
-// form; results do not depend on timing.  Every wait is bounded; on expiry the CTA records
-// CHAI_ERR_TIMEOUT, stops consuming, still joins the grid barrier and returns.
-#include <cooperative_groups.h>
+// There is no grid-wide barrier and no state that must be cleared between launches: flags compare
+// against a token that never repeats, and the few words that must start at zero (work counter, status,
+// tickets) are reset by the warps that own the first key tile of the layer / of a plane, before their
+// flags go up.  The softmax is the exact two-pass form; all sums are taken in a fixed order, so results
+// are bitwise repeatable whatever the schedule.  Every wait is bounded; on expiry the CTA records
+// CHAI_ERR_TIMEOUT, stops consuming and returns.
 #include <stdlib.h>
 
-#include "decode_layout.cuh"
+#include <atomic>
+#include <chrono>
 
-namespace cg = cooperative_groups;
+#include "decode_layout.cuh"
 
 namespace chai {
 namespace pd {
 
-// per-CTA phase timestamps (ns) of the most recent launch: debugging aid read by chai_debug_decode_stats
-__device__ unsigned long long g_cta_stats[1024][4];
-
 constexpr int CONSUMER_WARPS = 8;
-constexpr int CONSUMERS = CONSUMER_WARPS * 32;
-constexpr int THREADS = CONSUMERS + 32;
-constexpr int STAGES = 5;                  // 176 KB of cache rows in flight per SM
+constexpr int THREADS = CONSUMER_WARPS * 32 + 32;
+constexpr int STAGES = 5;                  // 160 KB of cache rows in flight per SM
+constexpr int MAX_IV = 4;                  // tiles per value item
+constexpr int ITEM_SLOTS = 8;              // value items whose tile partials may be open in one CTA
 constexpr int TABLE_CAP = 2048;            // heads whose cluster id is cached in shared memory
 constexpr long long TIMEOUT_CYCLES = 2000000000ll;
 
+struct TileMeta {
+    int item;      // value item id (phase V), -1: end of work for the warp that owns this ring position
+    int t;         // tile index within the item
+    int ntiles;    // real tiles of the item
+    int islot;     // shared-memory slot of the item's tile partials
+};
+
 struct Smem {
     alignas(128) unsigned char ring[STAGES][kTileBytes];
+    alignas(16) float part[ITEM_SLOTS][MAX_IV][128];  // per-tile partial sums of open items
+    float lpart[ITEM_SLOTS][MAX_IV];
     alignas(8) unsigned long long full[STAGES];
     unsigned long long empty[STAGES];
+    TileMeta meta[STAGES];
+    int seq[STAGES];            // sequence number of the tile most recently issued into each slot
+    int item_cnt[ITEM_SLOTS];   // tiles of the open item finished so far
+    int item_free[ITEM_SLOTS];  // 1 when the slot may be given to a new item
     int table[TABLE_CAP];
-    int seq[STAGES];   // sequence number of the tile most recently issued into each slot
+    unsigned ready[TABLE_CAP / 32];  // bit p: every key tile of plane p is known to carry this launch's token
     int abort_flag;
 };
 
@@ -56,16 +71,16 @@ struct Params {
     const int32_t* reps;
     void* out;
     WsHeader* hdr;
-    int* counters;
+    int* counters;               // tickets, one per head
+    unsigned long long* flags;   // one word per key tile
+    unsigned long long token;    // value unique to this launch (never seen in the flags before)
     float* scores;
     float* cmax;
     float* lpart;
     float* opart;
     int B, H, k, T, T_cap;
-    int IK, IV;      // tiles per key / value item
-    int nKi, nVi;    // items per plane
+    int IV, nVi;                 // tiles per value item, items per head
     float scale;
-    int debug;       // bit 0: consumers only drain the ring (streaming-rate experiments; results are garbage)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -89,49 +104,79 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          long long* stall_cycles = nullptr) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    bool done = false;
     while (true) {
-        if (mbar_try_wait(bar, parity)) {
-            done = true;
-            break;
-        }
-        if (*abort_flag) break;
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
         if (clock64() - t0 > TIMEOUT_CYCLES) {
             *abort_flag = 1;
-            break;
+            return false;
         }
     }
-    if (stall_cycles) *stall_cycles += clock64() - t0;
-    return done;
 }
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait until a ring slot carries the tile with sequence number n (see the producer's tagging).
-__device__ __forceinline__ bool seq_wait(const int* seq_word, int n, volatile int* abort_flag, long long* stall_cycles) {
-    const volatile int* w = seq_word;
-    if (*w == n) return true;
+// Bounded wait on a shared-memory word (slot tags, item-slot hand-back).
+__device__ __forceinline__ bool word_wait(const int* word, int want, volatile int* abort_flag) {
+    const volatile int* w = word;
+    if (*w == want) return true;
     const long long t0 = clock64();
-    bool done = false;
     while (true) {
-        if (*w == n) {
-            done = true;
-            break;
-        }
-        if (*abort_flag) break;
+        if (*w == want) return true;
+        if (*abort_flag) return false;
         if (clock64() - t0 > TIMEOUT_CYCLES) {
             *abort_flag = 1;
-            break;
+            return false;
         }
     }
-    if (stall_cycles) *stall_cycles += clock64() - t0;
-    return done;
+}
+// Flag words carry the token of the launch that wrote them.  Tokens come from a host-side counter that
+// never repeats, so whatever earlier launches (or the allocator) left in a flag word cannot be mistaken
+// for "ready".  Bounded wait by ONE thread for one flag ...
+__device__ __forceinline__ bool flag_wait_one(const unsigned long long* flag, unsigned long long token,
+                                              volatile int* abort_flag) {
+    long long t0 = 0;
+    bool first = true;
+    while (true) {
+        unsigned long long v;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(flag) : "memory");
+        if (v == token) return true;
+        if (first) {
+            t0 = clock64();
+            first = false;
+        }
+        if (*abort_flag) return false;
+        if (clock64() - t0 > TIMEOUT_CYCLES) {
+            *abort_flag = 1;
+            return false;
+        }
+        __nanosleep(100);
+    }
+}
+// ... and by a whole warp for `n` consecutive flags.
+__device__ __forceinline__ bool flags_wait(const unsigned long long* flags, int n, unsigned long long token, int lane,
+                                           volatile int* abort_flag) {
+    long long t0 = 0;
+    bool first = true;
+    while (true) {
+        bool all = true;
+        for (int i = lane; i < n; i += 32) {
+            unsigned long long v;
+            asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(flags + i) : "memory");
+            all = all && (v == token);
+        }
+        if (__all_sync(0xffffffffu, all)) return true;
+        if (first) {
+            t0 = clock64();
+            first = false;
+        }
+        const bool give_up = *abort_flag != 0 || clock64() - t0 > TIMEOUT_CYCLES;
+        if (__any_sync(0xffffffffu, give_up)) {
+            *abort_flag = 1;
+            return false;
+        }
+        __nanosleep(100);
+    }
 }
 // 1-D bulk async copy global -> shared, completion counted in bytes on an mbarrier
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -139,11 +184,12 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+
 template <typename T, int D>
 struct Geom {
     static constexpr int EPV = 16 / (int)sizeof(T);   // elements per 16-byte vector
     static constexpr int ROW_BYTES = D * (int)sizeof(T);
-    static constexpr int TR = kTileBytes / ROW_BYTES;  // rows per tile (32, 64 or 128)
+    static constexpr int TR = kTileBytes / ROW_BYTES;  // rows per tile
     static constexpr int LPR = ROW_BYTES / 16;         // lanes per row
     static constexpr int RPW = 32 / LPR;               // rows per warp-wide load
     static constexpr int PV = TR / 32;                 // probabilities per lane per tile
@@ -158,22 +204,6 @@ struct Ring {
     __device__ __forceinline__ uint32_t data(int slot) const { return data0 + kTileBytes * slot; }
 };
 
-// Work decomposition (identical arithmetic on the producer and consumer side).
-//   tp   tiles per cache plane = ceil(T / TR)
-//   phase K: this CTA's key tiles are the global tile ids g = cta, cta + ncta, ...  (g = plane * tp + tile);
-//            its t-th tile has ring sequence number t and belongs to consumer warp t mod W.
-//   phase V: value items (head, chunk of IV tiles), item id i = cta + jc * ncta for the CTA's jc-th item;
-//            item jc belongs to warp jc mod W (its j = jc / W -th item).  The ring interleaves the warps'
-//            tile streams: full rows of W warps first, then the last row of R = NI mod W warps.
-struct Work {
-    int tp, nkt, ni, full_rows, rem;  // tiles/plane, key tiles and value items of this CTA, NI / W, NI % W
-    int IV;
-    __device__ __forceinline__ int vseq(int w, int j, int t) const {  // ring sequence number of a value tile
-        if (j < full_rows) return nkt + (j * IV + t) * CONSUMER_WARPS + w;
-        return nkt + full_rows * IV * CONSUMER_WARPS + t * rem + w;
-    }
-};
-
 template <typename T, int D>
 __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Params P) {
     using G = Geom<T, D>;
@@ -186,22 +216,11 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
     const Ring ring{smem_u32(&sm.full[0]), smem_u32(&sm.empty[0]), smem_u32(&sm.ring[0][0])};
     const int B = P.B, H = P.H, k = P.k, T_len = P.T;
     const bool use_table = B * H <= TABLE_CAP;
-    Work wk;
-    wk.tp = (T_len + G::TR - 1) / G::TR;
-    wk.IV = P.IV;
-    {
-        const long long kt = (long long)B * k * wk.tp, vi = (long long)B * H * P.nVi;
-        wk.nkt = (int)((kt - cta + ncta - 1) / ncta);
-        wk.ni = (int)((vi - cta + ncta - 1) / ncta);
-        if (wk.nkt < 0) wk.nkt = 0;
-        if (wk.ni < 0) wk.ni = 0;
-        wk.full_rows = wk.ni / W;
-        wk.rem = wk.ni % W;
-    }
-    // timing breadcrumbs of CTA 0 (debugging aid): header words 16.. as 64-bit values
-    unsigned long long* stats = reinterpret_cast<unsigned long long*>(&P.hdr->pad[1]);
-    if (cta == 0 && tid == 0) stats[0] = global_ns();
-    if (tid == 0 && cta < 1024) g_cta_stats[cta][0] = global_ns();
+    const int tp = (T_len + G::TR - 1) / G::TR;          // tiles per cache plane
+    const long long n_ktiles = (long long)B * k * tp;    // key tiles of the layer
+    const int nkt = n_ktiles > cta ? (int)((n_ktiles - cta + ncta - 1) / ncta) : 0;  // this CTA's share
+    const int n_items = B * H * P.nVi;                   // value items of the layer
+    int* work_counter = &P.hdr->pad[0];
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -209,17 +228,15 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
             mbar_init(ring.empty(s), 1);
             sm.seq[s] = -1;
         }
+        for (int s = 0; s < ITEM_SLOTS; ++s) {
+            sm.item_cnt[s] = 0;
+            sm.item_free[s] = 1;
+        }
+        for (int i = 0; i < TABLE_CAP / 32; ++i) sm.ready[i] = 0;
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    // housekeeping for phase V (ordered by the grid barrier): tickets, status word, head table
-    if (cta == 0 && tid == 0) {
-        P.hdr->status = CHAI_OK;
-        P.hdr->bad_b = -1;
-        P.hdr->bad_h = -1;
-    }
-    for (int i = cta * THREADS + tid; i < B * H; i += ncta * THREADS) P.counters[i] = 0;
     if (use_table) {
         for (int i = tid; i < B * H; i += THREADS) {
             int c, r;
@@ -227,127 +244,97 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
         }
     }
     __syncthreads();
-
+    auto cluster_of = [&](int b, int h) -> int {
+        if (use_table) return sm.table[b * H + h];
+        int c, r;
+        return resolve_head(P.membership, P.reps, b, h, H, k, &c, &r) ? c : -1;
+    };
+    auto tile_rows = [&](int tile) { return max(0, min(G::TR, T_len - tile * G::TR)); };
     const unsigned char* kc = static_cast<const unsigned char*>(P.k_rep);
     const unsigned char* vc = static_cast<const unsigned char*>(P.v);
-    auto tile_rows = [&](int tile) { return max(0, min(G::TR, T_len - tile * G::TR)); };
 
     if (warp == W) {
-        // ------------------------------ producer warp ------------------------------
-        // Tiles are issued in strict ring order (ascending sequence number), which keeps the one-bit phase
-        // parity of the slot barriers unambiguous on the producer side.  The loop control is uniform over
-        // the warp; lane w (< W) keeps the addresses of consumer warp w's stream and is the one lane that
-        // waits for the slot and issues when a tile of that stream is due, so the address arithmetic of
-        // the W streams runs in parallel and a tile costs the warp a few dozen instructions.
-        long long stall_k = 0, stall_v = 0;
-        int n = 0, slot = 0;
-        uint32_t parity = 1;  // parity to wait for on empty[slot]: ((n / STAGES) & 1) ^ 1
-        auto next_slot = [&]() {
-            ++n;
-            if (++slot == STAGES) {
-                slot = 0;
-                parity ^= 1u;
-            }
-        };
-        auto emit = [&](const unsigned char* base, int plane, int tile) {
-            const int rows = tile_rows(tile);
-            // Consumer warps run independently and bulk copies complete out of order, so a consumer may
-            // reach this slot while the previous occupant's copy is still in flight; the one-bit phase
-            // parity of the full barrier cannot tell those two fills apart.  The tag can: a consumer first
-            // waits until the slot is tagged with its own sequence number (the previous occupant has then
-            // been consumed, hence its phase completed) and only then waits on the barrier.
-            *reinterpret_cast<volatile int*>(&sm.seq[slot]) = n;
-            if (rows > 0) {
-                const uint32_t bytes = (uint32_t)rows * G::ROW_BYTES;
-                mbar_expect_tx(ring.full(slot), bytes);
-                bulk_load(ring.data(slot), base + ((size_t)plane * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES, bytes,
-                          ring.full(slot));
-            } else {
-                mbar_arrive(ring.full(slot));  // padding tile past the end of the cache: nothing to copy
-            }
-        };
-        // ---- key tiles: tile t of this CTA belongs to stream t mod W ----
-        bool ok = true;
-        {
-            const long long g = (long long)cta + (long long)lane * ncta;  // meaningful for lanes < W
-            int kplane = (int)(g / wk.tp), ktile = (int)(g % wk.tp);
-            const int dplane = (int)(((long long)W * ncta) / wk.tp), dtile = (int)(((long long)W * ncta) % wk.tp);
-            int w = 0;
-            for (int t = 0; t < wk.nkt && ok; ++t) {
-                int res = 1;
-                if (lane == w) {
-                    res = mbar_wait(ring.empty(slot), parity, abort_flag, &stall_k) ? 1 : 0;
-                    if (res) {
-                        emit(kc, kplane, ktile);
-                        kplane += dplane;
-                        ktile += dtile;
-                        if (ktile >= wk.tp) {
-                            ktile -= wk.tp;
-                            ++kplane;
-                        }
-                    }
+        // ------------------------------ producer (one thread) ------------------------------
+        // Tiles are issued in ring order (ascending sequence number): that keeps the one-bit phase parity
+        // of the slot barriers unambiguous on this side.  Consumer warps run independently and bulk copies
+        // complete out of order, so a consumer may reach a slot while the previous occupant's copy is
+        // still in flight; the parity of the full barrier cannot tell those two fills apart, the slot's
+        // sequence tag can: a consumer waits for its own sequence number in the tag (the previous occupant
+        // has then been consumed, hence its phase completed) before it waits on the barrier.
+        if (lane == 0) {
+            int n = 0, slot = 0;
+            uint32_t parity = 1;  // parity to wait for on empty[slot]: ((n / STAGES) & 1) ^ 1
+            bool ok = true;
+            auto issue = [&](const unsigned char* src, uint32_t bytes, const TileMeta& m) -> bool {
+                if (!mbar_wait(ring.empty(slot), parity, abort_flag)) return false;
+                sm.meta[slot] = m;
+                __threadfence_block();
+                *reinterpret_cast<volatile int*>(&sm.seq[slot]) = n;
+                if (bytes > 0) {
+                    mbar_expect_tx(ring.full(slot), bytes);
+                    bulk_load(ring.data(slot), src, bytes, ring.full(slot));
+                } else {
+                    mbar_arrive(ring.full(slot));  // marker without data
                 }
-                ok = __shfl_sync(0xffffffffu, res, w) != 0;
-                next_slot();
-                if (++w == W) w = 0;
-            }
-        }
-        // ---- value tiles: row j of items (one per stream), tile t of each, streams in order ----
-        int j = 0, t = 0, w = 0, vplane = 0, vtile0 = 0;
-        bool loaded = false;
-        const int last_row = wk.rem > 0 ? wk.full_rows : wk.full_rows - 1;
-        // returns 1 when every tile has been issued, 0 when a non-blocking probe found the slot busy, -1 on expiry
-        auto pump_values = [&](bool blocking) -> int {
-            while (j <= last_row) {
-                const int nact = j < wk.full_rows ? W : wk.rem;
-                if (!loaded) {  // every stream looks up its item of this row at once
-                    if (lane < nact) {
-                        const long long item = (long long)cta + (long long)(lane + j * W) * ncta;
-                        vplane = (int)(item / P.nVi);
-                        vtile0 = (int)(item % P.nVi) * wk.IV;
-                    }
-                    loaded = true;
+                ++n;
+                if (++slot == STAGES) {
+                    slot = 0;
+                    parity ^= 1u;
                 }
-                int res = 1;
-                if (lane == w) {
-                    if (blocking)
-                        res = mbar_wait(ring.empty(slot), parity, abort_flag, &stall_v) ? 1 : -1;
-                    else
-                        res = mbar_try_wait(ring.empty(slot), parity) ? 1 : 0;
-                    if (res == 1) emit(vc, vplane, vtile0 + t);
-                }
-                res = __shfl_sync(0xffffffffu, res, w);
-                if (res != 1) return res;
-                next_slot();
-                if (++w == nact) {
-                    w = 0;
-                    if (++t == wk.IV) {
-                        t = 0;
-                        ++j;
-                        loaded = false;
+                return true;
+            };
+            // ---- key tiles: global tile ids cta, cta + ncta, ... ----
+            {
+                int plane = cta / tp, tile = cta % tp;
+                const int dplane = ncta / tp, dtile = ncta % tp;
+                const TileMeta m{0, 0, 0, 0};
+                for (int t = 0; t < nkt && ok; ++t) {
+                    ok = issue(kc + ((size_t)plane * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
+                               (uint32_t)tile_rows(tile) * G::ROW_BYTES, m);
+                    plane += dplane;
+                    tile += dtile;
+                    if (tile >= tp) {
+                        tile -= tp;
+                        ++plane;
                     }
                 }
             }
-            return 1;
-        };
-        // before the grid barrier value tiles only go into slots that are already free: the consumers
-        // release value slots after the barrier, so a blocking wait here could never be satisfied
-        const int r1 = ok ? pump_values(false) : -1;
-        cg::this_grid().sync();
-        if (r1 == 0) pump_values(true);
-        if (cta == 0 && lane == 0) {
-            stats[4] = (unsigned long long)stall_k;
-            stats[5] = (unsigned long long)stall_v;
+            // ---- value items, claimed one at a time; the next claim is in flight while this item streams ----
+            // (the work counter is reset by the owner of the layer's first key tile before that tile's flag)
+            if (ok) ok = flag_wait_one(P.flags, P.token, abort_flag);
+            int n_open = 0;  // items this CTA has opened (item slots are handed out round-robin)
+            int next = ok ? atomicAdd(work_counter, 1) : n_items;
+            while (ok && next < n_items) {
+                const int item = next;
+                next = atomicAdd(work_counter, 1);
+                const int head = item / P.nVi, chunk = item % P.nVi;
+                const int tile0 = chunk * P.IV;
+                const int ntiles = min(P.IV, tp - tile0);
+                const int islot = n_open % ITEM_SLOTS;
+                ++n_open;
+                ok = word_wait(&sm.item_free[islot], 1, abort_flag);  // the slot's previous item is fully reduced
+                if (!ok) break;
+                *reinterpret_cast<volatile int*>(&sm.item_free[islot]) = 0;
+                for (int t = 0; t < ntiles && ok; ++t) {
+                    const int tile = tile0 + t;
+                    const TileMeta m{item, t, ntiles, islot};
+                    ok = issue(vc + ((size_t)head * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
+                               (uint32_t)tile_rows(tile) * G::ROW_BYTES, m);
+                }
+            }
+            // ---- one end marker per consumer warp ----
+            const TileMeta end{-1, 0, 0, 0};
+            for (int w = 0; w < W && ok; ++w) ok = issue(nullptr, 0, end);
         }
     } else {
         // ------------------------------ consumers: every warp works alone ------------------------------
         const int sub = lane / G::LPR, part = lane % G::LPR;
         bool ok = true;
-        long long stall_c = 0;
+        int n = warp;  // this warp owns ring positions warp, warp + W, ...
         // ---- phase K: one tile = TR scores and their maximum ----
-        for (int t = warp; t < wk.nkt; t += W) {
-            const long long g = (long long)cta + (long long)t * ncta;
-            const int plane = (int)(g / wk.tp), tile = (int)(g % wk.tp);
+        for (; n < nkt; n += W) {
+            const long long g = (long long)cta + (long long)n * ncta;
+            const int plane = (int)(g / tp), tile = (int)(g % tp);
             const int b = plane / k;
             const int rows = tile_rows(tile);
             const int rep = P.reps[plane];
@@ -359,10 +346,10 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                 const uint4 qv = *reinterpret_cast<const uint4*>(static_cast<const T*>(P.q) + ((size_t)b * H + rep) * D + part * G::EPV);
                 Vec16<T>::unpack(qv, qf);
             }
-            const int slot = t % STAGES;
-            if (ok) ok = __all_sync(0xffffffffu, seq_wait(&sm.seq[slot], t, abort_flag, &stall_c) &&
-                                                     mbar_wait(ring.full(slot), (t / STAGES) & 1, abort_flag, &stall_c));
-            if (ok && live && !(P.debug & 1)) {
+            const int slot = n % STAGES;
+            if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag) &&
+                                                     mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
+            if (ok && live) {
                 const unsigned char* data = sm.ring[slot];
                 float* srow = P.scores + (size_t)plane * T_len + (size_t)tile * G::TR;
                 float lmax = -INFINITY;
@@ -406,75 +393,78 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                 }
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) lmax = fmaxf(lmax, __shfl_xor_sync(0xffffffffu, lmax, o));
-                if (lane == 0) P.cmax[(size_t)plane * wk.tp + tile] = lmax;
+                if (lane == 0) P.cmax[(size_t)plane * tp + tile] = lmax;
             }
             __syncwarp();
             if (lane == 0 && ok) mbar_arrive(ring.empty(slot));
+            if (ok) {
+                if (g == 0 && lane == 0) {  // first key tile of the layer: reset status and work counter before its flag
+                    P.hdr->status = CHAI_OK;
+                    P.hdr->bad_b = -1;
+                    P.hdr->bad_h = -1;
+                    *work_counter = 0;
+                }
+                // the warp that owns tile 0 of a plane also clears the tickets of the plane's heads: every value
+                // tile of those heads waits for all of the plane's flags, this tile's included
+                if (tile == 0 && live) {
+                    const int c = plane % k;
+                    for (int h = lane; h < H; h += 32)
+                        if (cluster_of(b, h) == c) P.counters[(size_t)b * H + h] = 0;
+                }
+                __syncwarp();
+                if (lane == 0)
+                    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(P.flags + (size_t)plane * tp + tile), "l"(P.token) : "memory");
+            }
         }
-        if (cta == 0 && tid == 0) {
-            stats[1] = global_ns();
-            stats[6] = (unsigned long long)stall_c;
-        }
-        if (tid == 0 && cta < 1024) g_cta_stats[cta][1] = global_ns();
-        cg::this_grid().sync();
-        if (cta == 0 && tid == 0) stats[2] = global_ns();
-        if (tid == 0 && cta < 1024) g_cta_stats[cta][2] = global_ns();
-        // ---- phase V: one item = IV tiles of one head; partial sums; combine by the last arriver ----
+        // ---- phase V: tiles of claimed items ----
         T* outp = static_cast<T*>(P.out);
-        for (int j = 0;; ++j) {
-            const int jc = warp + j * W;
-            if (jc >= wk.ni) break;
-            const long long item = (long long)cta + (long long)jc * ncta;
-            const int head = (int)(item / P.nVi), chunk = (int)(item % P.nVi);
+        for (;; n += W) {
+            const int slot = n % STAGES;
+            if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag) &&
+                                                     mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
+            if (!ok) break;
+            const TileMeta m = sm.meta[slot];
+            if (m.item < 0) {  // end marker
+                __syncwarp();
+                if (lane == 0) mbar_arrive(ring.empty(slot));
+                break;
+            }
+            const int head = m.item / P.nVi, chunk = m.item % P.nVi;
             const int b = head / H, h = head % H;
-            int c;
-            if (use_table) {
-                c = sm.table[head];
-            } else {
-                int rr;
-                c = resolve_head(P.membership, P.reps, b, h, H, k, &c, &rr) ? c : -1;
-            }
+            const int tile = chunk * P.IV + m.t;
+            const int rows = tile_rows(tile);
+            const int c = cluster_of(b, h);
             const bool live = c >= 0;
-            const size_t plane = (size_t)b * k + (live ? c : 0);
-            float m = -INFINITY;
-            if (live) {
-                for (int x = lane; x < wk.tp; x += 32) m = fmaxf(m, __ldcg(&P.cmax[plane * wk.tp + x]));
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            } else if (chunk == 0) {
-                if (lane == 0) flag_bad_membership(P.hdr, b, h);
-                for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<T>(0.f);
-            }
             float acc[G::EPV];
 #pragma unroll
             for (int e = 0; e < G::EPV; ++e) acc[e] = 0.f;
             float lsum = 0.f;
-            const float* srow = P.scores + plane * T_len;
-            float sraw[G::PV];  // raw scores of the next tile, fetched one tile ahead
-            auto fetch_scores = [&](int tile) {
-                const int rows = tile_rows(tile);
-#pragma unroll
-                for (int u = 0; u < G::PV; ++u) {
-                    const int r = u * 32 + lane;
-                    sraw[u] = (live && r < rows) ? __ldcg(&srow[(size_t)tile * G::TR + r]) : -INFINITY;
+            if (live) {
+                const size_t plane = (size_t)b * k + c;
+                // all scores of the plane must exist; once seen, remembered per CTA (planes complete in order, so
+                // after the first tiles of phase V this is a shared-memory bit test)
+                const bool cached = plane < TABLE_CAP && ((*reinterpret_cast<volatile unsigned*>(&sm.ready[plane >> 5]) >> (plane & 31)) & 1u);
+                if (!cached) {
+                    ok = flags_wait(P.flags + plane * tp, tp, P.token, lane, abort_flag);
+                    if (ok && lane == 0 && plane < TABLE_CAP) atomicOr(&sm.ready[plane >> 5], 1u << (plane & 31));
                 }
-            };
-            fetch_scores(chunk * wk.IV);
-            for (int t = 0; t < wk.IV; ++t) {
-                const int tile = chunk * wk.IV + t;
-                const int rows = tile_rows(tile);
-                float pv[G::PV];
+                if (ok) {
+                    float mx = -INFINITY;
+                    for (int x = lane; x < tp; x += 32) mx = fmaxf(mx, __ldcg(&P.cmax[plane * tp + x]));
+                    const float* srow = P.scores + plane * T_len + (size_t)tile * G::TR;
+                    float pv[G::PV];
 #pragma unroll
-                for (int u = 0; u < G::PV; ++u) {
-                    pv[u] = sraw[u] == -INFINITY ? 0.f : expf(sraw[u] - m);
-                    lsum += pv[u];
-                }
-                if (t + 1 < wk.IV) fetch_scores(tile + 1);
-                const int n = wk.vseq(warp, j, t);
-                const int slot = n % STAGES;
-                if (ok) ok = __all_sync(0xffffffffu, seq_wait(&sm.seq[slot], n, abort_flag, &stall_c) &&
-                                                         mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag, &stall_c));
-                if (ok && live && rows > 0 && !(P.debug & 1)) {
+                    for (int u = 0; u < G::PV; ++u) {
+                        const int r = u * 32 + lane;
+                        pv[u] = r < rows ? __ldcg(&srow[r]) : -INFINITY;
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+#pragma unroll
+                    for (int u = 0; u < G::PV; ++u) {
+                        pv[u] = pv[u] == -INFINITY ? 0.f : expf(pv[u] - mx);
+                        lsum += pv[u];
+                    }
                     const unsigned char* data = sm.ring[slot];
                     if (rows == G::TR) {
 #pragma unroll
@@ -509,11 +499,16 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                         }
                     }
                 }
-                __syncwarp();
-                if (lane == 0 && ok) mbar_arrive(ring.empty(slot));
+            } else if (chunk == 0 && m.t == 0) {
+                // unresolved head: zero output, flagged after the status reset (ordered by the layer's first flag)
+                ok = flags_wait(P.flags, 1, P.token, lane, abort_flag);
+                if (ok && lane == 0) flag_bad_membership(P.hdr, b, h);
+                for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<T>(0.f);
             }
-            if (!live || !ok) continue;  // warp-uniform
-            // fold the RPW row slots of the warp; lanes 0..LPR-1 then hold the head's D partial sums
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ring.empty(slot));  // the tile's bytes are no longer needed
+            if (!ok) break;
+            // fold the RPW row slots of the warp; lanes 0..LPR-1 then hold the tile's D partial sums
 #pragma unroll
             for (int o = G::LPR; o < 32; o <<= 1) {
 #pragma unroll
@@ -521,22 +516,47 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, o);
-            float* op = P.opart + ((size_t)head * P.nVi + chunk) * D;
             if (lane < G::LPR) {
 #pragma unroll
-                for (int e = 0; e < G::EPV; e += 4)
-                    *reinterpret_cast<float4*>(op + part * G::EPV + e) = make_float4(acc[e], acc[e + 1], acc[e + 2], acc[e + 3]);
+                for (int e = 0; e < G::EPV; ++e) sm.part[m.islot][m.t][part * G::EPV + e] = acc[e];
             }
-            if (lane == 0) P.lpart[(size_t)head * P.nVi + chunk] = lsum;
+            if (lane == 0) sm.lpart[m.islot][m.t] = lsum;
+            __threadfence_block();
+            __syncwarp();
+            int done = 0;
+            if (lane == 0) done = atomicAdd(&sm.item_cnt[m.islot], 1);
+            done = __shfl_sync(0xffffffffu, done, 0);
+            if (done != m.ntiles - 1) continue;
+            // this warp finished the item's last open tile: add the tile partials in tile order
+            __threadfence_block();
+            constexpr int DPL = D / 32;  // output columns per lane
+            float o[DPL];
+#pragma unroll
+            for (int e = 0; e < DPL; ++e) o[e] = 0.f;
+            float l = 0.f;
+            for (int t = 0; t < m.ntiles; ++t) {
+#pragma unroll
+                for (int e = 0; e < DPL; ++e) o[e] += *reinterpret_cast<volatile float*>(&sm.part[m.islot][t][lane * DPL + e]);
+                l += *reinterpret_cast<volatile float*>(&sm.lpart[m.islot][t]);
+            }
+            __syncwarp();
+            if (lane == 0) {
+                sm.item_cnt[m.islot] = 0;
+                __threadfence_block();
+                *reinterpret_cast<volatile int*>(&sm.item_free[m.islot]) = 1;  // hand the slot back to the producer
+            }
+            if (!live) continue;
+            float* op = P.opart + ((size_t)head * P.nVi + chunk) * D;
+#pragma unroll
+            for (int e = 0; e < DPL; ++e) op[lane * DPL + e] = o[e];
+            if (lane == 0) P.lpart[(size_t)head * P.nVi + chunk] = l;
             __threadfence();
             __syncwarp();
             int ticket = 0;
             if (lane == 0) ticket = atomicAdd(&P.counters[head], 1);
             ticket = __shfl_sync(0xffffffffu, ticket, 0);
-            if (ticket == P.nVi - 1) {  // this warp completed the head: add the partials in chunk order
+            if (ticket == P.nVi - 1) {  // this warp completed the head: add the item partials in chunk order
                 __threadfence();
-                constexpr int DPL = D / 32;  // output columns per lane
-                float o[DPL];
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) o[e] = 0.f;
                 float ll = 0.f;
@@ -550,11 +570,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                 for (int e = 0; e < DPL; ++e) outp[(size_t)head * D + lane * DPL + e] = from_float<T>(o[e] / ll);
             }
         }
-        if (cta == 0 && tid == 0) stats[7] = (unsigned long long)stall_c;
     }
-    if (cta == 0 && tid == 0) stats[3] = global_ns();
     __syncthreads();
-    if (tid == 0 && cta < 1024) g_cta_stats[cta][3] = global_ns();
     if (tid == 0 && sm.abort_flag) atomicExch(&P.hdr->status, CHAI_ERR_TIMEOUT);
 }
 
@@ -591,6 +608,7 @@ static int launch(const Params& P0, int ncta, int dev, cudaStream_t s) {
         configured = true;
     }
     void* args[] = {&P};
+    // cooperative launch: value tiles wait for flags set by other CTAs, so all CTAs must be resident at once
     cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_persistent_kernel<T, D>), dim3(ncta),
                                                 dim3(THREADS), args, smem, s);
     if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel launch");
@@ -612,25 +630,24 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     P.q = q; P.k_rep = k_rep; P.v = v; P.membership = membership; P.reps = reps; P.out = out;
     P.hdr = reinterpret_cast<WsHeader*>(ws);
     P.counters = reinterpret_cast<int*>(ws + L.off_counters);
+    P.flags = reinterpret_cast<unsigned long long*>(ws + L.off_flags);
     P.scores = reinterpret_cast<float*>(ws + L.off_scores);
     P.cmax = reinterpret_cast<float*>(ws + L.off_cmax);
     P.lpart = reinterpret_cast<float*>(ws + L.off_lpart);
     P.opart = reinterpret_cast<float*>(ws + L.off_opart);
+    {
+        // launch tokens never repeat within a process and start from a time-dependent value, so stale flag
+        // words (earlier launches, other processes, fresh allocations) cannot look like "ready"
+        static std::atomic<unsigned long long> counter{
+            (unsigned long long)std::chrono::steady_clock::now().time_since_epoch().count() * 2654435761ull + 0x9E3779B97F4A7C15ull};
+        P.token = counter.fetch_add(1) + 1;
+    }
     P.B = B; P.H = H; P.k = k; P.T = T; P.T_cap = T_cap;
-    // key work is dealt tile by tile; value items are runs of 4 tiles of one head (one consumer warp each)
-    P.IK = 1;
-    P.IV = tiles < 4 ? tiles : 4;
-    P.nKi = tiles;
+    // key work is dealt tile by tile; value items are runs of up to 4 tiles of one head
+    P.IV = tiles < pd::MAX_IV ? tiles : pd::MAX_IV;
     P.nVi = (tiles + P.IV - 1) / P.IV;
     P.scale = scale;
-    {
-        static const int dbg = [] {
-            const char* e = getenv("CHAI_DECODE_DEBUG");
-            return e ? atoi(e) : 0;
-        }();
-        P.debug = dbg;
-    }
-    if (P.nKi > L.capK || P.nVi > L.capV) return kDecodeNotLaunched;
+    if (tiles > L.capK || P.nVi > L.capV || (long long)B * H * P.nVi > 0x7fffffffll) return kDecodeNotLaunched;
     if (dtype == CHAI_BF16) {
         if (D == 128) return pd::launch<__nv_bfloat16, 128>(P, ncta, dev, s);
         return pd::launch<__nv_bfloat16, 64>(P, ncta, dev, s);
@@ -640,10 +657,3 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
 }
 
 }  // namespace chai
-
-// Debugging aid (not part of the public interface): per-CTA phase timestamps of the last persistent launch.
-extern "C" int chai_debug_decode_stats(unsigned long long* host_out, int n_ctas) {
-    if (host_out == nullptr || n_ctas <= 0 || n_ctas > 1024) return CHAI_ERR_INVALID_ARG;
-    cudaError_t e = cudaMemcpyFromSymbol(host_out, chai::pd::g_cta_stats, sizeof(unsigned long long) * 4 * n_ctas);
-    return e == cudaSuccess ? CHAI_OK : chai::cuda_fail(e, "chai_debug_decode_stats");
-}
