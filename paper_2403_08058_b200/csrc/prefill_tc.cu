@@ -3,8 +3,8 @@
 // One CTA = (request, member group of <= 2 heads of one cluster, tile of 128 query rows).  The
 // representative's Q tile and K tiles and the members' V tiles arrive by TMA (128-byte swizzle);
 // S = Q K^T and O_g += P V_g are tcgen05.mma instructions issued by one thread with fp32
-// accumulators in tensor memory (two S buffers of 128 columns, one O accumulator of 128 columns
-// per member: 512 columns).  Four warps own one query row per thread: they read S from tensor
+// accumulators in tensor memory (one S buffer of 128 columns, two P buffers of 64 columns, one O
+// accumulator of 128 columns per member: 512 columns).  Four warps own one query row per thread: they read S from tensor
 // memory, keep the running maximum and sum of the softmax (rescaling O only when the maximum grew
 // by more than 2^8, which leaves the result exact because p and l use the same reference), write
 // P as bf16 into shared memory in the operand layout, and at the end scale O by 1/l and store it.
@@ -40,7 +40,7 @@ constexpr int SOFTMAX_WARPS = 8;    // two per TMEM lane quadrant: each thread o
 constexpr int EPILOGUE_WARPS = 4;   // one thread per query row: O / l -> bf16 -> global while the next item computes
 constexpr int THREADS = 64 + (SOFTMAX_WARPS + EPILOGUE_WARPS) * 32;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t S_COL0 = 0, O_COL0 = 256;   // S buffers at columns 0 and 128, O_g at 256 + 128 g
+constexpr uint32_t S_COL0 = 0, P_COL0 = 128, O_COL0 = 256;  // S at 0..127, P buffers at 128 + 64 i, O_g at 256 + 128 g
 constexpr long long TIMEOUT_CYCLES = 2000000000ll;  // about a second
 
 // shared memory map (offsets from a 1024-byte aligned base)
@@ -48,7 +48,7 @@ constexpr int OFF_Q = 0;
 constexpr int OFF_K = OFF_Q + TILE_BYTES;
 constexpr int OFF_V = OFF_K + KST * TILE_BYTES;
 constexpr int OFF_BAR = OFF_V + VST * TILE_BYTES;
-constexpr int NUM_BARS = 18;
+constexpr int NUM_BARS = 19;
 constexpr int OFF_XCH = OFF_BAR + 8 * NUM_BARS + 16;               // after the barriers and the tmem slot / abort word
 constexpr int XCH_BYTES = 2 * BM * 4;                              // row maxima exchanged between the two halves
 constexpr int OFF_LSUM = OFF_XCH + XCH_BYTES;                      // row sums handed to the epilogue warps
@@ -206,8 +206,9 @@ struct Bars {
     __device__ __forceinline__ uint32_t pv_done(int i) const { return base + 8 * (14 + i); }
     __device__ __forceinline__ uint32_t epi_full() const { return base + 8 * 16; }
     __device__ __forceinline__ uint32_t epi_empty() const { return base + 8 * 17; }
+    __device__ __forceinline__ uint32_t s_free() const { return base + 8 * 18; }
 };
-static_assert(NUM_BARS == 18, "barrier count");
+static_assert(NUM_BARS == 19, "barrier count");
 
 // One unit of work, published by the producer to the other roles through shared memory.
 struct Item {
@@ -250,6 +251,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         mbar_init(bar.o_free(), EPILOGUE_WARPS * 32);
         mbar_init(bar.epi_full(), SOFTMAX_WARPS * 32);
         mbar_init(bar.epi_empty(), EPILOGUE_WARPS * 32);
+        mbar_init(bar.s_free(), SOFTMAX_WARPS * 32);
         mbar_init(bar.p_full(), SOFTMAX_WARPS * 32);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar.item_full(i), 1);
@@ -376,12 +378,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     continue;
                 }
                 ok = mbar_wait(bar.q_full(), qi & 1, abort_flag);
-                // S(tile kt) = Q K^T into S buffer kt & 1
+                // S(tile kt) = Q K^T into the S buffer, once the softmax warps hold the previous tile's scores in registers
                 auto issue_qk = [&](bool last) -> bool {
                     const int ts = kt & 1;
                     if (!mbar_wait(bar.k_full(ts), (kt >> 1) & 1, abort_flag)) return false;
+                    if (kt > 0 && !mbar_wait(bar.s_free(), (kt - 1) & 1, abort_flag)) return false;
                     tc_fence_after();
-                    const uint32_t d = tmem_base + S_COL0 + ts * BN;
+                    const uint32_t d = tmem_base + S_COL0;
                     const uint32_t kb = k_lo + ts * (TILE_BYTES >> 4);
 #pragma unroll
                     for (int s = 0; s < HD / 16; ++s) {
@@ -403,7 +406,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (ok && j == 0 && qi > 0) ok = mbar_wait(bar.o_free(), (qi - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t p_addr = tmem_base + S_COL0 + ts * BN;  // P: first 64 columns of its S buffer
+                    const uint32_t p_addr = tmem_base + P_COL0 + ts * 64;  // P buffer of this tile
                     for (int g = 0; g < n_members; ++g) {
                         const uint32_t d = tmem_base + O_COL0 + g * HD;
                         const uint32_t vb = v_lo + (ts * G + g) * (TILE_BYTES >> 4);
@@ -421,8 +424,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // ---------------- softmax / correction: two threads per query row ----------------
         // Warps 2..5 own columns 0..63 of their rows, warps 6..9 columns 64..127; the two threads of a row
         // sit in different warps of the same TMEM lane quadrant and meet once per tile at a 64-thread
-        // named barrier, where they exchange their half-row maxima.  By then both have their 64 scores in
-        // registers, so writing P over the S buffer afterwards cannot clobber anything still needed.
+        // named barrier, where they exchange their half-row maxima.
         const int quad = warp & 3;               // TMEM lanes this warp may touch
         const int half = (warp - 2) >> 2;        // which 64 columns of the tile
         const int row = quad * 32 + lane;        // row of the tile
@@ -461,7 +463,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 ok = __all_sync(0xffffffffu, mbar_wait(bar.qk_done(sb), (kt >> 1) & 1, abort_flag));
                 if (!ok) break;  // warp-uniform: the tcgen05 loads below are warp-collective
                 tc_fence_after();
-                const uint32_t s_addr = lane_addr + S_COL0 + sb * BN;
+                const uint32_t s_addr = lane_addr + S_COL0;
+                const uint32_t p_st = lane_addr + P_COL0 + sb * 64 + half * 32;  // this thread's 32 columns of P(kt)
                 const int col0 = j * BN;
                 // columns of this thread's half that the row may see: col_abs < T and (causal: col_abs <= row_abs)
                 int vis = T_len - col0;
@@ -472,6 +475,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_ld32(s_addr + cbase, r);
                 tc_ld32(s_addr + cbase + 32, r + 32);
                 tc_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bar.s_free());  // the scores are in registers: the next S = Q K^T may overwrite the buffer
                 float mx0 = -INFINITY, mx1 = -INFINITY;
                 if (full_tile) {
 #pragma unroll
@@ -496,8 +501,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     corr = fast_exp2(m_used - m_new);  // 0 on the first tile (m_used = -inf)
                 }
                 const float m_ref = m_new == -INFINITY ? 0.f : m_new;
-                // probabilities, rounded to bf16, two per 32-bit column, written over the first half of the S
-                // buffer: the layout of an A operand in tensor memory.  S columns 64 h + c map to P column 32 h + c / 2.
+                // probabilities, rounded to bf16, two per 32-bit column: the layout of an A operand in tensor
+                // memory.  Score columns 64 h + c map to column 32 h + c / 2 of the tile's P buffer.
                 float ls0 = 0.f, ls1 = 0.f, ls2 = 0.f, ls3 = 0.f;
                 uint32_t packed[32];
                 if (full_tile) {
@@ -528,14 +533,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         packed[i >> 1] = *reinterpret_cast<uint32_t*>(&pk);
                     }
                 }
-                tc_st16(s_addr + half * 32, packed);
-                tc_st16(s_addr + half * 32 + 16, packed + 16);
+                // P buffer kt & 1 was last read by the P V of tile kt - 2
+                if (kt >= 2) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done(sb), ((kt >> 1) & 1) ^ 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
+                }
+                tc_st16(p_st, packed);
+                tc_st16(p_st + 16, packed + 16);
                 l_run = l_run * corr + ((ls0 + ls1) + (ls2 + ls3));
                 m_used = m_new;
                 // Rescaling touches the O accumulators, so the previous tile's P V must be complete first; a warp
                 // whose rows all keep their reference (the usual case after the first tiles) has nothing to wait
-                // for.  Skipping the wait cannot confuse the barrier's phase parity: S of this tile exists, so
-                // every P V up to tile kt - 2 has completed (the tensor core executes in issue order).
+                // for.  Skipping the wait cannot confuse the barrier's phase parity: the P V of tile kt - 3 (same
+                // barrier, previous phase) was awaited before P(kt - 1) was written.
                 if (j > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
                     ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done((kt - 1) & 1), ((kt - 1) >> 1) & 1, abort_flag));
                     if (!ok) break;
