@@ -1,17 +1,21 @@
 // Clustered causal prefill attention on the 5th-generation tensor cores (tcgen05 + TMEM + TMA).
 //
-// One CTA = (request, member group of <= 2 heads of one cluster, tile of 128 query rows).  The
+// A persistent kernel, one CTA per SM.  A unit of work = (request, member group of <= 2 heads of one
+// cluster, tile of 128 query rows); units are handed out by an atomic counter, heaviest first.  The
 // representative's Q tile and K tiles and the members' V tiles arrive by TMA (128-byte swizzle);
-// S = Q K^T and O_g += P V_g are tcgen05.mma instructions issued by one thread with fp32
-// accumulators in tensor memory (one S buffer of 128 columns, two P buffers of 64 columns, one O
-// accumulator of 128 columns per member: 512 columns).  Four warps own one query row per thread: they read S from tensor
-// memory, keep the running maximum and sum of the softmax (rescaling O only when the maximum grew
-// by more than 2^8, which leaves the result exact because p and l use the same reference), write
-// P as bf16 into shared memory in the operand layout, and at the end scale O by 1/l and store it.
+// S = Q K^T and O_g += P V_g are tcgen05.mma instructions with fp32 accumulators in tensor memory
+// (one S buffer of 128 columns, two P buffers of 64 columns, one O accumulator of 128 columns per
+// member: 512 columns).  The softmax threads read S from tensor memory, keep the running reference
+// and sum of the softmax (rescaling O only when the maximum grew by more than 2^8, which leaves the
+// result exact because p and l use the same reference) and write P as bf16 back into tensor memory,
+// from where it is the A operand of the P V product; the probabilities of a cluster are therefore
+// computed once and applied to every member's values (Fig. 3(b)).
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer (also owns the TMEM allocation),
-// warps 2..9 = softmax / correction / epilogue, two threads per query row (TMEM lane quadrant = warp
-// index mod 4; warps 2..5 take columns 0..63 of a tile, warps 6..9 columns 64..127).
+// Warp roles: warp 0 = work distribution and TMA producer; warp 1 = issuer of the S = Q K^T batches
+// (also owns the TMEM allocation); warps 2..9 = softmax / correction, two threads per query row
+// (TMEM lane quadrant = warp index mod 4; warps 2..5 take columns 0..63 of a tile, warps 6..9
+// columns 64..127); warps 10..13 = epilogue (O / l -> bf16 -> global) of the previous unit while
+// the next one computes; warp 14 = issuer of the P V batches.
 // Every mbarrier wait is bounded: on expiry the CTA records CHAI_ERR_TIMEOUT in the workspace
 // status word, skips the rest of its work, frees its tensor memory and returns.
 #include <cuda.h>
@@ -38,7 +42,8 @@ constexpr int TILE_BYTES = BN * HD * 2;        // 32 KB: one 128 x 128 bf16 tile
 constexpr int HALF_BYTES = TILE_BYTES / 2;     // 16 KB: one 128-row x 64-column swizzled box
 constexpr int SOFTMAX_WARPS = 8;    // two per TMEM lane quadrant: each thread owns half a row (64 columns)
 constexpr int EPILOGUE_WARPS = 4;   // one thread per query row: O / l -> bf16 -> global while the next item computes
-constexpr int THREADS = 64 + (SOFTMAX_WARPS + EPILOGUE_WARPS) * 32;
+constexpr int PV_WARP = 2 + SOFTMAX_WARPS + EPILOGUE_WARPS;  // the warp that issues the P V batches
+constexpr int THREADS = 96 + (SOFTMAX_WARPS + EPILOGUE_WARPS) * 32;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t S_COL0 = 0, P_COL0 = 128, O_COL0 = 256;  // S at 0..127, P buffers at 128 + 64 i, O_g at 256 + 128 g
 constexpr long long TIMEOUT_CYCLES = 2000000000ll;  // about a second
@@ -97,6 +102,33 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
+// The same for the MMA issuers, whose reaction time is on the critical path: a suspended try_wait takes
+// about 150 cycles to wake after the barrier completes, a polling test_wait sees it within one poll.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_polling(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_test_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_test_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > TIMEOUT_CYCLES) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
 // one 128-row x 128-column bf16 tile = box (64 columns, 128 rows, 2 column halves, 1 plane): lands as two
 // consecutive 16 KB blocks of 128-byte swizzled rows, which is the layout the MMA descriptors describe
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int row, int plane, uint32_t bar) {
@@ -104,6 +136,16 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(0), "r"(row), "r"(0), "r"(plane), "r"(bar)
         : "memory");
+}
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+    uint32_t is_leader;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(is_leader));
+    return is_leader != 0;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -167,6 +209,19 @@ __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+// 2^x on the FMA pipe, for the share of the exponentials that the special-function unit (16 results
+// per cycle and SM) has no time for.  x = n + f with n = round(x), |f| <= 1/2: 2^f by a cubic fitted
+// for relative error (1.2e-4, a twentieth of the bf16 rounding that follows), 2^n by adding n to the
+// exponent field.  Arguments below -125 give 2^-125 instead of 0, which no sum can see.
+__device__ __forceinline__ float poly_exp2(float x) {
+    x = fmaxf(x, -125.f);
+    const float t = x + 12582912.f;  // 1.5 * 2^23: the low mantissa bits of the sum hold round(x)
+    const float f = x - (t - 12582912.f);
+    float y = fmaf(f, 0.05459283f, 0.24221784f);
+    y = fmaf(y, f, 0.69336861f);
+    y = fmaf(y, f, 1.f);
+    return __int_as_float(__float_as_int(y) + (__float_as_int(t) << 23));
 }
 
 // Shared-memory matrix descriptor (tcgen05): 128-byte swizzle, descriptor version 1.
@@ -255,7 +310,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         mbar_init(bar.p_full(), SOFTMAX_WARPS * 32);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar.item_full(i), 1);
-            mbar_init(bar.item_empty(i), 1 + SOFTMAX_WARPS * 32);
+            mbar_init(bar.item_empty(i), 2 + SOFTMAX_WARPS * 32);
             mbar_init(bar.k_full(i), 1);
             mbar_init(bar.v_full(i), 1);
             mbar_init(bar.qk_done(i), 1);
@@ -352,73 +407,86 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 ++qi;
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc(true);
-            // Descriptors are built once; inside the loops only the 14-bit start-address field (low word)
-            // moves, by compile-time offsets, so issuing an MMA costs the thread an add and the instruction.
-            const uint64_t dq = make_desc(sbase + OFF_Q, 16, 1024);
-            const uint64_t dk = make_desc(sbase + OFF_K, 16, 1024);
-            const uint64_t dv = make_desc(sbase + OFF_V, HALF_BYTES, 1024);
-            const uint32_t hi_k = (uint32_t)(dq >> 32), hi_v = (uint32_t)(dv >> 32);
-            const uint32_t q_lo = (uint32_t)dq, k_lo = (uint32_t)dk, v_lo = (uint32_t)dv;
-            auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
-            bool ok = true;
-            int it = 0, qi = 0, kt = 0;  // items seen, items computed, key tiles whose S has been issued
-            while (ok) {
-                const int is = it & 1;
-                ok = mbar_wait(bar.item_full(is), (it >> 1) & 1, abort_flag);
-                if (!ok) break;
-                const int n_kv = items[is].n_kv, n_members = items[is].n_members;
-                mbar_arrive(bar.item_empty(is));  // the two fields are in registers
-                if (n_kv < 0) break;
-                if (n_kv == 0) {
-                    ++it;
-                    continue;
-                }
-                ok = mbar_wait(bar.q_full(), qi & 1, abort_flag);
-                // S(tile kt) = Q K^T into the S buffer, once the softmax warps hold the previous tile's scores in registers
-                auto issue_qk = [&](bool last) -> bool {
+    } else if (warp == 1 || warp == PV_WARP) {
+        // ---------------- MMA issuers ----------------
+        // Two warps issue the tensor-core work, one the S = Q K^T batches and one the O += P V batches, so
+        // that the barrier polling of either overlaps the other's instruction issue (issuing an MMA blocks
+        // the thread for about as long as the tensor pipe needs to run it).  Every ordering between the two
+        // streams goes through an mbarrier, and tcgen05.commit tracks the issuing thread's own MMAs, so the
+        // streams need no program order between them.  Each warp walks its loop as a whole, which keeps the
+        // control flow and the descriptor arithmetic warp-uniform; one elected lane issues.
+        constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc(true);
+        auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
+        auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_polling(b, parity, abort_flag)); };
+        const bool qk_role = warp == 1;
+        // Descriptors are built once; inside the loops only the 14-bit start-address field (low word)
+        // moves, by compile-time offsets, so issuing an MMA costs an add and the instruction.
+        const uint64_t dq = make_desc(sbase + OFF_Q, 16, 1024);
+        const uint64_t dk = make_desc(sbase + OFF_K, 16, 1024);
+        const uint64_t dv = make_desc(sbase + OFF_V, HALF_BYTES, 1024);
+        const uint32_t hi_k = (uint32_t)(dq >> 32), hi_v = (uint32_t)(dv >> 32);
+        const uint32_t q_lo = (uint32_t)dq, k_lo = (uint32_t)dk, v_lo = (uint32_t)dv;
+        bool ok = true;
+        int it = 0, qi = 0, kt = 0;  // items seen, items computed, key tiles issued so far
+        while (ok) {
+            const int is = it & 1;
+            ok = wait_all(bar.item_full(is), (it >> 1) & 1);
+            if (!ok) break;
+            const int n_kv = items[is].n_kv, n_members = items[is].n_members;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar.item_empty(is));  // the two fields are in registers
+            if (n_kv < 0) break;
+            if (n_kv == 0) {
+                ++it;
+                continue;
+            }
+            if (qk_role) {
+                ok = wait_all(bar.q_full(), qi & 1);
+                for (int j = 0; j < n_kv && ok; ++j, ++kt) {
+                    // S(tile kt) = Q K^T into the S buffer, once the softmax warps hold the previous tile's scores
                     const int ts = kt & 1;
-                    if (!mbar_wait(bar.k_full(ts), (kt >> 1) & 1, abort_flag)) return false;
-                    if (kt > 0 && !mbar_wait(bar.s_free(), (kt - 1) & 1, abort_flag)) return false;
+                    ok = wait_all(bar.k_full(ts), (kt >> 1) & 1) && (kt == 0 || wait_all(bar.s_free(), (kt - 1) & 1));
+                    if (!ok) break;
                     tc_fence_after();
                     const uint32_t d = tmem_base + S_COL0;
                     const uint32_t kb = k_lo + ts * (TILE_BYTES >> 4);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int s = 0; s < HD / 16; ++s) {
-                        const uint32_t off = ((s >> 2) * HALF_BYTES + (s & 3) * 32) >> 4;
-                        tc_mma(d, desc(hi_k, q_lo + off), desc(hi_k, kb + off), IDESC_QK, s > 0);
+                        for (int s = 0; s < HD / 16; ++s) {
+                            const uint32_t off = ((s >> 2) * HALF_BYTES + (s & 3) * 32) >> 4;
+                            tc_mma(d, desc(hi_k, q_lo + off), desc(hi_k, kb + off), IDESC_QK, s > 0);
+                        }
+                        tc_commit(bar.qk_done(ts));
+                        if (j + 1 == n_kv) tc_commit(bar.q_empty());  // Q may be overwritten by the next item's tile
                     }
-                    tc_commit(bar.qk_done(ts));
-                    if (last) tc_commit(bar.q_empty());  // Q may be overwritten by the next item's tile
-                    ++kt;
-                    return true;
-                };
-                if (ok) ok = issue_qk(n_kv == 1);
-                for (int j = 0; j < n_kv && ok; ++j) {
-                    if (j + 1 < n_kv) ok = issue_qk(j + 2 == n_kv);
-                    if (!ok) break;
-                    const int pt = kt - (j + 1 < n_kv ? 2 : 1), ts = pt & 1;  // global index of tile j
-                    ok = mbar_wait(bar.p_full(), pt & 1, abort_flag) && mbar_wait(bar.v_full(ts), (pt >> 1) & 1, abort_flag);
+                    __syncwarp();
+                }
+            } else {
+                for (int j = 0; j < n_kv && ok; ++j, ++kt) {
+                    const int ts = kt & 1;
+                    ok = wait_all(bar.p_full(), kt & 1) && wait_all(bar.v_full(ts), (kt >> 1) & 1);
                     // the previous item's output must have left tensor memory before its accumulators are reused
-                    if (ok && j == 0 && qi > 0) ok = mbar_wait(bar.o_free(), (qi - 1) & 1, abort_flag);
+                    if (ok && j == 0 && qi > 0) ok = wait_all(bar.o_free(), (qi - 1) & 1);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t p_addr = tmem_base + P_COL0 + ts * 64;  // P buffer of this tile
-                    for (int g = 0; g < n_members; ++g) {
-                        const uint32_t d = tmem_base + O_COL0 + g * HD;
-                        const uint32_t vb = v_lo + (ts * G + g) * (TILE_BYTES >> 4);
+                    if (elect_one()) {
 #pragma unroll
-                        for (int s = 0; s < BN / 16; ++s)  // 16 keys per step: 8 TMEM columns of P, 2048 bytes of V
-                            tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV, (j > 0 || s > 0) ? 1u : 0u);
+                        for (int g = 0; g < G; ++g) {
+                            if (g >= n_members) break;
+                            const uint32_t d = tmem_base + O_COL0 + g * HD;
+                            const uint32_t vb = v_lo + (ts * G + g) * (TILE_BYTES >> 4);
+#pragma unroll
+                            for (int s = 0; s < BN / 16; ++s)  // 16 keys per step: 8 TMEM columns of P, 2048 bytes of V
+                                tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV, (j > 0 || s > 0) ? 1u : 0u);
+                        }
+                        tc_commit(bar.pv_done(ts));
                     }
-                    tc_commit(bar.pv_done(ts));
+                    __syncwarp();
                 }
-                ++it;
-                ++qi;
             }
+            ++it;
+            ++qi;
         }
     } else if (warp < 2 + SOFTMAX_WARPS) {
         // ---------------- softmax / correction: two threads per query row ----------------
@@ -430,7 +498,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int row = quad * 32 + lane;        // row of the tile
         const int cbase = half * 64;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
-        float* xch = reinterpret_cast<float*>(smem + OFF_XCH);    // [half][row]
+        __nv_bfloat16* xch = reinterpret_cast<__nv_bfloat16*>(smem + OFF_XCH);  // [tile parity][half][row]
         float* lsum = reinterpret_cast<float*>(smem + OFF_LSUM);  // [half][row]
         auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quad) : "memory"); };
         bool ok = true;
@@ -489,11 +557,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     for (int i = 0; i < 64; ++i)
                         if (i < vis) mx0 = fmaxf(mx0, __uint_as_float(r[i]));
                 }
-                float mx = fmaxf(mx0, mx1);
-                xch[half * BM + row] = mx;
+                // The two threads of a row must agree on one reference.  Each rounds its half-row maximum up to
+                // bf16 and both take the larger of the two rounded values (a reference slightly above the true
+                // maximum is as good); the slots alternate with the tile's parity, so one meeting per tile is
+                // enough: a slot is rewritten two tiles later, after the meeting in between.
+                const __nv_bfloat16 mx_up = __float2bfloat16_ru(fmaxf(mx0, mx1));
+                __nv_bfloat16* xs = xch + (kt & 1) * 2 * BM;
+                xs[half * BM + row] = mx_up;
                 pair_sync();
-                mx = fmaxf(mx, xch[(half ^ 1) * BM + row]);
-                pair_sync();  // both values read before either slot is written again
+                const float mx = fmaxf(__bfloat162float(mx_up), __bfloat162float(xs[(half ^ 1) * BM + row]));
                 const float m_tile = mx * scale_log2;
                 float m_new = m_used, corr = 1.f;
                 if (m_tile > m_used + 8.f) {  // lazy rescale: only when the reference would be off by > 2^8
@@ -505,13 +577,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // memory.  Score columns 64 h + c map to column 32 h + c / 2 of the tile's P buffer.
                 float ls0 = 0.f, ls1 = 0.f, ls2 = 0.f, ls3 = 0.f;
                 uint32_t packed[32];
+                // P buffer kt & 1 was last read by the P V of tile kt - 2 (long complete as a rule)
+                if (kt >= 2) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done(sb), ((kt >> 1) & 1) ^ 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
+                }
                 if (full_tile) {
 #pragma unroll
                     for (int i = 0; i < 64; i += 4) {
+                        if (i == 32) tc_st16(p_st, packed);  // the first half goes out while the second is computed
                         const float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
                         const float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
                         const float p2 = fast_exp2(fmaf(__uint_as_float(r[i + 2]), scale_log2, -m_ref));
-                        const float p3 = fast_exp2(fmaf(__uint_as_float(r[i + 3]), scale_log2, -m_ref));
+                        const float p3 = poly_exp2(fmaf(__uint_as_float(r[i + 3]), scale_log2, -m_ref));
                         ls0 += p0;
                         ls1 += p1;
                         ls2 += p2;
@@ -523,6 +602,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 } else {
 #pragma unroll
                     for (int i = 0; i < 64; i += 2) {
+                        if (i == 32) tc_st16(p_st, packed);
                         float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
                         float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
                         if (i >= vis) p0 = 0.f;
@@ -533,13 +613,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         packed[i >> 1] = *reinterpret_cast<uint32_t*>(&pk);
                     }
                 }
-                // P buffer kt & 1 was last read by the P V of tile kt - 2
-                if (kt >= 2) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done(sb), ((kt >> 1) & 1) ^ 1, abort_flag));
-                    if (!ok) break;
-                    tc_fence_after();
-                }
-                tc_st16(p_st, packed);
                 tc_st16(p_st + 16, packed + 16);
                 l_run = l_run * corr + ((ls0 + ls1) + (ls2 + ls3));
                 m_used = m_new;
