@@ -53,7 +53,7 @@ constexpr int OFF_Q = 0;
 constexpr int OFF_K = OFF_Q + TILE_BYTES;
 constexpr int OFF_V = OFF_K + KST * TILE_BYTES;
 constexpr int OFF_BAR = OFF_V + VST * TILE_BYTES;
-constexpr int NUM_BARS = 19;
+constexpr int NUM_BARS = 36;
 constexpr int OFF_XCH = OFF_BAR + 8 * NUM_BARS + 16;               // after the barriers and the tmem slot / abort word
 constexpr int XCH_BYTES = 2 * BM * 4;                              // row maxima exchanged between the two halves
 constexpr int OFF_LSUM = OFF_XCH + XCH_BYTES;                      // row sums handed to the epilogue warps
@@ -170,6 +170,13 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// one full 32-byte sector per lane (rows are 256 bytes apart, so a 16-byte store would leave every
+// sector half written and double the number of write requests)
+__device__ __forceinline__ void st_global_32B(void* p, const uint32_t* w) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -197,6 +204,12 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+        : "memory");
+}
 __device__ __forceinline__ void tc_st16(uint32_t taddr, const uint32_t* r) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
@@ -210,18 +223,35 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// 2^x on the FMA pipe, for the share of the exponentials that the special-function unit (16 results
-// per cycle and SM) has no time for.  x = n + f with n = round(x), |f| <= 1/2: 2^f by a cubic fitted
-// for relative error (1.2e-4, a twentieth of the bf16 rounding that follows), 2^n by adding n to the
-// exponent field.  Arguments below -125 give 2^-125 instead of 0, which no sum can see.
-__device__ __forceinline__ float poly_exp2(float x) {
-    x = fmaxf(x, -125.f);
-    const float t = x + 12582912.f;  // 1.5 * 2^23: the low mantissa bits of the sum hold round(x)
-    const float f = x - (t - 12582912.f);
-    float y = fmaf(f, 0.05459283f, 0.24221784f);
-    y = fmaf(y, f, 0.69336861f);
-    y = fmaf(y, f, 1.f);
-    return __int_as_float(__float_as_int(y) + (__float_as_int(t) << 23));
+// Two fp32 operations per instruction (register pairs): the softmax warps are bound by instruction
+// issue, so the scale-and-shift of the scores and the row sums go through these.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
 }
 
 // Shared-memory matrix descriptor (tcgen05): 128-byte swizzle, descriptor version 1.
@@ -251,7 +281,7 @@ struct Bars {
     uint32_t base;
     __device__ __forceinline__ uint32_t q_full() const { return base; }
     __device__ __forceinline__ uint32_t q_empty() const { return base + 8; }
-    __device__ __forceinline__ uint32_t o_free() const { return base + 16; }
+    __device__ __forceinline__ uint32_t o_free(int g) const { return g == 0 ? base + 16 : base + 8 * 35; }  // per member
     __device__ __forceinline__ uint32_t p_full() const { return base + 24; }
     __device__ __forceinline__ uint32_t item_full(int i) const { return base + 8 * (4 + i); }
     __device__ __forceinline__ uint32_t item_empty(int i) const { return base + 8 * (6 + i); }
@@ -262,8 +292,14 @@ struct Bars {
     __device__ __forceinline__ uint32_t epi_full() const { return base + 8 * 16; }
     __device__ __forceinline__ uint32_t epi_empty() const { return base + 8 * 17; }
     __device__ __forceinline__ uint32_t s_free() const { return base + 8 * 18; }
+    // Softmax half `half` of TMEM lane quadrant `quad` has published its row maxima of a tile.  Tiles
+    // alternate between two barriers: the publisher may be a whole tile ahead of the reader (who looks at
+    // the end of its own tile), and one phase bit can tell apart only adjacent phases.
+    __device__ __forceinline__ uint32_t pair(int quad, int half, int tile) const {
+        return base + 8 * (19 + ((quad * 2 + half) * 2 + (tile & 1)));
+    }
 };
-static_assert(NUM_BARS == 19, "barrier count");
+static_assert(NUM_BARS == 36, "barrier count");
 
 // One unit of work, published by the producer to the other roles through shared memory.
 struct Item {
@@ -303,14 +339,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (tid == 0) {
         mbar_init(bar.q_full(), 1);
         mbar_init(bar.q_empty(), 1);
-        mbar_init(bar.o_free(), EPILOGUE_WARPS * 32);
-        mbar_init(bar.epi_full(), SOFTMAX_WARPS * 32);
-        mbar_init(bar.epi_empty(), EPILOGUE_WARPS * 32);
-        mbar_init(bar.s_free(), SOFTMAX_WARPS * 32);
-        mbar_init(bar.p_full(), SOFTMAX_WARPS * 32);
+        // Barriers that a whole role signals count warps, not threads: the lanes of a warp meet first and one
+        // lane arrives (hundreds of arrivals on one barrier word serialise and cost more than the work between them).
+        mbar_init(bar.o_free(0), EPILOGUE_WARPS);
+        mbar_init(bar.o_free(1), EPILOGUE_WARPS);
+        mbar_init(bar.epi_full(), SOFTMAX_WARPS);
+        mbar_init(bar.epi_empty(), EPILOGUE_WARPS);
+        mbar_init(bar.s_free(), SOFTMAX_WARPS);
+        mbar_init(bar.p_full(), SOFTMAX_WARPS);
+        for (int i = 0; i < 16; ++i) mbar_init(bar.pair(i >> 2, (i >> 1) & 1, i & 1), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar.item_full(i), 1);
-            mbar_init(bar.item_empty(i), 2 + SOFTMAX_WARPS * 32);
+            mbar_init(bar.item_empty(i), 2 + SOFTMAX_WARPS);
             mbar_init(bar.k_full(i), 1);
             mbar_init(bar.v_full(i), 1);
             mbar_init(bar.qk_done(i), 1);
@@ -339,25 +379,41 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const int n_items = n_pairs * n_qtiles;        // heaviest query tiles first
             bool ok = true;
             int it = 0, qi = 0, kt = 0;                    // items published, items with loads, key tiles issued
-            while (ok) {
-                const int id = atomicAdd(&hdr->pad[counter_slot], 1);  // next unit of work (the header was cleared by the host)
-                const int is = it & 1;
-                ok = mbar_wait(bar.item_empty(is), ((it >> 1) & 1) ^ 1, abort_flag);
-                if (!ok) break;
-                Item& item = items[is];
-                if (id >= n_items) {
-                    item.n_kv = -1;
-                    mbar_arrive(bar.item_full(is));
-                    break;
-                }
-                const int qt = n_qtiles - 1 - id / n_pairs, pair = id % n_pairs;
+            // Work items are fetched one ahead: the atomic that claims the next item is issued before the
+            // current item's tiles are streamed and its group entry is read while they stream, so the two
+            // dependent round trips to global memory never stall the pipeline between items.
+            struct Claim {
+                int id, qt, b;
+                GroupEntry e;
+            };
+            auto resolve = [&](Claim& c) {                 // c.id -> query tile, request, group entry
+                if (c.id >= n_items) return;
+                const int pair = c.id % n_pairs;
+                c.qt = n_qtiles - 1 - c.id / n_pairs;
                 int lo = 0, hi = B;                        // largest b with prefix[b] <= pair
                 while (hi - lo > 1) {
                     const int mid = (lo + hi) >> 1;
                     if (prefix[mid] <= pair) lo = mid; else hi = mid;
                 }
-                const int b = b_begin + lo, slot = pair - prefix[lo];
-                const GroupEntry e = groups[(size_t)b * H + slot];
+                c.b = b_begin + lo;
+                c.e = groups[(size_t)c.b * H + (pair - prefix[lo])];
+            };
+            Claim cur, nxt;
+            cur.id = atomicAdd(&hdr->pad[counter_slot], 1);  // (the counter was cleared by the planning kernel)
+            resolve(cur);
+            while (ok) {
+                nxt.id = atomicAdd(&hdr->pad[counter_slot], 1);
+                const int is = it & 1;
+                ok = mbar_wait(bar.item_empty(is), ((it >> 1) & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                Item& item = items[is];
+                if (cur.id >= n_items) {
+                    item.n_kv = -1;
+                    mbar_arrive(bar.item_full(is));
+                    break;
+                }
+                const int qt = cur.qt, b = cur.b;
+                const GroupEntry e = cur.e;
                 const int n_members = min(e.n, G);
                 item.q0 = qt * BM;
                 item.n_members = n_members;
@@ -367,6 +423,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     item.q_plane = item.k_plane = 0;
                     mbar_arrive(bar.item_full(is));
                     ++it;
+                    resolve(nxt);
+                    cur = nxt;
                     continue;
                 }
                 const int n_kv = causal ? min(qt + 1, (T_len + BN - 1) / BN) : (T_len + BN - 1) / BN;
@@ -401,10 +459,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     mbar_expect_tx(bar.v_full(ts), n_members * TILE_BYTES);
                     for (int g = 0; g < n_members; ++g)
                         tma_load_4d(sbase + OFF_V + (ts * G + g) * TILE_BYTES, &map_v, j * BN, v_plane[g], bar.v_full(ts));
+                    if (j == 0) resolve(nxt);  // two tiles are on their way: time to look at the claim's answer
                 }
                 kt += n_kv;
                 ++it;
                 ++qi;
+                cur = nxt;
             }
         }
     } else if (warp == 1 || warp == PV_WARP) {
@@ -465,24 +525,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 for (int j = 0; j < n_kv && ok; ++j, ++kt) {
                     const int ts = kt & 1;
                     ok = wait_all(bar.p_full(), kt & 1) && wait_all(bar.v_full(ts), (kt >> 1) & 1);
-                    // the previous item's output must have left tensor memory before its accumulators are reused
-                    if (ok && j == 0 && qi > 0) ok = wait_all(bar.o_free(), (qi - 1) & 1);
                     if (!ok) break;
-                    tc_fence_after();
                     const uint32_t p_addr = tmem_base + P_COL0 + ts * 64;  // P buffer of this tile
-                    if (elect_one()) {
+                    const bool reuse = j == 0 && qi > 0;  // the accumulators still hold the previous item's output
 #pragma unroll
-                        for (int g = 0; g < G; ++g) {
-                            if (g >= n_members) break;
+                    for (int g = 0; g < G; ++g) {
+                        if (g >= n_members) break;
+                        // each member's accumulator is released by the epilogue warps on its own
+                        if (reuse && !wait_all(bar.o_free(g), (qi - 1) & 1)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
+                        if (elect_one()) {
                             const uint32_t d = tmem_base + O_COL0 + g * HD;
                             const uint32_t vb = v_lo + (ts * G + g) * (TILE_BYTES >> 4);
 #pragma unroll
                             for (int s = 0; s < BN / 16; ++s)  // 16 keys per step: 8 TMEM columns of P, 2048 bytes of V
                                 tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV, (j > 0 || s > 0) ? 1u : 0u);
+                            if (g + 1 == n_members) tc_commit(bar.pv_done(ts));
                         }
-                        tc_commit(bar.pv_done(ts));
+                        __syncwarp();
                     }
-                    __syncwarp();
                 }
             }
             ++it;
@@ -500,7 +564,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
         __nv_bfloat16* xch = reinterpret_cast<__nv_bfloat16*>(smem + OFF_XCH);  // [tile parity][half][row]
         float* lsum = reinterpret_cast<float*>(smem + OFF_LSUM);  // [half][row]
-        auto pair_sync = [&]() { asm volatile("bar.sync %0, 64;" ::"r"(1 + quad) : "memory"); };
         bool ok = true;
         int it = 0, ei = 0, kt = 0;  // items seen, items handed to the epilogue, key tiles processed so far
         uint32_t r[64];
@@ -511,7 +574,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (!ok) break;
             const Item item = items[is];
             __syncwarp();
-            mbar_arrive(bar.item_empty(is));  // the item is in registers
+            if (lane == 0) mbar_arrive(bar.item_empty(is));  // the item is in registers (all lanes: __syncwarp above)
             if (item.n_kv < 0) break;
             const int n_kv = item.n_kv, n_members = item.n_members, q0 = item.q0;
             const int row_abs = q0 + row;
@@ -544,76 +607,105 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_ld32(s_addr + cbase + 32, r + 32);
                 tc_wait_ld();
                 tc_fence_before();
-                mbar_arrive(bar.s_free());  // the scores are in registers: the next S = Q K^T may overwrite the buffer
-                float mx0 = -INFINITY, mx1 = -INFINITY;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar.s_free());  // the scores are in registers: the next S = Q K^T may overwrite the buffer
+                // own half-row maximum (eight independent chains)
+                float mxa[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) mxa[c] = -INFINITY;
                 if (full_tile) {
 #pragma unroll
-                    for (int i = 0; i < 64; i += 2) {
-                        mx0 = fmaxf(mx0, __uint_as_float(r[i]));
-                        mx1 = fmaxf(mx1, __uint_as_float(r[i + 1]));
-                    }
+                    for (int i = 0; i < 64; i += 2) mxa[(i >> 1) & 7] = max3(mxa[(i >> 1) & 7], __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
                 } else {
 #pragma unroll
                     for (int i = 0; i < 64; ++i)
-                        if (i < vis) mx0 = fmaxf(mx0, __uint_as_float(r[i]));
+                        if (i < vis) mxa[i & 7] = fmaxf(mxa[i & 7], __uint_as_float(r[i]));
                 }
                 // The two threads of a row must agree on one reference.  Each rounds its half-row maximum up to
-                // bf16 and both take the larger of the two rounded values (a reference slightly above the true
-                // maximum is as good); the slots alternate with the tile's parity, so one meeting per tile is
-                // enough: a slot is rewritten two tiles later, after the meeting in between.
-                const __nv_bfloat16 mx_up = __float2bfloat16_ru(fmaxf(mx0, mx1));
+                // bf16 and publishes it (slots alternate with the tile's parity); both take the larger of the two
+                // rounded values, a reference slightly above the true maximum being as good.
+                const __nv_bfloat16 mx_up =
+                    __float2bfloat16_ru(max3(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
                 __nv_bfloat16* xs = xch + (kt & 1) * 2 * BM;
                 xs[half * BM + row] = mx_up;
-                pair_sync();
-                const float mx = fmaxf(__bfloat162float(mx_up), __bfloat162float(xs[(half ^ 1) * BM + row]));
-                const float m_tile = mx * scale_log2;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar.pair(quad, half, kt));
                 float m_new = m_used, corr = 1.f;
-                if (m_tile > m_used + 8.f) {  // lazy rescale: only when the reference would be off by > 2^8
-                    m_new = m_tile;
-                    corr = fast_exp2(m_used - m_new);  // 0 on the first tile (m_used = -inf)
-                }
-                const float m_ref = m_new == -INFINITY ? 0.f : m_new;
+                // Meet the partner: reference of this tile, by the lazy-rescale rule (it moves only when the
+                // maximum outgrew it by more than 2^8).
+                auto meet = [&]() -> bool {
+                    if (!__all_sync(0xffffffffu, mbar_wait(bar.pair(quad, half ^ 1, kt), (kt >> 1) & 1, abort_flag))) return false;
+                    const float mx = fmaxf(__bfloat162float(mx_up), __bfloat162float(xs[(half ^ 1) * BM + row]));
+                    const float m_tile = mx * scale_log2;
+                    if (m_tile > m_used + 8.f) {
+                        m_new = m_tile;
+                        corr = fast_exp2(m_used - m_new);  // 0 on the first tile (m_used = -inf)
+                    }
+                    return true;
+                };
                 // probabilities, rounded to bf16, two per 32-bit column: the layout of an A operand in tensor
                 // memory.  Score columns 64 h + c map to column 32 h + c / 2 of the tile's P buffer.
                 float ls0 = 0.f, ls1 = 0.f, ls2 = 0.f, ls3 = 0.f;
-                uint32_t packed[32];
                 // P buffer kt & 1 was last read by the P V of tile kt - 2 (long complete as a rule)
                 if (kt >= 2) {
                     ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done(sb), ((kt >> 1) & 1) ^ 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
                 }
-                if (full_tile) {
+                // After an item's first tile the reference hardly ever moves, so a full tile is computed
+                // against the current reference at once, without waiting for the partner's maximum, and goes
+                // to tensor memory in chunks of 16 probabilities as they are ready; the meeting follows the
+                // arithmetic, and only if some row's reference did move is the tile computed and stored again.
+                const bool speculate = j > 0 && full_tile;
+                bool redo = !speculate;
+                if (speculate) {
+                    const float m_ref = m_used == -INFINITY ? 0.f : m_used;
+                    const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m_ref, -m_ref);
+                    uint64_t acc01 = 0ull, acc23 = 0ull;  // two packed pairs of partial row sums
 #pragma unroll
-                    for (int i = 0; i < 64; i += 4) {
-                        if (i == 32) tc_st16(p_st, packed);  // the first half goes out while the second is computed
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
-                        const float p2 = fast_exp2(fmaf(__uint_as_float(r[i + 2]), scale_log2, -m_ref));
-                        const float p3 = poly_exp2(fmaf(__uint_as_float(r[i + 3]), scale_log2, -m_ref));
-                        ls0 += p0;
-                        ls1 += p1;
-                        ls2 += p2;
-                        ls3 += p3;
-                        __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
-                        packed[i >> 1] = *reinterpret_cast<uint32_t*>(&pa);
-                        packed[(i >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t packed[8];
+#pragma unroll
+                        for (int u = 0; u < 16; u += 4) {
+                            const int i = c * 16 + u;
+                            float x0, x1, x2, x3;
+                            unpack2(fma2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2), x0, x1);
+                            unpack2(fma2(pack2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), sc2, nm2), x2, x3);
+                            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+                            acc01 = add2(acc01, pack2(p0, p1));
+                            acc23 = add2(acc23, pack2(p2, p3));
+                            __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
+                            packed[u >> 1] = *reinterpret_cast<uint32_t*>(&pa);
+                            packed[(u >> 1) + 1] = *reinterpret_cast<uint32_t*>(&pb);
+                        }
+                        tc_st8(p_st + c * 8, packed);
                     }
-                } else {
+                    unpack2(add2(acc01, acc23), ls0, ls1);
+                }
+                ok = meet();
+                if (!ok) break;
+                if (speculate) redo = __any_sync(0xffffffffu, m_new != m_used);
+                if (redo) {
+                    const float m_ref = m_new == -INFINITY ? 0.f : m_new;
+                    ls0 = ls1 = ls2 = ls3 = 0.f;
 #pragma unroll
-                    for (int i = 0; i < 64; i += 2) {
-                        if (i == 32) tc_st16(p_st, packed);
-                        float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
-                        if (i >= vis) p0 = 0.f;
-                        if (i + 1 >= vis) p1 = 0.f;
-                        ls0 += p0;
-                        ls1 += p1;
-                        __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                        packed[i >> 1] = *reinterpret_cast<uint32_t*>(&pk);
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t packed[8];
+#pragma unroll
+                        for (int u = 0; u < 16; u += 2) {
+                            const int i = c * 16 + u;
+                            float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
+                            float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
+                            if (i >= vis) p0 = 0.f;
+                            if (i + 1 >= vis) p1 = 0.f;
+                            ls0 += p0;
+                            ls1 += p1;
+                            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+                            packed[u >> 1] = *reinterpret_cast<uint32_t*>(&pk);
+                        }
+                        tc_st8(p_st + c * 8, packed);
                     }
                 }
-                tc_st16(p_st + 16, packed + 16);
                 l_run = l_run * corr + ((ls0 + ls1) + (ls2 + ls3));
                 m_used = m_new;
                 // Rescaling touches the O accumulators, so the previous tile's P V must be complete first; a warp
@@ -637,7 +729,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 }
                 tc_wait_st();          // P (and any rescaled O) is in tensor memory
                 tc_fence_before();
-                mbar_arrive(bar.p_full());
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar.p_full());
             }
             // hand the item to the epilogue warps: row sums of both halves and where the output goes
             ok = __all_sync(0xffffffffu, ok && mbar_wait(bar.epi_empty(), (ei & 1) ^ 1, abort_flag));
@@ -648,14 +741,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 ep = item;
                 ep.n_kv = kt - 1;  // global index of the item's last key tile (its P V completion is awaited)
             }
-            mbar_arrive(bar.epi_full());
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar.epi_full());
             ++ei;
             ++it;
         }
         // tell the epilogue warps that nothing more will come
         if (__all_sync(0xffffffffu, mbar_wait(bar.epi_empty(), (ei & 1) ^ 1, abort_flag))) {
             if (tid == 64) items[2].n_members = -1;
-            mbar_arrive(bar.epi_full());
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar.epi_full());
         }
     } else {
         // ---------------- epilogue: O_g / l -> bf16 -> global, one thread per query row ----------------
@@ -663,7 +758,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int row = quad * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
         const float* lsum = reinterpret_cast<const float*>(smem + OFF_LSUM);
-        uint32_t r[32];
+        uint32_t r[64];
         for (int ei = 0;; ++ei) {
             bool ok = __all_sync(0xffffffffu, mbar_wait(bar.epi_full(), ei & 1, abort_flag));
             if (!ok) break;
@@ -675,30 +770,37 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (!ok) break;
             tc_fence_after();
             __syncwarp();
-            mbar_arrive(bar.epi_empty());  // the hand-over area is in registers
+            if (lane == 0) mbar_arrive(bar.epi_empty());  // the hand-over area is in registers (all lanes: __syncwarp above)
             const int row_abs = ep.q0 + row;
             const float inv = l > 0.f ? 1.f / l : 0.f;
+            const uint64_t inv2 = pack2(inv, inv);
             for (int g = 0; g < ep.n_members; ++g) {
                 __nv_bfloat16* orow = out + ((size_t)ep.o_plane[g] * T_len + row_abs) * HD;
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    tc_ld32(lane_addr + O_COL0 + g * HD + ch * 32, r);
+                for (int ch = 0; ch < 2; ++ch) {  // 64 columns per round: two loads in flight
+                    tc_ld32(lane_addr + O_COL0 + g * HD + ch * 64, r);
+                    tc_ld32(lane_addr + O_COL0 + g * HD + ch * 64 + 32, r + 32);
                     tc_wait_ld();
-                    if (g == ep.n_members - 1 && ch == 3) {  // this row's accumulators are in registers
+                    if (ch == 1) {  // this row of the member's accumulator is in registers
                         tc_fence_before();
-                        mbar_arrive(bar.o_free());
+                        __syncwarp();
+                        if (lane == 0) {
+                            mbar_arrive(bar.o_free(g));
+                            if (ep.n_members == 1) mbar_arrive(bar.o_free(1));  // keep the unused barrier's phase in step
+                        }
                     }
                     if (row_abs < T_len) {
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            uint32_t w[4];
+                            uint32_t w[8];
 #pragma unroll
-                            for (int x = 0; x < 4; ++x) {
-                                __nv_bfloat162 pk = __floats2bfloat162_rn(__uint_as_float(r[8 * u + 2 * x]) * inv,
-                                                                          __uint_as_float(r[8 * u + 2 * x + 1]) * inv);
+                            for (int x = 0; x < 8; ++x) {
+                                float y0, y1;
+                                unpack2(mul2(pack2(__uint_as_float(r[16 * u + 2 * x]), __uint_as_float(r[16 * u + 2 * x + 1])), inv2), y0, y1);
+                                __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
                                 w[x] = *reinterpret_cast<uint32_t*>(&pk);
                             }
-                            *reinterpret_cast<uint4*>(orow + ch * 32 + u * 8) = make_uint4(w[0], w[1], w[2], w[3]);
+                            st_global_32B(orow + ch * 64 + u * 16, w);
                         }
                     }
                 }

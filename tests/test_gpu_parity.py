@@ -278,6 +278,38 @@ def test_prefill_cluster_shapes(H, k, kind):
     assert_parity(got, ref, "bf16", f"H {H} k {k}")
 
 
+@pytest.mark.parametrize("direction", ["growing", "shrinking", "late_spike"])
+@pytest.mark.parametrize("causal", [True, False])
+def test_prefill_reference_moves(direction, causal):
+    """Scores that drift by more than 2^8 from one key tile to the next: the running softmax reference has
+    to move (and the accumulated output has to be rescaled) in every tile, or never after the first, or
+    once near the end: the paths of the online softmax that ordinary random inputs rarely reach."""
+    B, H, T, k, D = 1, 6, 640, 2, 128
+    r = synth.batch_partitions(B, H, k, "uneven", 11, 78, T)
+    g = torch.Generator().manual_seed(5)
+    u = torch.randn(D, generator=g)
+    u = u / u.norm()
+    t = torch.arange(T, dtype=torch.float32)
+    if direction == "growing":
+        ramp = 0.1 * t                      # log2-domain score grows by ~18 per tile of 128 keys
+    elif direction == "shrinking":
+        ramp = 0.1 * (T - 1 - t)
+    else:
+        ramp = torch.where(t >= 600, torch.full_like(t, 40.0), torch.zeros_like(t))
+    scale = 1.0 / np.sqrt(D)
+    # q . k_t * scale * log2(e) = ramp_t  (up to bf16 rounding), plus a little noise in other directions
+    q = (u * 4.0).expand(B, H, T, D) + 0.05 * torch.randn(B, H, T, D, generator=g)
+    kr = (ramp[:, None] * u[None, :] / (4.0 * scale * 1.4426950408889634)).expand(B, k, T, D) \
+        + 0.05 * torch.randn(B, k, T, D, generator=g)
+    v = 0.5 * torch.randn(B, H, T, D, generator=g)
+    case = dict(q=q.to(torch.bfloat16), k_rep=kr.to(torch.bfloat16), v=v.to(torch.bfloat16),
+                membership=torch.as_tensor(r[0]), reps=torch.as_tensor(r[1]), scale=scale, dtype="bf16")
+    got = run_prefill(case, causal)
+    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], scale, causal)
+    assert np.isfinite(got).all()
+    assert_parity(got, ref, "bf16", f"reference moves: {direction} causal {causal}")
+
+
 def test_prefill_head_dim_64():
     case = prefill_inputs(9, 2, 6, 150, 2, "bf16", D=64, peaked=4.0)
     got = run_prefill(case)
