@@ -56,6 +56,9 @@ prefill_plan_kernel(const int32_t* __restrict__ membership, const int32_t* __res
     GroupEntry* ent = reinterpret_cast<GroupEntry*>(s_plan + ((2 * k + 2 * H + 3) & ~3));  // [H], 16-byte aligned
     __shared__ int s_next, s_nbad;
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+    // a kernel launched as a programmatic dependent may start its own set-up now; it still waits for this
+    // grid to finish (griddepcontrol.wait) before it reads anything written here
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (b == 0)
         for (int i = tid; i < 60; i += nt) hdr->pad[i] = 0;
     for (int h = tid; h < H; h += nt) mem[h] = membership[(size_t)b * H + h];

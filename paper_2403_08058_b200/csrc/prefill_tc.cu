@@ -327,6 +327,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     uint8_t* smem = smem_raw;
     const uint32_t sbase = smem_u32(smem);
     if ((sbase & 1023u) != 0) {  // swizzled tiles need 1024-byte alignment; never observed, but refuse rather than corrupt
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // the planner resets the header
         if (tid == 0) atomicExch(&hdr->status, CHAI_ERR_TIMEOUT);
         return;
     }
@@ -357,15 +358,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             mbar_init(bar.pv_done(i), 1);
         }
         *abort_flag = 0;
-        if (blockIdx.x == 0 && counter_slot == 0) publish_plan_status(hdr, bad, B_total);
-        prefix[0] = 0;
-        for (int bb = 0; bb < B; ++bb) prefix[bb + 1] = prefix[bb] + n_groups[b_begin + bb];
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_proxy();
     }
     if (warp == 1) {  // whole warp: allocate all 512 TMEM columns (one CTA per SM by shared-memory size)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // Everything above is independent of the planning kernel, which may still be running (the launch is
+    // programmatically dependent); its results are read only after this point.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (tid == 0) {
+        if (blockIdx.x == 0 && counter_slot == 0) publish_plan_status(hdr, bad, B_total);
+        prefix[0] = 0;
+        for (int bb = 0; bb < B; ++bb) prefix[bb + 1] = prefix[bb] + n_groups[b_begin + bb];
     }
     tc_fence_before();
     __syncthreads();
@@ -885,11 +891,24 @@ extern "C" int chai_prefill_attention(const void* q, const void* k_rep, const vo
     // a chunk are kept in shared memory), each chunk with its own work counter in the workspace header
     for (int b0 = 0, chunk = 0; b0 < B; b0 += tc::MAX_B, ++chunk) {
         const int nb = B - b0 < tc::MAX_B ? B - b0 : tc::MAX_B;
-        tc::prefill_tc_kernel<<<n_sms, tc::THREADS, tc::SMEM_BYTES, s>>>(
-            mq, mk, mv, reinterpret_cast<const int*>(ws + L.off_ngroups),
+        // launched as a programmatic dependent of the planning kernel: the set-up of this kernel's CTAs
+        // overlaps the planner's run, and the kernel itself waits for the planner before it reads the plan
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(n_sms);
+        cfg.blockDim = dim3(tc::THREADS);
+        cfg.dynamicSmemBytes = tc::SMEM_BYTES;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t le = cudaLaunchKernelEx(
+            &cfg, tc::prefill_tc_kernel, mq, mk, mv, reinterpret_cast<const int*>(ws + L.off_ngroups),
             reinterpret_cast<const GroupEntry*>(ws + L.off_groups), static_cast<__nv_bfloat16*>(out),
             reinterpret_cast<WsHeader*>(ws), reinterpret_cast<const int*>(ws + L.off_bad), B, b0, nb, H, k, T,
             scale * 1.4426950408889634f, causal, n_qtiles, chunk);
+        if (le != cudaSuccess) return cuda_fail(le, "prefill_tc_kernel launch");
         CHAI_LAUNCH_CHECK("prefill_tc_kernel launch");
     }
     return CHAI_OK;
