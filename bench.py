@@ -301,6 +301,70 @@ def bench_compaction(device, peaks, iters=20, warmup=3):
                          "peak_source": peaks["source"], "traffic": None}, "l2": "flushed by a 256 MB write"}
 
 
+def bench_serving(device, peaks, iters=20, warmup=3):
+    """The serving-shaped steps at workload 2's layer shape (k = 8): a ragged batch whose lengths are spread
+    over 1/4..1 of the capacity, read from a cache that was compacted in place; the per-token append; the
+    in-place compaction itself."""
+    w = synth.WORKLOADS[2]
+    k, B, H, T_cap, D, es = 8, w.B, w.H, w.T, w.D, 2
+    c = synth.decode_layer(2, 0, 1, device=device, B=B, H=H, T=T_cap, k=k, with_k_full=True)
+    rng = np.random.default_rng(7)
+    lens = rng.integers(T_cap // 4, T_cap, size=B).astype(np.int32)
+    lens[0] = T_cap - 1
+    seq = torch.as_tensor(lens, device=device)
+    reps_host = c["reps"].cpu().numpy()
+    cache = c["k_full"].clone()
+    ws = chai.new_workspace(chai.chai_decode_workspace_bytes(B, H, k, T_cap, D, chai.CHAI_BF16), device)
+    flush = torch.empty(256 << 20, device=device, dtype=torch.uint8)
+
+    def timed(fn, before=None):
+        ts = []
+        for i in range(warmup + iters):
+            if before is not None:
+                before()
+            flush.fill_(i & 1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= warmup:
+                ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    # in-place compaction (restore the full cache before every run)
+    ms_c = timed(lambda: chai.chai_compact_k_cache_inplace(cache, c["reps"], T=T_cap), before=lambda: cache.copy_(c["k_full"]))
+    moved = int(sum(1 for b in range(B) for cc in range(k) if reps_host[b, cc] >= 0 and reps_host[b, cc] != cc))
+    bytes_c = 2 * moved * T_cap * D * es
+    # ragged decode from the strided cache
+    out = torch.empty_like(c["q"])
+    ms_d = timed(lambda: chai.chai_decode_attention_ragged(c["q"], cache, c["v"], c["membership"], c["reps"], seq, c["scale"],
+                                                           T_max=T_cap, out=out, workspace=ws))
+    bytes_d = int(sum((k + H) * int(n) * D * es for n in lens)) + (k + H) * B * D * es
+    # the same call with every request at full length, timed the same way (single call after an L2 flush,
+    # launch latency included), as the yardstick for the ragged number
+    full = torch.full((B,), T_cap, dtype=torch.int32, device=device)
+    ms_f = timed(lambda: chai.chai_decode_attention_ragged(c["q"], cache, c["v"], c["membership"], c["reps"], full, c["scale"],
+                                                           T_max=T_cap, out=out, workspace=ws))
+    bytes_f = (k + H) * B * T_cap * D * es + (k + H) * B * D * es
+    # append (no advance, so every run writes the same rows)
+    k_new = torch.randn((B, H, D), device=device).to(torch.bfloat16)
+    v_new = torch.randn((B, H, D), device=device).to(torch.bfloat16)
+    ms_a = timed(lambda: chai.chai_append_kv(k_new, v_new, cache, c["v"], c["reps"], seq, advance=False))
+    gbs_d, gbs_c = bytes_d / (ms_d * 1e-3) / 1e9, bytes_c / (ms_c * 1e-3) / 1e9
+    return {"workload": "config2 layer shape, k=8, lengths uniform in [T/4, T), K cache compacted in place",
+            "seq_lens": [int(x) for x in lens],
+            "full_length_same_timing": {"us": ms_f * 1e3, "algorithmic_mb": bytes_f / 1e6, "gbs": bytes_f / (ms_f * 1e-3) / 1e9},
+            "ragged_decode": {"us": ms_d * 1e3, "algorithmic_mb": bytes_d / 1e6, "gbs": gbs_d,
+                              "roofline": {"bound": "hbm", "achieved": gbs_d, "peak": peaks["hbm"], "unit": "GB/s",
+                                           "frac": gbs_d / peaks["hbm"], "peak_source": peaks["source"], "traffic": None}},
+            "compact_inplace": {"us": ms_c * 1e3, "planes_moved": moved, "algorithmic_mb": bytes_c / 1e6, "gbs": gbs_c,
+                                "roofline": {"bound": "hbm", "achieved": gbs_c, "peak": peaks["hbm"], "unit": "GB/s",
+                                             "frac": gbs_c / peaks["hbm"], "peak_source": peaks["source"], "traffic": None}},
+            "append_kv": {"us": ms_a * 1e3, "bytes": 2 * (H + k) * B * D * es, "bound": "latency (one CTA per request)"},
+            "l2": "flushed by a 256 MB write before every timed call"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -394,6 +458,7 @@ def main():
             torch.cuda.empty_cache()
             line["prefill"] = bench_prefill(device, peaks)
             line["compaction"] = bench_compaction(device, peaks)
+            line["serving"] = bench_serving(device, peaks)
             line["cpu_baseline"] = cpu_baseline_decode(args.workload, 0)
         print(json.dumps(line))
     ranks.close()

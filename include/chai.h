@@ -50,7 +50,8 @@ typedef enum {
     CHAI_ERR_WORKSPACE = 3,      /* workspace_bytes smaller than the matching *_workspace_bytes() */
     CHAI_ERR_BAD_MEMBERSHIP = 4, /* device status word only: inconsistent membership / reps */
     CHAI_ERR_TIMEOUT = 5,        /* device status word only: a bounded device-side wait expired */
-    CHAI_ERR_CUDA = 6            /* a CUDA call failed; text in chai_last_error() */
+    CHAI_ERR_CUDA = 6,           /* a CUDA call failed; text in chai_last_error() */
+    CHAI_ERR_CACHE_FULL = 7      /* device status word only: chai_append_kv found seq_lens[b] outside [0, T_cap) */
 } chai_status_t;
 
 typedef enum { CHAI_F32 = 0, CHAI_BF16 = 1 } chai_dtype_t;
@@ -115,6 +116,51 @@ int chai_decode_attention(const void* q, const void* k_rep, const void* v, const
 size_t chai_decode_workspace_bytes(int B, int H, int k, int T, int D, int dtype);
 
 /*
+ * The same decode step for a ragged batch, as a serving loop holds it (Section 3.5: membership, hence the
+ * caches, are per request; requests of a batch are at different positions).
+ *   seq_lens [B] int32, device   cached positions of each request, INCLUDING the current token; values are
+ *                                clamped to [0, T_max]; a request with length 0 gets an all-zero output
+ *   T_max                        upper bound of seq_lens known to the host: sizes the workspace
+ *                                (chai_decode_workspace_bytes(B, H, k, T_max, D, dtype)) and the launch
+ *   k_batch_stride               elements between the first representative planes of two consecutive requests
+ *                                in k_rep: 0 or k*T_cap*D for a dense [B,k,T_cap,D] cache, H*T_cap*D for a
+ *                                full cache compacted in place by chai_compact_k_cache_inplace
+ * Everything else as chai_decode_attention.  Cache rows at or beyond a request's length are never read.
+ */
+int chai_decode_attention_ragged(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                 const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k,
+                                 int T_max, int T_cap, int D, size_t k_batch_stride, float scale, int dtype,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Cache append for one new token per request (Section 3.5 / 4.3: after clustering only the representative
+ * heads' keys are cached, every head's values are).
+ *   k_new, v_new [B,H,D]   the token's keys / values of all heads (the layer's projection output)
+ *   k_rep                  representative key cache, request stride k_batch_stride (see above), plane stride T_cap*D
+ *   v     [B,H,T_cap,D]    value cache
+ *   seq_lens [B] int32     device; the row written is pos = seq_lens[b] (the number of positions cached so far):
+ *                          k_rep[b][c][pos] = k_new[b][reps[b][c]],  v[b][h][pos] = v_new[b][h]
+ *   advance                non-zero: seq_lens[b] becomes pos + 1 afterwards, so that the following decode call
+ *                          sees the new token
+ *   workspace              NULL, or >= 256 bytes: its status word is set to CHAI_OK, or to CHAI_ERR_CACHE_FULL
+ *                          if some seq_lens[b] was outside [0, T_cap) (that request is skipped, nothing faults)
+ */
+int chai_append_kv(const void* k_new, const void* v_new, void* k_rep, void* v, const int32_t* reps, int32_t* seq_lens,
+                   int B, int H, int k, int T_cap, int D, size_t k_batch_stride, int dtype, int advance,
+                   void* workspace, void* stream);
+
+/*
+ * K-cache compaction in place (Section 3.5: "remove" the keys of the non-representative heads): afterwards
+ * planes 0..k-1 of every request of k_cache [B,H,T_cap,D] hold the representatives' keys, rows [0,T); the
+ * other planes are dead and may be reused by the caller; decode / append then address the buffer with
+ * k_batch_stride = H*T_cap*D.  Requires what chai_cluster_heads guarantees: reps strictly ascending with
+ * reps[b][c] >= c and unused slots (-1) only at the end.  A request whose reps break that rule is left
+ * untouched and CHAI_ERR_BAD_MEMBERSHIP is recorded in the status word of `workspace` (NULL or >= 256 bytes).
+ */
+int chai_compact_k_cache_inplace(void* k_cache, const int32_t* reps, int B, int H, int k, int T, int T_cap, int D,
+                                 int dtype, void* workspace, void* stream);
+
+/*
  * The same decode step with the per-step tensors in HOST memory: q_host [B,H,D] is
  * copied to q_stage, the kernels run, out_stage is copied to out_host [B,H,D] and
  * the call returns after the stream has drained.  q_stage / out_stage are device
@@ -167,6 +213,22 @@ int chai_prefill_attention_simt(const void* q, const void* k_rep, const void* v,
                                 float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
                                 void* stream);
 size_t chai_prefill_workspace_bytes(int B, int H, int k, int T, int D, int dtype);
+
+/*
+ * Prefill that leaves the first q_start query rows alone (Section 3.3 / Fig. 6(b): the first five tokens
+ * of a request run with plain multi-head attention, whose scores decide the clusters; clustered attention
+ * takes over after them).  Rows [q_start, T) of `out` are computed exactly as by chai_prefill_attention --
+ * they still attend to keys 0..i -- and rows [0, q_start) are neither computed nor written.
+ * 0 <= q_start < T.  The plain-MHA rows themselves are a call with k = H and identity membership.
+ */
+int chai_prefill_attention_from(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                const int32_t* reps, void* out, int B, int H, int k, int T, int q_start, int D,
+                                float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
+                                void* stream);
+int chai_prefill_attention_simt_from(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                     const int32_t* reps, void* out, int B, int H, int k, int T, int q_start, int D,
+                                     float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
+                                     void* stream);
 
 /* Blocking read of the status word a decode/prefill call left in `workspace`
  * (synchronises `stream`).  *status_out receives a chai_status_t. */

@@ -159,3 +159,49 @@ def compact_k_cache(k_full: np.ndarray, reps) -> tuple[np.ndarray, tuple[int, in
     if rc != 0:
         raise ValueError("oracle_compact_k_cache rejected its arguments")
     return out, (int(nbytes[0]), int(nbytes[1]))
+
+
+# ---- serving-shaped steps (Section 3.5 / 4.3): each is the plain definition applied request by request ----
+
+def decode_attention_ragged(q, k_rep, v, membership, reps, seq_lens, scale: float) -> np.ndarray:
+    """Decode step of a ragged batch: request b attends to its first seq_lens[b] cached positions only.
+    q [B,H,D], k_rep [B,k,T_cap,D], v [B,H,T_cap,D] -> float64 [B,H,D]; a request with length 0 gets zeros."""
+    q, k_rep, v = _f64(q), _f64(k_rep), _f64(v)
+    membership, reps = _i32(membership), _i32(reps)
+    B, H, D = q.shape
+    out = np.zeros((B, H, D), dtype=np.float64)
+    for b in range(B):
+        n = int(seq_lens[b])
+        if n <= 0:
+            continue
+        out[b] = cha_attention(q[b:b + 1], k_rep[b:b + 1, :, :n], v[b:b + 1, :, :n], membership[b:b + 1],
+                               reps[b:b + 1], scale, False)[0]
+    return out
+
+
+def append_kv(k_new, v_new, k_rep, v, reps, seq_lens):
+    """One new token per request, written at row seq_lens[b]: the representatives' keys and every head's
+    values.  Arrays of any dtype (bit copies); returns (k_rep', v', seq_lens + 1) as new arrays."""
+    k_rep, v = np.array(k_rep, copy=True), np.array(v, copy=True)
+    reps = _i32(reps)
+    lens = np.array(seq_lens, dtype=np.int64, copy=True)
+    B, k = reps.shape
+    for b in range(B):
+        pos = int(lens[b])
+        if not 0 <= pos < v.shape[2]:
+            continue  # no room: the request is skipped
+        v[b, :, pos] = v_new[b]
+        for c in range(k):
+            r = int(reps[b, c])
+            if 0 <= r < v.shape[1]:
+                k_rep[b, c, pos] = k_new[b, r]
+        lens[b] = pos + 1
+    return k_rep, v, lens
+
+
+def compact_k_cache_inplace(k_full: np.ndarray, reps, T: int) -> np.ndarray:
+    """What the first k planes of each request hold after in-place compaction: the gather of
+    compact_k_cache over rows [0,T).  Returns [B,k,T,D]; slots with reps = -1 are returned as zeros and are
+    not compared (the in-place call leaves them as they were)."""
+    k_rep, _ = compact_k_cache(k_full[:, :, :T], reps)
+    return k_rep

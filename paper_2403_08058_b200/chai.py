@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_PKG, "libchai.so")
 
 CHAI_OK = 0
 CHAI_ERR_INVALID_ARG, CHAI_ERR_UNSUPPORTED, CHAI_ERR_WORKSPACE = 1, 2, 3
-CHAI_ERR_BAD_MEMBERSHIP, CHAI_ERR_TIMEOUT, CHAI_ERR_CUDA = 4, 5, 6
+CHAI_ERR_BAD_MEMBERSHIP, CHAI_ERR_TIMEOUT, CHAI_ERR_CUDA, CHAI_ERR_CACHE_FULL = 4, 5, 6, 7
 CHAI_F32, CHAI_BF16 = 0, 1
 
 # every symbol include/chai.h declares
@@ -25,6 +25,8 @@ EXPORTS = [
     "chai_decode_workspace_bytes", "chai_decode_attention_host", "chai_prefill_attention",
     "chai_prefill_attention_simt", "chai_prefill_workspace_bytes", "chai_device_status",
     "chai_status_string", "chai_last_error", "chai_version", "chai_decode_attention_static",
+    "chai_decode_attention_ragged", "chai_append_kv", "chai_compact_k_cache_inplace",
+    "chai_prefill_attention_from", "chai_prefill_attention_simt_from",
 ]
 DECODE_STATIC_SCRATCH_BYTES = 8 << 20   # CHAI_DECODE_STATIC_SCRATCH_BYTES
 
@@ -58,6 +60,11 @@ def load() -> ctypes.CDLL:
     for name in ("chai_decode_workspace_bytes", "chai_prefill_workspace_bytes"):
         getattr(lib, name).argtypes = [ci, ci, ci, ci, ci, ci]
         getattr(lib, name).restype = sz
+    lib.chai_decode_attention_ragged.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, sz, cf, ci, vp, sz, vp]
+    lib.chai_append_kv.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, sz, ci, ci, vp, vp]
+    lib.chai_compact_k_cache_inplace.argtypes = [vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, vp]
+    for name in ("chai_prefill_attention_from", "chai_prefill_attention_simt_from"):
+        getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
     lib.chai_decode_attention_static.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
     lib.chai_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
     lib.chai_status_string.argtypes = [ci]
@@ -192,6 +199,49 @@ def chai_decode_attention_static(q, k_rep, v, membership, reps, scale: float, T:
     return out
 
 
+def chai_decode_attention_ragged(q, k_rep, v, membership, reps, seq_lens, scale: float, T_max: int, k_planes=None,
+                                 out=None, workspace=None):
+    """Ragged batch: seq_lens [B] int32 (device) gives each request's cached positions, T_max bounds them.
+    k_rep is [B,k,T_cap,D], or (k_planes=k) a full [B,H,T_cap,D] cache whose first k planes hold the
+    representatives (after chai_compact_k_cache_inplace)."""
+    _dev(q, k_rep, v, membership, reps, seq_lens, out, workspace)
+    B, H, D = q.shape
+    k = reps.shape[1] if k_planes is None else k_planes
+    T_cap = k_rep.shape[2]
+    stride = k_rep.shape[1] * T_cap * D
+    dt = _dt(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(chai_decode_workspace_bytes(B, H, k, T_max, D, dt), q.device)
+    _check(load().chai_decode_attention_ragged(_ptr(q), _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps),
+                                               _ptr(seq_lens), _ptr(out), B, H, k, T_max, T_cap, D, stride, scale, dt,
+                                               _ptr(workspace), workspace.numel(), _stream()))
+    return out
+
+
+def chai_append_kv(k_new, v_new, k_rep, v, reps, seq_lens, advance: bool = True, workspace=None):
+    """One new token per request: k_rep[b][c][seq_lens[b]] = k_new[b][reps[b][c]], v[b][h][seq_lens[b]] = v_new[b][h];
+    seq_lens is incremented afterwards when `advance`.  k_rep may be the full cache compacted in place."""
+    _dev(k_new, v_new, k_rep, v, reps, seq_lens, workspace)
+    B, H, D = k_new.shape
+    k, T_cap = reps.shape[1], v.shape[2]
+    stride = k_rep.shape[1] * T_cap * D
+    _check(load().chai_append_kv(_ptr(k_new), _ptr(v_new), _ptr(k_rep), _ptr(v), _ptr(reps), _ptr(seq_lens), B, H, k,
+                                 T_cap, D, stride, _dt(k_new), int(bool(advance)), _ptr(workspace), _stream()))
+
+
+def chai_compact_k_cache_inplace(k_cache, reps, T: int | None = None, workspace=None):
+    """k_cache [B,H,T_cap,D]: planes 0..k-1 of each request receive the representatives' keys (rows [0,T))."""
+    _dev(k_cache, reps, workspace)
+    B, H, T_cap, D = k_cache.shape
+    k = reps.shape[1]
+    T = T_cap if T is None else T
+    _check(load().chai_compact_k_cache_inplace(_ptr(k_cache), _ptr(reps), B, H, k, T, T_cap, D, _dt(k_cache),
+                                               _ptr(workspace), _stream()))
+    return k_cache
+
+
 def chai_decode_attention_host(q_host, out_host, q_stage, out_stage, k_rep, v, membership, reps, scale: float,
                                workspace, T: int | None = None):
     """Decode step with q / out in (pinned) host memory; returns after the stream has drained."""
@@ -219,6 +269,34 @@ def _prefill(fn_name, q, k_rep, v, membership, reps, scale, causal, out, workspa
                                     T, D, scale, int(bool(causal)), dt, _ptr(workspace), workspace.numel(),
                                     _stream()))
     return out
+
+
+def _prefill_from(fn_name, q, k_rep, v, membership, reps, scale, q_start, causal, out, workspace):
+    _dev(q, k_rep, v, membership, reps, out, workspace)
+    B, H, T, D = q.shape
+    k = k_rep.shape[1]
+    dt = _dt(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(chai_prefill_workspace_bytes(B, H, k, T, D, dt), q.device)
+    _check(getattr(load(), fn_name)(_ptr(q), _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps), _ptr(out), B, H, k,
+                                    T, int(q_start), D, scale, int(bool(causal)), dt, _ptr(workspace),
+                                    workspace.numel(), _stream()))
+    return out
+
+
+def chai_prefill_attention_from(q, k_rep, v, membership, reps, scale: float, q_start: int, causal: bool = True,
+                                out=None, workspace=None):
+    """Rows [q_start, T) of the clustered prefill; rows before q_start of `out` are left untouched."""
+    return _prefill_from("chai_prefill_attention_from", q, k_rep, v, membership, reps, scale, q_start, causal, out,
+                         workspace)
+
+
+def chai_prefill_attention_simt_from(q, k_rep, v, membership, reps, scale: float, q_start: int, causal: bool = True,
+                                     out=None, workspace=None):
+    return _prefill_from("chai_prefill_attention_simt_from", q, k_rep, v, membership, reps, scale, q_start, causal, out,
+                         workspace)
 
 
 def chai_prefill_attention(q, k_rep, v, membership, reps, scale: float, causal: bool = True, out=None,

@@ -33,6 +33,7 @@ const char* chai_status_string(int status) {
         case CHAI_ERR_BAD_MEMBERSHIP: return "inconsistent membership / representatives";
         case CHAI_ERR_TIMEOUT: return "device-side wait expired";
         case CHAI_ERR_CUDA: return "CUDA error";
+        case CHAI_ERR_CACHE_FULL: return "cache position outside [0, T_cap)";
         default: return "unknown status";
     }
 }

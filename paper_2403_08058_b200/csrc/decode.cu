@@ -57,8 +57,9 @@ __device__ __forceinline__ float block_sum(float v, float* s_w) {
 template <typename T, int D>
 __global__ void __launch_bounds__(kDecThreads)
 decode_scores_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const int32_t* __restrict__ reps,
-                     WsHeader* __restrict__ hdr, int* __restrict__ counters, float* __restrict__ scores,
-                     float* __restrict__ cmax, int H, int k, int T_len, int T_cap, float scale, int nK) {
+                     const int32_t* __restrict__ seq_lens, WsHeader* __restrict__ hdr, int* __restrict__ counters,
+                     float* __restrict__ scores, float* __restrict__ cmax, int H, int k, int T_len, int T_cap,
+                     size_t k_batch_stride, float scale, int nK) {
     using G = DecodeGeom<T, D>;
     __shared__ float s_w[kDecWarps];
     const int chunk = blockIdx.x, c = blockIdx.y, b = blockIdx.z;
@@ -75,6 +76,7 @@ decode_scores_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const
     }
     const int r = reps[(size_t)b * k + c];
     if (r < 0 || r >= H) return;  // unused cluster slot: nothing reads its scores
+    const int len = seq_lens ? min(max(seq_lens[b], 0), T_len) : T_len;  // this request's context length
 
     const int sub = lane / G::LPR, part = lane % G::LPR;
     float qf[G::EPV];
@@ -82,7 +84,7 @@ decode_scores_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const
         const uint4 qv = *reinterpret_cast<const uint4*>(q + ((size_t)b * H + r) * D + part * G::EPV);
         Vec16<T>::unpack(qv, qf);
     }
-    const T* kbase = k_rep + ((size_t)b * k + c) * (size_t)T_cap * D + part * G::EPV;
+    const T* kbase = k_rep + (size_t)b * k_batch_stride + (size_t)c * T_cap * D + part * G::EPV;
     const int row0 = chunk * G::CK + warp * G::RPW + sub;
 
     uint4 buf[kStepsK];
@@ -90,7 +92,7 @@ decode_scores_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const
     for (int u = 0; u < kStepsK; ++u) {
         const int row = row0 + u * G::RPS;
         buf[u] = make_uint4(0, 0, 0, 0);
-        if (row < T_len) buf[u] = ld_stream16(kbase + (size_t)row * D);
+        if (row < len) buf[u] = ld_stream16(kbase + (size_t)row * D);
     }
     float lmax = -INFINITY;
     float* srow = scores + ((size_t)b * k + c) * (size_t)T_len;
@@ -105,7 +107,7 @@ decode_scores_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const
 #pragma unroll
         for (int o = G::LPR / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         s *= scale;
-        if (row < T_len) {
+        if (row < len) {
             if (part == 0) srow[row] = s;
             lmax = fmaxf(lmax, s);
         }
@@ -117,7 +119,7 @@ decode_scores_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const
 template <typename T, int D>
 __global__ void __launch_bounds__(kDecThreads)
 decode_pv_kernel(const T* __restrict__ v, const int32_t* __restrict__ membership, const int32_t* __restrict__ reps,
-                 WsHeader* __restrict__ hdr, int* __restrict__ counters, const float* __restrict__ scores,
+                 const int32_t* __restrict__ seq_lens, WsHeader* __restrict__ hdr, int* __restrict__ counters, const float* __restrict__ scores,
                  const float* __restrict__ cmax, float* __restrict__ lpart, float* __restrict__ opart,
                  T* __restrict__ out, int H, int k, int T_len, int T_cap, int nK, int nV) {
     using G = DecodeGeom<T, D>;
@@ -137,6 +139,7 @@ decode_pv_kernel(const T* __restrict__ v, const int32_t* __restrict__ membership
         return;
     }
 
+    const int len = seq_lens ? min(max(seq_lens[b], 0), T_len) : T_len;  // this request's context length
     // reference maximum of the whole row of scores (exact two-pass softmax)
     float m = -INFINITY;
     for (int i = tid; i < nK; i += kDecThreads) m = fmaxf(m, cmax[((size_t)b * k + c) * nK + i]);
@@ -147,7 +150,7 @@ decode_pv_kernel(const T* __restrict__ v, const int32_t* __restrict__ membership
     float lsum = 0.f;
     for (int t = tid; t < G::CV; t += kDecThreads) {
         const int row = row_base + t;
-        const float p = row < T_len ? expf(srow[row] - m) : 0.f;
+        const float p = row < len ? expf(srow[row] - m) : 0.f;
         s_p[t] = p;
         lsum += p;
     }
@@ -165,7 +168,7 @@ decode_pv_kernel(const T* __restrict__ v, const int32_t* __restrict__ membership
         for (int u = 0; u < 8; ++u) {
             const int lrow = (half * 8 + u) * G::RPS + warp * G::RPW + sub;
             buf[u] = make_uint4(0, 0, 0, 0);
-            if (row_base + lrow < T_len) buf[u] = ld_stream16(vbase + (size_t)(row_base + lrow) * D);
+            if (row_base + lrow < len) buf[u] = ld_stream16(vbase + (size_t)(row_base + lrow) * D);
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -210,15 +213,15 @@ decode_pv_kernel(const T* __restrict__ v, const int32_t* __restrict__ membership
             o += __ldcg(&opart[(head * nV + i) * D + tid]);
             ll += __ldcg(&lpart[head * nV + i]);
         }
-        out[head * D + tid] = from_float<T>(o / ll);
+        out[head * D + tid] = from_float<T>(ll > 0.f ? o / ll : 0.f);  // empty context: zero output
     }
     if (tid == 0) counters[head] = 0;
 }
 
 template <typename T, int D>
 static int launch_decode(const void* q, const void* k_rep, const void* v, const int32_t* membership,
-                         const int32_t* reps, void* out, int B, int H, int k, int T_len, int T_cap, float scale,
-                         char* ws, const DecodeLayout& L, cudaStream_t s) {
+                         const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T_len,
+                         int T_cap, size_t k_batch_stride, float scale, char* ws, const DecodeLayout& L, cudaStream_t s) {
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
     int* counters = reinterpret_cast<int*>(ws + L.off_counters);
     float* scores = reinterpret_cast<float*>(ws + L.off_scores);
@@ -226,11 +229,11 @@ static int launch_decode(const void* q, const void* k_rep, const void* v, const 
     float* lpart = reinterpret_cast<float*>(ws + L.off_lpart);
     float* opart = reinterpret_cast<float*>(ws + L.off_opart);
     decode_scores_kernel<T, D><<<dim3(L.nK, k, B), kDecThreads, 0, s>>>(
-        static_cast<const T*>(q), static_cast<const T*>(k_rep), reps, hdr, counters, scores, cmax, H, k, T_len, T_cap,
-        scale, L.nK);
+        static_cast<const T*>(q), static_cast<const T*>(k_rep), reps, seq_lens, hdr, counters, scores, cmax, H, k, T_len,
+        T_cap, k_batch_stride, scale, L.nK);
     CHAI_LAUNCH_CHECK("decode_scores_kernel launch");
-    decode_pv_kernel<T, D><<<dim3(L.nV, H, B), kDecThreads, 0, s>>>(static_cast<const T*>(v), membership, reps, hdr,
-                                                                   counters, scores, cmax, lpart, opart,
+    decode_pv_kernel<T, D><<<dim3(L.nV, H, B), kDecThreads, 0, s>>>(static_cast<const T*>(v), membership, reps, seq_lens,
+                                                                   hdr, counters, scores, cmax, lpart, opart,
                                                                    static_cast<T*>(out), H, k, T_len, T_cap, L.nK, L.nV);
     CHAI_LAUNCH_CHECK("decode_pv_kernel launch");
     return CHAI_OK;
@@ -247,24 +250,30 @@ size_t chai_decode_workspace_bytes(int B, int H, int k, int T, int D, int dtype)
     return L.total;
 }
 
-int chai_decode_attention(const void* q, const void* k_rep, const void* v, const int32_t* membership,
-                          const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D, float scale,
-                          int dtype, void* workspace, size_t workspace_bytes, void* stream) {
+namespace {
+// Common body of the decode entry points.  `fn` names the caller in messages.
+int decode_impl(const char* fn, const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T, int T_cap, int D,
+                size_t k_batch_stride, float scale, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
     using namespace chai;
-    CHAI_REQUIRE(q && k_rep && v && membership && reps && out && workspace, CHAI_ERR_INVALID_ARG,
-                 "chai_decode_attention: null pointer");
+    CHAI_REQUIRE(q && k_rep && v && membership && reps && out && workspace, CHAI_ERR_INVALID_ARG, "%s: null pointer", fn);
     CHAI_REQUIRE(aligned16(q) && aligned16(k_rep) && aligned16(v) && aligned16(out) && aligned16(workspace),
-                 CHAI_ERR_INVALID_ARG, "chai_decode_attention: pointers must be 16-byte aligned");
-    CHAI_REQUIRE(B > 0 && H > 0 && T > 0 && D > 0, CHAI_ERR_INVALID_ARG, "chai_decode_attention: sizes must be positive");
-    CHAI_REQUIRE(k >= 1 && k <= H, CHAI_ERR_INVALID_ARG, "chai_decode_attention: need 1 <= k <= H (k=%d, H=%d)", k, H);
-    CHAI_REQUIRE(T <= T_cap, CHAI_ERR_INVALID_ARG, "chai_decode_attention: T=%d exceeds T_cap=%d", T, T_cap);
-    CHAI_REQUIRE(dtype == CHAI_F32 || dtype == CHAI_BF16, CHAI_ERR_UNSUPPORTED, "chai_decode_attention: unknown dtype %d", dtype);
-    CHAI_REQUIRE(D == 64 || D == 128, CHAI_ERR_UNSUPPORTED, "chai_decode_attention: head_dim %d (64 or 128 supported)", D);
-    CHAI_REQUIRE(H <= 65535 && B <= 65535, CHAI_ERR_UNSUPPORTED, "chai_decode_attention: H and B must be <= 65535");
+                 CHAI_ERR_INVALID_ARG, "%s: pointers must be 16-byte aligned", fn);
+    CHAI_REQUIRE(B > 0 && H > 0 && T > 0 && D > 0, CHAI_ERR_INVALID_ARG, "%s: sizes must be positive", fn);
+    CHAI_REQUIRE(k >= 1 && k <= H, CHAI_ERR_INVALID_ARG, "%s: need 1 <= k <= H (k=%d, H=%d)", fn, k, H);
+    CHAI_REQUIRE(T <= T_cap, CHAI_ERR_INVALID_ARG, "%s: T=%d exceeds T_cap=%d", fn, T, T_cap);
+    CHAI_REQUIRE(dtype == CHAI_F32 || dtype == CHAI_BF16, CHAI_ERR_UNSUPPORTED, "%s: unknown dtype %d", fn, dtype);
+    CHAI_REQUIRE(D == 64 || D == 128, CHAI_ERR_UNSUPPORTED, "%s: head_dim %d (64 or 128 supported)", fn, D);
+    CHAI_REQUIRE(H <= 65535 && B <= 65535, CHAI_ERR_UNSUPPORTED, "%s: H and B must be <= 65535", fn);
+    const size_t dense = (size_t)k * T_cap * D;
+    if (k_batch_stride == 0) k_batch_stride = dense;
+    CHAI_REQUIRE(k_batch_stride >= dense && (k_batch_stride * elem_size(dtype)) % 16 == 0, CHAI_ERR_INVALID_ARG,
+                 "%s: k_batch_stride=%zu must be at least k*T_cap*D=%zu elements and a multiple of 16 bytes", fn,
+                 k_batch_stride, dense);
     DecodeLayout L;
     decode_layout(B, H, k, T, D, dtype, &L);
-    CHAI_REQUIRE(workspace_bytes >= L.total, CHAI_ERR_WORKSPACE,
-                 "chai_decode_attention: workspace has %zu bytes, %zu needed", workspace_bytes, L.total);
+    CHAI_REQUIRE(workspace_bytes >= L.total, CHAI_ERR_WORKSPACE, "%s: workspace has %zu bytes, %zu needed", fn,
+                 workspace_bytes, L.total);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
     // The persistent streaming kernel is the product path; the split kernels remain for devices
@@ -274,16 +283,39 @@ int chai_decode_attention(const void* q, const void* k_rep, const void* v, const
         return e != nullptr && strcmp(e, "split") == 0;
     }();
     if (!force_split) {
-        const int rc = launch_decode_persistent(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, D, scale, dtype,
-                                                ws, L, s);
+        const int rc = launch_decode_persistent(q, k_rep, v, membership, reps, seq_lens, out, B, H, k, T, T_cap, D,
+                                                k_batch_stride, scale, dtype, ws, L, s);
         if (rc != kDecodeNotLaunched) return rc;
     }
     if (dtype == CHAI_BF16) {
-        if (D == 128) return launch_decode<__nv_bfloat16, 128>(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, scale, ws, L, s);
-        return launch_decode<__nv_bfloat16, 64>(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, scale, ws, L, s);
+        if (D == 128)
+            return launch_decode<__nv_bfloat16, 128>(q, k_rep, v, membership, reps, seq_lens, out, B, H, k, T, T_cap,
+                                                     k_batch_stride, scale, ws, L, s);
+        return launch_decode<__nv_bfloat16, 64>(q, k_rep, v, membership, reps, seq_lens, out, B, H, k, T, T_cap,
+                                                k_batch_stride, scale, ws, L, s);
     }
-    if (D == 128) return launch_decode<float, 128>(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, scale, ws, L, s);
-    return launch_decode<float, 64>(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, scale, ws, L, s);
+    if (D == 128)
+        return launch_decode<float, 128>(q, k_rep, v, membership, reps, seq_lens, out, B, H, k, T, T_cap, k_batch_stride,
+                                         scale, ws, L, s);
+    return launch_decode<float, 64>(q, k_rep, v, membership, reps, seq_lens, out, B, H, k, T, T_cap, k_batch_stride, scale,
+                                    ws, L, s);
+}
+}  // namespace
+
+int chai_decode_attention(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                          const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D, float scale,
+                          int dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    return decode_impl("chai_decode_attention", q, k_rep, v, membership, reps, nullptr, out, B, H, k, T, T_cap, D, 0,
+                       scale, dtype, workspace, workspace_bytes, stream);
+}
+
+int chai_decode_attention_ragged(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                 const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k,
+                                 int T_max, int T_cap, int D, size_t k_batch_stride, float scale, int dtype,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+    CHAI_REQUIRE(seq_lens != nullptr, CHAI_ERR_INVALID_ARG, "chai_decode_attention_ragged: seq_lens is null");
+    return decode_impl("chai_decode_attention_ragged", q, k_rep, v, membership, reps, seq_lens, out, B, H, k, T_max,
+                       T_cap, D, k_batch_stride, scale, dtype, workspace, workspace_bytes, stream);
 }
 
 int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage, void* out_stage, const void* k_rep,

@@ -54,8 +54,13 @@ inline bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLa
 // Persistent decode kernel (decode_persist.cu).  Returns CHAI_OK, an error, or kDecodeNotLaunched
 // when the device cannot run it (no cooperative launch), in which case the caller uses the split kernels.
 constexpr int kDecodeNotLaunched = -1;
+// seq_lens: per-request context lengths on the device (null: every request has T positions; otherwise T is
+// the upper bound the workspace was sized for).  k_batch_stride: elements between two requests' first
+// representative plane in k_rep (k * T_cap * D for a dense representative cache, H * T_cap * D for a cache
+// compacted in place).
 int launch_decode_persistent(const void* q, const void* k_rep, const void* v, const int32_t* membership,
-                             const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D, float scale,
-                             int dtype, char* ws, const DecodeLayout& L, cudaStream_t s);
+                             const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T,
+                             int T_cap, int D, size_t k_batch_stride, float scale, int dtype, char* ws,
+                             const DecodeLayout& L, cudaStream_t s);
 
 }  // namespace chai

@@ -69,6 +69,8 @@ struct Params {
     const void* v;
     const int32_t* membership;
     const int32_t* reps;
+    const int32_t* seq_lens;     // per-request context length, or null (all T)
+    size_t k_batch_bytes;        // bytes between two requests' representative planes in k_rep
     void* out;
     WsHeader* hdr;
     int* counters;               // tickets, one per head
@@ -204,7 +206,10 @@ struct Ring {
     __device__ __forceinline__ uint32_t data(int slot) const { return data0 + kTileBytes * slot; }
 };
 
-template <typename T, int D>
+// RAGGED = false is the equal-length, dense-cache case: per-request lengths, the K batch stride and the
+// skipping of tiles beyond a request's end compile away (the streaming loops are sensitive to every
+// instruction on the producer thread and in the per-tile consumer chain).
+template <typename T, int D, bool RAGGED>
 __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Params P) {
     using G = Geom<T, D>;
     constexpr int W = CONSUMER_WARPS;
@@ -249,7 +254,24 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
         int c, r;
         return resolve_head(P.membership, P.reps, b, h, H, k, &c, &r) ? c : -1;
     };
-    auto tile_rows = [&](int tile) { return max(0, min(G::TR, T_len - tile * G::TR)); };
+    // rows of request b's tile: requests shorter than T leave whole tiles empty (they pass through the ring as
+    // markers without data and contribute nothing)
+    auto len_of = [&](int b) {
+        if constexpr (RAGGED) return P.seq_lens ? min(max(__ldg(P.seq_lens + b), 0), T_len) : T_len;
+        return T_len;
+    };
+    auto tile_rows = [&](int b, int tile) { return max(0, min(G::TR, len_of(b) - tile * G::TR)); };
+    // Tiles that hold cached rows of request b (tile 0 always counts, so that an empty request still runs
+    // through the bookkeeping once), and the value items (runs of IV tiles) they make.  Tiles and items
+    // beyond these are skipped by the producer and the consumers alike: they never enter the ring.
+    auto tiles_of = [&](int b) {
+        if constexpr (RAGGED) return max(1, (len_of(b) + G::TR - 1) / G::TR);
+        return tp;
+    };
+    auto items_of = [&](int b) {
+        if constexpr (RAGGED) return (tiles_of(b) + P.IV - 1) / P.IV;
+        return P.nVi;
+    };
     const unsigned char* kc = static_cast<const unsigned char*>(P.k_rep);
     const unsigned char* vc = static_cast<const unsigned char*>(P.v);
 
@@ -288,9 +310,17 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                 int plane = cta / tp, tile = cta % tp;
                 const int dplane = ncta / tp, dtile = ncta % tp;
                 const TileMeta m{0, 0, 0, 0};
+                constexpr bool plain = !RAGGED;
                 for (int t = 0; t < nkt && ok; ++t) {
-                    ok = issue(kc + ((size_t)plane * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
-                               (uint32_t)tile_rows(tile) * G::ROW_BYTES, m);
+                    if constexpr (plain) {  // equal lengths, dense cache: no per-tile division on this (single) thread
+                        ok = issue(kc + ((size_t)plane * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
+                                   (uint32_t)tile_rows(0, tile) * G::ROW_BYTES, m);
+                    } else {
+                        const int b = plane / k, c = plane - b * k;
+                        if (tile < tiles_of(b))
+                            ok = issue(kc + (size_t)b * P.k_batch_bytes + ((size_t)c * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
+                                       (uint32_t)tile_rows(b, tile) * G::ROW_BYTES, m);
+                    }
                     plane += dplane;
                     tile += dtile;
                     if (tile >= tp) {
@@ -309,7 +339,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                 next = atomicAdd(work_counter, 1);
                 const int head = item / P.nVi, chunk = item % P.nVi;
                 const int tile0 = chunk * P.IV;
-                const int ntiles = min(P.IV, tp - tile0);
+                const int b_item = RAGGED ? head / H : 0;
+                const int ntiles = min(P.IV, tiles_of(b_item) - tile0);
+                if (RAGGED && ntiles <= 0) continue;  // the request is shorter: this item does not exist
                 const int islot = n_open % ITEM_SLOTS;
                 ++n_open;
                 ok = word_wait(&sm.item_free[islot], 1, abort_flag);  // the slot's previous item is fully reduced
@@ -319,7 +351,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                     const int tile = tile0 + t;
                     const TileMeta m{item, t, ntiles, islot};
                     ok = issue(vc + ((size_t)head * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
-                               (uint32_t)tile_rows(tile) * G::ROW_BYTES, m);
+                               (uint32_t)tile_rows(b_item, tile) * G::ROW_BYTES, m);
                 }
             }
             // ---- one end marker per consumer warp ----
@@ -330,13 +362,22 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
         // ------------------------------ consumers: every warp works alone ------------------------------
         const int sub = lane / G::LPR, part = lane % G::LPR;
         bool ok = true;
-        int n = warp;  // this warp owns ring positions warp, warp + W, ...
+        // this warp owns ring positions warp, warp + W, ...; the key tiles of this CTA take positions in the
+        // order of their ids, those beyond their request's length take none
+        constexpr bool ragged = RAGGED;
+        int n_issued = ragged ? 0 : nkt;
         // ---- phase K: one tile = TR scores and their maximum ----
-        for (; n < nkt; n += W) {
-            const long long g = (long long)cta + (long long)n * ncta;
+        for (int t_idx = ragged ? 0 : warp; t_idx < nkt; t_idx += ragged ? 1 : W) {
+            const long long g = (long long)cta + (long long)t_idx * ncta;
             const int plane = (int)(g / tp), tile = (int)(g % tp);
             const int b = plane / k;
-            const int rows = tile_rows(tile);
+            int n = t_idx;  // ring position of this tile
+            if constexpr (ragged) {
+                if (tile >= tiles_of(b)) continue;
+                if ((n_issued++ % W) != warp) continue;
+                n = n_issued - 1;
+            }
+            const int rows = tile_rows(b, tile);
             const int rep = P.reps[plane];
             const bool live = rep >= 0 && rep < H;  // unused cluster slot: the tile is drained, nothing computed
             float qf[G::EPV];
@@ -349,7 +390,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
             const int slot = n % STAGES;
             if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag) &&
                                                      mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
-            if (ok && live) {
+            if (ok && live && rows == 0) {  // tile beyond this request's length: no scores, neutral maximum
+                if (lane == 0) P.cmax[(size_t)plane * tp + tile] = -INFINITY;
+            } else if (ok && live) {
                 const unsigned char* data = sm.ring[slot];
                 float* srow = P.scores + (size_t)plane * T_len + (size_t)tile * G::TR;
                 float lmax = -INFINITY;
@@ -418,7 +461,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
         }
         // ---- phase V: tiles of claimed items ----
         T* outp = static_cast<T*>(P.out);
-        for (;; n += W) {
+        for (int n = n_issued + ((warp - n_issued) % W + W) % W;; n += W) {  // this warp's next position
             const int slot = n % STAGES;
             if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag) &&
                                                      mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
@@ -432,7 +475,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
             const int head = m.item / P.nVi, chunk = m.item % P.nVi;
             const int b = head / H, h = head % H;
             const int tile = chunk * P.IV + m.t;
-            const int rows = tile_rows(tile);
+            const int rows = tile_rows(b, tile);
             const int c = cluster_of(b, h);
             const bool live = c >= 0;
             float acc[G::EPV];
@@ -445,12 +488,13 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                 // after the first tiles of phase V this is a shared-memory bit test)
                 const bool cached = plane < TABLE_CAP && ((*reinterpret_cast<volatile unsigned*>(&sm.ready[plane >> 5]) >> (plane & 31)) & 1u);
                 if (!cached) {
-                    ok = flags_wait(P.flags + plane * tp, tp, P.token, lane, abort_flag);
+                    ok = flags_wait(P.flags + plane * tp, tiles_of(b), P.token, lane, abort_flag);
                     if (ok && lane == 0 && plane < TABLE_CAP) atomicOr(&sm.ready[plane >> 5], 1u << (plane & 31));
                 }
-                if (ok) {
+                if (ok && rows > 0) {  // (the only tile of an empty request has no rows: it just passes the ticket on,
+                                       //  which the flag wait above has ordered after the ticket's reset)
                     float mx = -INFINITY;
-                    for (int x = lane; x < tp; x += 32) mx = fmaxf(mx, __ldcg(&P.cmax[plane * tp + x]));
+                    for (int x = lane, nx = tiles_of(b); x < nx; x += 32) mx = fmaxf(mx, __ldcg(&P.cmax[plane * tp + x]));
                     const float* srow = P.scores + plane * T_len + (size_t)tile * G::TR;
                     float pv[G::PV];
 #pragma unroll
@@ -555,19 +599,21 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
             int ticket = 0;
             if (lane == 0) ticket = atomicAdd(&P.counters[head], 1);
             ticket = __shfl_sync(0xffffffffu, ticket, 0);
-            if (ticket == P.nVi - 1) {  // this warp completed the head: add the item partials in chunk order
+            const int n_chunks = items_of(b);  // items this head really has
+            if (ticket == n_chunks - 1) {  // this warp completed the head: add the item partials in chunk order
                 __threadfence();
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) o[e] = 0.f;
                 float ll = 0.f;
-                for (int i = 0; i < P.nVi; ++i) {
+                for (int i = 0; i < n_chunks; ++i) {
                     const float* src = P.opart + ((size_t)head * P.nVi + i) * D + lane * DPL;
 #pragma unroll
                     for (int e = 0; e < DPL; ++e) o[e] += __ldcg(src + e);
                     ll += __ldcg(&P.lpart[(size_t)head * P.nVi + i]);
                 }
 #pragma unroll
-                for (int e = 0; e < DPL; ++e) outp[(size_t)head * D + lane * DPL + e] = from_float<T>(o[e] / ll);
+                for (int e = 0; e < DPL; ++e)  // (an empty context has no probabilities: the output is zero)
+                    outp[(size_t)head * D + lane * DPL + e] = from_float<T>(ll > 0.f ? o[e] / ll : 0.f);
             }
         }
     }
@@ -592,24 +638,24 @@ static DeviceInfo& device_info(int dev) {
     return d;
 }
 
-template <typename T, int D>
+template <typename T, int D, bool RAGGED>
 static int launch(const Params& P0, int ncta, int dev, cudaStream_t s) {
     Params P = P0;
     const size_t smem = sizeof(Smem) + 128;
     static bool configured_dev[64] = {};
     bool& configured = configured_dev[dev & 63];
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(decode_persistent_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(decode_persistent_kernel<T, D, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel shared-memory opt-in");
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_persistent_kernel<T, D>, THREADS, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_persistent_kernel<T, D, RAGGED>, THREADS, smem);
         if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel occupancy query");
         if (per_sm < 1) return kDecodeNotLaunched;
         configured = true;
     }
     void* args[] = {&P};
     // cooperative launch: value tiles wait for flags set by other CTAs, so all CTAs must be resident at once
-    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_persistent_kernel<T, D>), dim3(ncta),
+    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_persistent_kernel<T, D, RAGGED>), dim3(ncta),
                                                 dim3(THREADS), args, smem, s);
     if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel launch");
     return CHAI_OK;
@@ -618,8 +664,9 @@ static int launch(const Params& P0, int ncta, int dev, cudaStream_t s) {
 }  // namespace pd
 
 int launch_decode_persistent(const void* q, const void* k_rep, const void* v, const int32_t* membership,
-                             const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D, float scale,
-                             int dtype, char* ws, const DecodeLayout& L, cudaStream_t s) {
+                             const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T,
+                             int T_cap, int D, size_t k_batch_stride, float scale, int dtype, char* ws,
+                             const DecodeLayout& L, cudaStream_t s) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return kDecodeNotLaunched;
     const pd::DeviceInfo& info = pd::device_info(dev);
@@ -628,6 +675,8 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     const int tiles = (T + L.TR - 1) / L.TR;
     pd::Params P;
     P.q = q; P.k_rep = k_rep; P.v = v; P.membership = membership; P.reps = reps; P.out = out;
+    P.seq_lens = seq_lens;
+    P.k_batch_bytes = k_batch_stride * elem_size(dtype);
     P.hdr = reinterpret_cast<WsHeader*>(ws);
     P.counters = reinterpret_cast<int*>(ws + L.off_counters);
     P.flags = reinterpret_cast<unsigned long long*>(ws + L.off_flags);
@@ -648,12 +697,13 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     P.nVi = (tiles + P.IV - 1) / P.IV;
     P.scale = scale;
     if (tiles > L.capK || P.nVi > L.capV || (long long)B * H * P.nVi > 0x7fffffffll) return kDecodeNotLaunched;
+    const bool ragged = seq_lens != nullptr || k_batch_stride != (size_t)k * T_cap * D;
     if (dtype == CHAI_BF16) {
-        if (D == 128) return pd::launch<__nv_bfloat16, 128>(P, ncta, dev, s);
-        return pd::launch<__nv_bfloat16, 64>(P, ncta, dev, s);
+        if (D == 128) return ragged ? pd::launch<__nv_bfloat16, 128, true>(P, ncta, dev, s) : pd::launch<__nv_bfloat16, 128, false>(P, ncta, dev, s);
+        return ragged ? pd::launch<__nv_bfloat16, 64, true>(P, ncta, dev, s) : pd::launch<__nv_bfloat16, 64, false>(P, ncta, dev, s);
     }
-    if (D == 128) return pd::launch<float, 128>(P, ncta, dev, s);
-    return pd::launch<float, 64>(P, ncta, dev, s);
+    if (D == 128) return ragged ? pd::launch<float, 128, true>(P, ncta, dev, s) : pd::launch<float, 128, false>(P, ncta, dev, s);
+    return ragged ? pd::launch<float, 64, true>(P, ncta, dev, s) : pd::launch<float, 64, false>(P, ncta, dev, s);
 }
 
 }  // namespace chai

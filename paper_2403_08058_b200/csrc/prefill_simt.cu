@@ -14,8 +14,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
 prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const T* __restrict__ v,
                     const int* __restrict__ n_groups, const GroupEntry* __restrict__ groups, T* __restrict__ out,
-                    WsHeader* __restrict__ hdr, const int* __restrict__ bad, int H, int k, int T_len, float scale,
-                    int causal, int n_qtiles) {
+                    WsHeader* __restrict__ hdr, const int* __restrict__ bad, int H, int k, int T_len, int q_start,
+                    float scale, int causal, int n_qtiles) {
     constexpr int DP = D + 1;         // padded row: conflict-free column walks
     constexpr int DPT = D / 4;        // output columns per thread
     extern __shared__ float smem_f[];
@@ -37,7 +37,8 @@ prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const 
         for (int g = 0; g < e.n; ++g)
             for (int idx = tid; idx < kSimtBQ * D; idx += kSimtThreads) {
                 const int row = q0 + idx / D;
-                if (row < T_len) out[(((size_t)b * H + e.heads[g]) * T_len + row) * D + idx % D] = from_float<T>(0.f);
+                if (row >= q_start && row < T_len)
+                    out[(((size_t)b * H + e.heads[g]) * T_len + row) * D + idx % D] = from_float<T>(0.f);
             }
         return;
     }
@@ -116,7 +117,7 @@ prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const 
             }
         }
     }
-    if (i_abs < T_len) {
+    if (i_abs >= q_start && i_abs < T_len) {  // rows before q_start belong to the caller (prefix computed earlier)
         const float inv = 1.f / l_run;
 #pragma unroll
         for (int gg = 0; gg < kSimtG; ++gg) {
@@ -131,14 +132,15 @@ prefill_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const 
 template <typename T, int D>
 static int launch_prefill_simt(const void* q, const void* k_rep, const void* v, const int* n_groups,
                                const GroupEntry* groups, void* out, WsHeader* hdr, const int* bad, int B, int H, int k,
-                               int T_len, float scale, int causal, cudaStream_t s) {
+                               int T_len, int q_start, float scale, int causal, cudaStream_t s) {
     const int n_qtiles = (T_len + kSimtBQ - 1) / kSimtBQ;
+    const int qt0 = q_start / kSimtBQ;  // query tiles below this one hold no row to compute
     const size_t smem = sizeof(float) * ((size_t)kSimtBQ * (D + 1) + (size_t)kSimtBK * (D + 1) + (size_t)kSimtBK * D + 32 * 33);
     cudaError_t e = cudaFuncSetAttribute(prefill_simt_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e, "prefill_simt_kernel shared-memory opt-in");
-    prefill_simt_kernel<T, D><<<dim3(n_qtiles, H, B), kSimtThreads, smem, s>>>(
+    prefill_simt_kernel<T, D><<<dim3(n_qtiles - qt0, H, B), kSimtThreads, smem, s>>>(
         static_cast<const T*>(q), static_cast<const T*>(k_rep), static_cast<const T*>(v), n_groups, groups,
-        static_cast<T*>(out), hdr, bad, H, k, T_len, scale, causal, n_qtiles);
+        static_cast<T*>(out), hdr, bad, H, k, T_len, q_start, scale, causal, n_qtiles);
     CHAI_LAUNCH_CHECK("prefill_simt_kernel launch");
     return CHAI_OK;
 }
@@ -187,13 +189,16 @@ size_t chai_prefill_workspace_bytes(int B, int H, int k, int T, int D, int dtype
     return chai::prefill_layout(B, H).total;
 }
 
-int chai_prefill_attention_simt(const void* q, const void* k_rep, const void* v, const int32_t* membership,
-                                const int32_t* reps, void* out, int B, int H, int k, int T, int D, float scale,
-                                int causal, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
+int chai_prefill_attention_simt_from(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                     const int32_t* reps, void* out, int B, int H, int k, int T, int q_start, int D,
+                                     float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
+                                     void* stream) {
     using namespace chai;
-    int rc = prefill_check_args("chai_prefill_attention_simt", q, k_rep, v, membership, reps, out, B, H, k, T, D, dtype,
-                                workspace, workspace_bytes);
+    const char* fn = "chai_prefill_attention_simt";
+    int rc = prefill_check_args(fn, q, k_rep, v, membership, reps, out, B, H, k, T, D, dtype, workspace, workspace_bytes);
     if (rc != CHAI_OK) return rc;
+    CHAI_REQUIRE(q_start >= 0 && q_start < T, CHAI_ERR_INVALID_ARG, "%s: need 0 <= q_start < T (q_start=%d, T=%d)", fn,
+                 q_start, T);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
     rc = prefill_run_plan(membership, reps, B, H, k, kSimtG, ws, s);
@@ -204,11 +209,19 @@ int chai_prefill_attention_simt(const void* q, const void* k_rep, const void* v,
     WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
     const int* bad = reinterpret_cast<const int*>(ws + L.off_bad);
     if (dtype == CHAI_BF16) {
-        if (D == 128) return launch_prefill_simt<__nv_bfloat16, 128>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, scale, causal, s);
-        return launch_prefill_simt<__nv_bfloat16, 64>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, scale, causal, s);
+        if (D == 128)
+            return launch_prefill_simt<__nv_bfloat16, 128>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, q_start, scale, causal, s);
+        return launch_prefill_simt<__nv_bfloat16, 64>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, q_start, scale, causal, s);
     }
-    if (D == 128) return launch_prefill_simt<float, 128>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, scale, causal, s);
-    return launch_prefill_simt<float, 64>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, scale, causal, s);
+    if (D == 128) return launch_prefill_simt<float, 128>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, q_start, scale, causal, s);
+    return launch_prefill_simt<float, 64>(q, k_rep, v, ng, gr, out, hdr, bad, B, H, k, T, q_start, scale, causal, s);
+}
+
+int chai_prefill_attention_simt(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                const int32_t* reps, void* out, int B, int H, int k, int T, int D, float scale,
+                                int causal, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    return chai_prefill_attention_simt_from(q, k_rep, v, membership, reps, out, B, H, k, T, 0, D, scale, causal, dtype,
+                                            workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

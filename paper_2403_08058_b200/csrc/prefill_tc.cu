@@ -320,8 +320,8 @@ __global__ void __launch_bounds__(THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int* __restrict__ n_groups,
                   const GroupEntry* __restrict__ groups, __nv_bfloat16* __restrict__ out, WsHeader* __restrict__ hdr,
-                  const int* __restrict__ bad, int B_total, int b_begin, int B, int H, int k, int T_len, float scale_log2,
-                  int causal, int n_qtiles, int counter_slot) {
+                  const int* __restrict__ bad, int B_total, int b_begin, int B, int H, int k, int T_len, int q_start,
+                  float scale_log2, int causal, int n_qtiles, int counter_slot) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw;
@@ -382,7 +382,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // ---------------- producer: work distribution and TMA loads ----------------
         if (lane == 0) {
             const int n_pairs = prefix[B];                 // (request, group) pairs that exist
-            const int n_items = n_pairs * n_qtiles;        // heaviest query tiles first
+            const int n_items = n_pairs * (n_qtiles - q_start / BM);  // heaviest query tiles first; tiles below q_start hold no row to compute
             bool ok = true;
             int it = 0, qi = 0, kt = 0;                    // items published, items with loads, key tiles issued
             // Work items are fetched one ahead: the atomic that claims the next item is issued before the
@@ -585,7 +585,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const int n_kv = item.n_kv, n_members = item.n_members, q0 = item.q0;
             const int row_abs = q0 + row;
             if (n_kv == 0) {  // unresolved heads: zero rows
-                if (row_abs < T_len)
+                if (row_abs >= q_start && row_abs < T_len)
                     for (int g = 0; g < n_members; ++g) {
                         uint4* o = reinterpret_cast<uint4*>(out + ((size_t)item.o_plane[g] * T_len + row_abs) * HD + cbase);
 #pragma unroll
@@ -795,7 +795,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             if (ep.n_members == 1) mbar_arrive(bar.o_free(1));  // keep the unused barrier's phase in step
                         }
                     }
-                    if (row_abs < T_len) {
+                    if (row_abs >= q_start && row_abs < T_len) {  // rows before q_start belong to the caller
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
                             uint32_t w[8];
@@ -857,16 +857,24 @@ static bool make_map(CUtensorMap* map, const void* base, int planes, int T) {
 }  // namespace tc
 }  // namespace chai
 
-extern "C" int chai_prefill_attention(const void* q, const void* k_rep, const void* v, const int32_t* membership,
-                                      const int32_t* reps, void* out, int B, int H, int k, int T, int D, float scale,
-                                      int causal, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
+extern "C" int chai_prefill_attention_simt_from(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                                const int32_t* reps, void* out, int B, int H, int k, int T, int q_start,
+                                                int D, float scale, int causal, int dtype, void* workspace,
+                                                size_t workspace_bytes, void* stream);
+
+extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                           const int32_t* reps, void* out, int B, int H, int k, int T, int q_start, int D,
+                                           float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
+                                           void* stream) {
     using namespace chai;
     if (dtype != CHAI_BF16 || D != tc::HD || B > 60 * tc::MAX_B)
-        return chai_prefill_attention_simt(q, k_rep, v, membership, reps, out, B, H, k, T, D, scale, causal, dtype,
-                                           workspace, workspace_bytes, stream);
+        return chai_prefill_attention_simt_from(q, k_rep, v, membership, reps, out, B, H, k, T, q_start, D, scale, causal,
+                                                dtype, workspace, workspace_bytes, stream);
     int rc = prefill_check_args("chai_prefill_attention", q, k_rep, v, membership, reps, out, B, H, k, T, D, dtype,
                                 workspace, workspace_bytes);
     if (rc != CHAI_OK) return rc;
+    CHAI_REQUIRE(q_start >= 0 && q_start < T, CHAI_ERR_INVALID_ARG,
+                 "chai_prefill_attention: need 0 <= q_start < T (q_start=%d, T=%d)", q_start, T);
     CUtensorMap mq, mk, mv;
     CHAI_REQUIRE(tc::make_map(&mq, q, B * H, T) && tc::make_map(&mk, k_rep, B * k, T) && tc::make_map(&mv, v, B * H, T),
                  CHAI_ERR_CUDA, "chai_prefill_attention: cuTensorMapEncodeTiled failed");
@@ -906,10 +914,17 @@ extern "C" int chai_prefill_attention(const void* q, const void* k_rep, const vo
         cudaError_t le = cudaLaunchKernelEx(
             &cfg, tc::prefill_tc_kernel, mq, mk, mv, reinterpret_cast<const int*>(ws + L.off_ngroups),
             reinterpret_cast<const GroupEntry*>(ws + L.off_groups), static_cast<__nv_bfloat16*>(out),
-            reinterpret_cast<WsHeader*>(ws), reinterpret_cast<const int*>(ws + L.off_bad), B, b0, nb, H, k, T,
+            reinterpret_cast<WsHeader*>(ws), reinterpret_cast<const int*>(ws + L.off_bad), B, b0, nb, H, k, T, q_start,
             scale * 1.4426950408889634f, causal, n_qtiles, chunk);
         if (le != cudaSuccess) return cuda_fail(le, "prefill_tc_kernel launch");
         CHAI_LAUNCH_CHECK("prefill_tc_kernel launch");
     }
     return CHAI_OK;
+}
+
+extern "C" int chai_prefill_attention(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                      const int32_t* reps, void* out, int B, int H, int k, int T, int D, float scale,
+                                      int causal, int dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    return chai_prefill_attention_from(q, k_rep, v, membership, reps, out, B, H, k, T, 0, D, scale, causal, dtype,
+                                       workspace, workspace_bytes, stream);
 }

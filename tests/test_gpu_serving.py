@@ -1,0 +1,159 @@
+"""GPU parity of the serving-shaped steps: ragged decode, cache append, in-place compaction, prefill that
+starts after the plain-attention prefix.  Each CUDA result is compared with the CPU oracle on the same bits."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import chai_oracle as orc
+from paper_2403_08058_b200 import chai, synth
+from parity import assert_parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def bits(t: torch.Tensor) -> np.ndarray:
+    """Bit pattern of a tensor as an integer numpy array (bf16 has no numpy dtype)."""
+    t = t.detach().cpu().contiguous()
+    return t.view(torch.int16).numpy() if t.dtype == torch.bfloat16 else t.view(torch.int32).numpy()
+
+
+def ragged_case(cfg, seed, B, H, k, T_cap, D=128):
+    case = synth.decode_layer(cfg, seed=seed, B=B, H=H, T=T_cap, T_cap=T_cap, k=k, with_k_full=True)
+    if D == 64:
+        for n in ("q", "k_rep", "v", "k_full"):
+            case[n] = case[n][..., :64].contiguous()
+        case["scale"] = 0.125
+    return case
+
+
+@pytest.mark.parametrize("cfg,D", [(1, 128), (2, 128), (2, 64)])
+@pytest.mark.parametrize("lens", [[700, 1, 129, 0, 333], [128, 256, 384, 512, 640], [5, 5, 5, 5, 5], [0, 0, 0, 0, 1]])
+def test_ragged_decode(cfg, D, lens):
+    case = ragged_case(cfg, sum(lens), 5, 12, 3, 700, D)
+    seq = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    out = chai.chai_decode_attention_ragged(case["q"].to(DEV), case["k_rep"].to(DEV), case["v"].to(DEV),
+                                            case["membership"].to(DEV), case["reps"].to(DEV), seq, case["scale"],
+                                            T_max=max(max(lens), 1))
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy()
+    ref = orc.decode_attention_ragged(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], lens,
+                                      case["scale"])
+    assert np.isfinite(got).all()
+    assert_parity(got, ref, case["dtype"], f"ragged decode cfg {cfg} D {D} lens {lens}")
+    for b, n in enumerate(lens):
+        if n == 0:
+            assert not got[b].any()
+
+
+def test_ragged_decode_never_reads_beyond_a_request():
+    """Rows at or after seq_lens[b] hold NaN: the output must not notice."""
+    lens = [300, 17, 129]
+    case = ragged_case(2, 4, 3, 8, 4, 300)
+    k_rep, v = case["k_rep"].clone(), case["v"].clone()
+    for b, n in enumerate(lens):
+        k_rep[b, :, n:] = float("nan")
+        v[b, :, n:] = float("nan")
+    seq = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    out = chai.chai_decode_attention_ragged(case["q"].to(DEV), k_rep.to(DEV), v.to(DEV), case["membership"].to(DEV),
+                                            case["reps"].to(DEV), seq, case["scale"], T_max=300)
+    got = out.float().cpu().numpy()
+    ref = orc.decode_attention_ragged(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], lens,
+                                      case["scale"])
+    assert np.isfinite(got).all()
+    assert_parity(got, ref, "bf16", "ragged decode with poisoned tails")
+
+
+@pytest.mark.parametrize("cfg", [1, 2])
+def test_inplace_compaction_then_decode_and_append(cfg):
+    """The whole serving hand-over on one buffer: compaction in place, decode from the strided cache, append a
+    token (representatives' keys only, every head's values), decode again over one more position."""
+    B, H, k, T_cap = 3, 12, 4, 260
+    lens = [200, 259, 64]
+    case = ragged_case(cfg, 21, B, H, k, T_cap)
+    reps = case["reps"]
+    assert all(int(reps[b, c]) >= c for b in range(B) for c in range(k))
+    cache = case["k_full"].to(DEV).clone()
+    before = bits(cache)
+    ws = chai.new_workspace(256, DEV)
+    chai.chai_compact_k_cache_inplace(cache, reps.to(DEV), T=T_cap, workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_OK
+    after = bits(cache)
+    want = orc.compact_k_cache_inplace(bits(case["k_full"]), reps, T_cap)
+    assert np.array_equal(after[:, :k], want)                       # bit copy of the representatives
+    seq = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    d = {n: case[n].to(DEV) for n in ("q", "v", "membership", "reps")}
+    v = d["v"].clone()
+    out = chai.chai_decode_attention_ragged(d["q"], cache, v, d["membership"], d["reps"], seq, case["scale"],
+                                            T_max=T_cap)
+    ref = orc.decode_attention_ragged(case["q"], case["k_rep"], case["v"], case["membership"], reps, lens, case["scale"])
+    assert_parity(out.float().cpu().numpy(), ref, case["dtype"], "decode from a cache compacted in place")
+    # append one token per request
+    g = torch.Generator().manual_seed(3)
+    k_new = (torch.randn(B, H, case["q"].shape[-1], generator=g) * 0.5).to(case["q"].dtype)
+    v_new = (torch.randn(B, H, case["q"].shape[-1], generator=g) * 0.5).to(case["q"].dtype)
+    chai.chai_append_kv(k_new.to(DEV), v_new.to(DEV), cache, v, d["reps"], seq, advance=True, workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_OK
+    assert seq.cpu().tolist() == [n + 1 for n in lens]
+    k_ref, v_ref, lens_ref = orc.append_kv(bits(k_new), bits(v_new), bits(case["k_rep"]), bits(case["v"]), reps, lens)
+    assert np.array_equal(bits(cache)[:, :k], k_ref) and np.array_equal(bits(v), v_ref)
+    assert np.array_equal(bits(cache)[:, k:], after[:, k:])          # dead planes are not touched by the append
+    out2 = chai.chai_decode_attention_ragged(d["q"], cache, v, d["membership"], d["reps"], seq, case["scale"],
+                                             T_max=T_cap)
+    kf, vf = case["k_rep"].clone(), case["v"].clone()
+    for b, n in enumerate(lens):
+        vf[b, :, n] = v_new[b]
+        for c in range(k):
+            kf[b, c, n] = k_new[b, int(reps[b, c])]
+    ref2 = orc.decode_attention_ragged(case["q"], kf, vf, case["membership"], reps, lens_ref, case["scale"])
+    assert_parity(out2.float().cpu().numpy(), ref2, case["dtype"], "decode after append")
+    assert before.shape == after.shape
+
+
+def test_append_full_cache_is_reported_and_skipped():
+    B, H, k, T_cap, D = 2, 4, 2, 8, 128
+    reps = torch.tensor([[0, 1], [0, 2]], dtype=torch.int32, device=DEV)
+    k_rep = torch.zeros(B, k, T_cap, D, dtype=torch.bfloat16, device=DEV)
+    v = torch.zeros(B, H, T_cap, D, dtype=torch.bfloat16, device=DEV)
+    new = torch.ones(B, H, D, dtype=torch.bfloat16, device=DEV)
+    seq = torch.tensor([T_cap, 3], dtype=torch.int32, device=DEV)
+    ws = chai.new_workspace(256, DEV)
+    chai.chai_append_kv(new, new, k_rep, v, reps, seq, advance=True, workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_ERR_CACHE_FULL
+    assert seq.cpu().tolist() == [T_cap, 4]
+    assert not k_rep[0].any() and not v[0].any()
+    assert v[1, :, 3].eq(1).all() and k_rep[1, :, 3].eq(1).all() and v[1].sum() == H * D
+
+
+def test_inplace_compaction_refuses_unordered_reps():
+    B, H, k, T, D = 2, 6, 3, 16, 128
+    g = torch.Generator().manual_seed(0)
+    cache = torch.randn(B, H, T, D, generator=g).to(torch.bfloat16).to(DEV)
+    before = bits(cache)
+    reps = torch.tensor([[0, 2, 4], [3, 1, 5]], dtype=torch.int32, device=DEV)   # request 1 is not ascending
+    ws = chai.new_workspace(256, DEV)
+    chai.chai_compact_k_cache_inplace(cache, reps, workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_ERR_BAD_MEMBERSHIP
+    after = bits(cache)
+    assert np.array_equal(after[1], before[1])                         # left untouched
+    assert np.array_equal(after[0, 1], before[0, 2]) and np.array_equal(after[0, 2], before[0, 4])
+
+
+@pytest.mark.parametrize("fn_name", ["chai_prefill_attention_from", "chai_prefill_attention_simt_from"])
+@pytest.mark.parametrize("T,q_start", [(300, 5), (300, 128), (300, 131), (64, 5), (129, 128), (640, 257)])
+def test_prefill_from_q_start(fn_name, T, q_start):
+    """Rows from q_start on equal the full clustered prefill; earlier rows of the output are not written."""
+    B, H, k, D = 2, 6, 2, 128
+    r = synth.batch_partitions(B, H, k, "uneven", T, 79, q_start)
+    g = torch.Generator().manual_seed(T + q_start)
+    q = (torch.randn(B, H, T, D, generator=g) * 2.0).to(torch.bfloat16)
+    kr = (torch.randn(B, k, T, D, generator=g) * 0.5).to(torch.bfloat16)
+    v = (torch.randn(B, H, T, D, generator=g) * 0.5).to(torch.bfloat16)
+    mem, reps = torch.as_tensor(r[0]), torch.as_tensor(r[1])
+    scale = 1.0 / np.sqrt(D)
+    out = torch.full((B, H, T, D), 7.0, dtype=torch.bfloat16, device=DEV)
+    getattr(chai, fn_name)(q.to(DEV), kr.to(DEV), v.to(DEV), mem.to(DEV), reps.to(DEV), scale, q_start, True, out=out)
+    got = out.float().cpu().numpy()
+    ref = orc.cha_attention(q, kr, v, mem, reps, scale, True)
+    assert (got[:, :, :q_start] == 7.0).all()
+    assert_parity(got[:, :, q_start:], ref[:, :, q_start:], "bf16", f"{fn_name} T {T} q_start {q_start}")

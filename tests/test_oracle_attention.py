@@ -263,3 +263,80 @@ def test_attention_on_compacted_cache_equals_direct():
     a = orc.cha_attention(q, krep, v, mem, reps, 1.0, True)
     b = orc.cha_attention(q, direct, v, mem, reps, 1.0, True)
     assert np.array_equal(a, b)
+
+
+# ---- serving-shaped helpers: pinned against brute force written out independently ----------------------
+
+def _brute_decode(q, k_rep, v, membership, reps, n, scale):
+    """Direct loops over one request: softmax over the first n positions, then the weighted sum of V."""
+    H, D = q.shape
+    out = np.zeros((H, D))
+    for h in range(H):
+        c = int(membership[h])
+        r = int(reps[c])
+        s = np.array([scale * float(np.dot(q[r], k_rep[c, t])) for t in range(n)])
+        p = np.exp(s - s.max())
+        p /= p.sum()
+        for t in range(n):
+            out[h] += p[t] * v[h, t]
+    return out
+
+
+def test_ragged_decode_matches_brute_force_per_request():
+    rng = np.random.default_rng(12)
+    B, H, k, T_cap, D = 3, 6, 3, 40, 16
+    membership = np.array([[0, 1, 0, 2, 1, 2], [0, 0, 1, 1, 2, 2], [0, 1, 2, 0, 1, 2]], dtype=np.int32)
+    reps = np.array([[0, 1, 3], [0, 2, 4], [0, 1, 2]], dtype=np.int32)
+    q = rng.normal(size=(B, H, D))
+    k_rep = rng.normal(size=(B, k, T_cap, D))
+    v = rng.normal(size=(B, H, T_cap, D))
+    lens = np.array([40, 7, 0])
+    scale = 0.31
+    got = orc.decode_attention_ragged(q, k_rep, v, membership, reps, lens, scale)
+    for b in range(B):
+        want = _brute_decode(q[b], k_rep[b], v[b], membership[b], reps[b], int(lens[b]), scale) if lens[b] else 0.0
+        assert np.allclose(got[b], want, rtol=1e-12, atol=1e-13)
+    # rows beyond a request's length must not matter
+    k2, v2 = k_rep.copy(), v.copy()
+    k2[1, :, 7:] = 1e6
+    v2[1, :, 7:] = -1e6
+    assert np.array_equal(orc.decode_attention_ragged(q, k2, v2, membership, reps, lens, scale), got)
+
+
+def test_append_then_decode_equals_decode_on_longer_cache():
+    """Appending a token and decoding over n + 1 positions = decoding on a cache that already held the token."""
+    rng = np.random.default_rng(13)
+    B, H, k, T_cap, D = 2, 4, 2, 12, 8
+    membership = np.array([[0, 1, 0, 1], [0, 0, 1, 1]], dtype=np.int32)
+    reps = np.array([[0, 1], [0, 2]], dtype=np.int32)
+    k_full = rng.normal(size=(B, H, T_cap, D))
+    v = rng.normal(size=(B, H, T_cap, D))
+    lens = np.array([5, 9])
+    k_rep, _ = orc.compact_k_cache(k_full, reps)
+    k_new, v_new = rng.normal(size=(B, H, D)), rng.normal(size=(B, H, D))
+    k_rep2, v2, lens2 = orc.append_kv(k_new, v_new, k_rep, v, reps, lens)
+    assert lens2.tolist() == [6, 10]
+    for b in range(B):
+        p = int(lens[b])
+        assert np.array_equal(v2[b, :, p], v_new[b])
+        for c in range(k):
+            assert np.array_equal(k_rep2[b, c, p], k_new[b, reps[b, c]])
+        # nothing else moved
+        mask = np.ones(T_cap, bool)
+        mask[p] = False
+        assert np.array_equal(v2[b][:, mask], v[b][:, mask]) and np.array_equal(k_rep2[b][:, mask], k_rep[b][:, mask])
+    # a full cache skips the request
+    k3, v3, lens3 = orc.append_kv(k_new, v_new, k_rep, v, reps, np.array([T_cap, 2]))
+    assert lens3.tolist() == [T_cap, 3] and np.array_equal(v3[0], v[0]) and np.array_equal(k3[0], k_rep[0])
+
+
+def test_inplace_compaction_definition():
+    rng = np.random.default_rng(14)
+    k_full = rng.integers(0, 2 ** 16, size=(2, 5, 9, 4)).astype(np.uint16)
+    reps = np.array([[0, 2, 4], [0, 1, -1]], dtype=np.int32)
+    got = orc.compact_k_cache_inplace(k_full, reps, 6)
+    assert got.shape == (2, 3, 6, 4)
+    for b in range(2):
+        for c in range(3):
+            if reps[b, c] >= 0:
+                assert np.array_equal(got[b, c], k_full[b, reps[b, c], :6])
