@@ -35,7 +35,7 @@ namespace pd {
 
 constexpr int CONSUMER_WARPS = 8;
 constexpr int THREADS = CONSUMER_WARPS * 32 + 32;
-constexpr int STAGES = 5;                  // 160 KB of cache rows in flight per SM
+constexpr int STAGES = 6;                  // 192 KB of cache rows in flight per SM
 constexpr int MAX_IV = 4;                  // tiles per value item
 constexpr int ITEM_SLOTS = 8;              // value items whose tile partials may be open in one CTA
 constexpr int TABLE_CAP = 2048;            // heads whose cluster id is cached in shared memory
