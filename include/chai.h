@@ -90,6 +90,18 @@ int chai_cluster_heads(const float* features, int B, int H, int F, int k, int ma
                        int32_t* membership, int32_t* reps, int32_t* k_eff, double* inertia, void* stream);
 
 /*
+ * Alternative choice of representatives: for every cluster the member whose feature vector is nearest
+ * (squared Euclidean distance, fp64) to the mean of the cluster's members; ties go to the lowest head index
+ * (the paper does not say which member stands for a cluster; chai_cluster_heads takes the lowest member).
+ *   features [B,H,F] fp32, membership [B,H] int32 (as written by chai_cluster_heads) -> reps [B,k] int32,
+ *   -1 for a cluster without members.  Cluster numbering is not changed, so reps[b][c] >= c still holds, but
+ *   the representatives are no longer ascending: chai_compact_k_cache_inplace refuses such reps (use the
+ *   out-of-place compaction).  Same size limits as chai_cluster_heads.
+ */
+int chai_select_representatives(const float* features, const int32_t* membership, int B, int H, int F, int k,
+                                int32_t* reps, void* stream);
+
+/*
  * K-cache compaction (Section 3.5: once membership is fixed the keys of pruned
  * heads are removed; Section 4.3: all values are kept).
  *   k_full [B,H,T_cap,D] -> k_rep [B,k,T_cap,D]:  k_rep[b][c][0..T) = k_full[b][reps[b][c]][0..T)
@@ -229,6 +241,36 @@ int chai_prefill_attention_simt_from(const void* q, const void* k_rep, const voi
                                      const int32_t* reps, void* out, int B, int H, int k, int T, int q_start, int D,
                                      float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
                                      void* stream);
+
+/*
+ * CHAI-QKV (Table 4 of the paper: besides Q and K, the V of non-representative heads is dropped as well, so a
+ * member head's output equals its representative's).  Caches hold representatives only:
+ *   k_rep, v_rep [B,k,T_cap,D] (decode) / [B,k,T,D] (prefill);  q and out keep all H heads:
+ *   out[b][h] = attention(q[b][reps[b][c]], k_rep[b][c], v_rep[b][c]),  c = membership[b][h].
+ * Decode: seq_lens may be NULL (every request has T positions) or a device array [B] as in
+ * chai_decode_attention_ragged.  Prefill: rows [q_start, T) are computed and written.  The workspace
+ * (chai_*_qkv_workspace_bytes) also holds the gathered query rows and the k per-cluster outputs.
+ * v_rep is produced from a full value cache by chai_compact_k_cache (the same gather).
+ * Heads whose membership cannot be resolved get zero rows and CHAI_ERR_BAD_MEMBERSHIP in the status word.
+ */
+size_t chai_decode_qkv_workspace_bytes(int B, int H, int k, int T, int D, int dtype);
+int chai_decode_attention_qkv(const void* q, const void* k_rep, const void* v_rep, const int32_t* membership,
+                              const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T,
+                              int T_cap, int D, float scale, int dtype, void* workspace, size_t workspace_bytes,
+                              void* stream);
+size_t chai_prefill_qkv_workspace_bytes(int B, int H, int k, int T, int D, int dtype);
+int chai_prefill_attention_qkv(const void* q, const void* k_rep, const void* v_rep, const int32_t* membership,
+                               const int32_t* reps, void* out, int B, int H, int k, int T, int q_start, int D,
+                               float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
+                               void* stream);
+
+/*
+ * CHAI-static (Section 3.5: a membership found offline is used for every request instead of clustering each
+ * request's prefix): expands one membership [H] / representatives [k] into the per-request arrays [B,H] /
+ * [B,k] that every other entry point takes.
+ */
+int chai_broadcast_membership(const int32_t* membership_static, const int32_t* reps_static, int32_t* membership,
+                              int32_t* reps, int B, int H, int k, void* stream);
 
 /* Blocking read of the status word a decode/prefill call left in `workspace`
  * (synchronises `stream`).  *status_out receives a chai_status_t. */

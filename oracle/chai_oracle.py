@@ -205,3 +205,45 @@ def compact_k_cache_inplace(k_full: np.ndarray, reps, T: int) -> np.ndarray:
     not compared (the in-place call leaves them as they were)."""
     k_rep, _ = compact_k_cache(k_full[:, :, :T], reps)
     return k_rep
+
+
+# ---- variants the paper evaluates (Table 4, Section 3.5) -----------------------------------------------
+
+def cha_attention_qkv(q, k_rep, v_rep, membership, reps, scale: float, causal: bool) -> np.ndarray:
+    """CHAI-QKV: the values of non-representative heads are dropped too, i.e. every member head uses its
+    representative's values.  Written as the main definition with V expanded accordingly:
+    v[b][h] = v_rep[b][membership[b][h]]."""
+    v_rep = _f64(v_rep)
+    membership = _i32(membership)
+    B, H = membership.shape
+    v = np.stack([v_rep[b, membership[b]] for b in range(B)])
+    return cha_attention(q, k_rep, v, membership, reps, scale, causal)
+
+
+def closest_representatives(features, membership, k: int) -> np.ndarray:
+    """Alternative to 'lowest member': per cluster the member nearest (squared Euclidean, fp64) to the mean of
+    the cluster's members; ties to the lowest head index; -1 for an empty cluster.  features [B,H,F],
+    membership [B,H] -> reps [B,k].  Sums run in ascending head / feature order, one rounding per operation."""
+    x = _f64(features)
+    membership = _i32(membership)
+    B, H, F = x.shape
+    reps = np.full((B, k), -1, dtype=np.int32)
+    for b in range(B):
+        for c in range(k):
+            members = [h for h in range(H) if membership[b, h] == c]
+            if not members:
+                continue
+            mean = np.zeros(F)
+            for h in members:
+                mean = mean + x[b, h]
+            mean = mean / float(len(members))
+            best, best_d = -1, 0.0
+            for h in members:
+                d = 0.0
+                for f in range(F):
+                    t = x[b, h, f] - mean[f]
+                    d = d + t * t
+                if best < 0 or d < best_d:
+                    best, best_d = h, d
+            reps[b, c] = best
+    return reps

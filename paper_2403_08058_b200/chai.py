@@ -27,6 +27,8 @@ EXPORTS = [
     "chai_status_string", "chai_last_error", "chai_version", "chai_decode_attention_static",
     "chai_decode_attention_ragged", "chai_append_kv", "chai_compact_k_cache_inplace",
     "chai_prefill_attention_from", "chai_prefill_attention_simt_from",
+    "chai_decode_qkv_workspace_bytes", "chai_decode_attention_qkv", "chai_prefill_qkv_workspace_bytes",
+    "chai_prefill_attention_qkv", "chai_broadcast_membership", "chai_select_representatives",
 ]
 DECODE_STATIC_SCRATCH_BYTES = 8 << 20   # CHAI_DECODE_STATIC_SCRATCH_BYTES
 
@@ -57,7 +59,12 @@ def load() -> ctypes.CDLL:
                                                vp, sz, vp]
     for name in ("chai_prefill_attention", "chai_prefill_attention_simt"):
         getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
-    for name in ("chai_decode_workspace_bytes", "chai_prefill_workspace_bytes"):
+    lib.chai_decode_attention_qkv.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp, sz, vp]
+    lib.chai_prefill_attention_qkv.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
+    lib.chai_broadcast_membership.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp]
+    lib.chai_select_representatives.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
+    for name in ("chai_decode_workspace_bytes", "chai_prefill_workspace_bytes", "chai_decode_qkv_workspace_bytes",
+                 "chai_prefill_qkv_workspace_bytes"):
         getattr(lib, name).argtypes = [ci, ci, ci, ci, ci, ci]
         getattr(lib, name).restype = sz
     lib.chai_decode_attention_ragged.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, sz, cf, ci, vp, sz, vp]
@@ -146,6 +153,15 @@ def chai_cluster_heads(features, k: int, max_iter: int = 20, seed: int = 0, want
     _check(load().chai_cluster_heads(_ptr(features), B, H, F, k, max_iter, seed, _ptr(membership), _ptr(reps),
                                      _ptr(k_eff), _ptr(inertia), _stream()))
     return membership, reps, k_eff, inertia
+
+
+def chai_select_representatives(features, membership, k: int):
+    """features [B,H,F] fp32, membership [B,H] -> reps [B,k]: each cluster's member nearest to the cluster mean."""
+    _dev(features, membership)
+    B, H, F = features.shape
+    reps = torch.empty((B, k), device=features.device, dtype=torch.int32)
+    _check(load().chai_select_representatives(_ptr(features), _ptr(membership), B, H, F, k, _ptr(reps), _stream()))
+    return reps
 
 
 def chai_compact_k_cache(k_full, reps, T: int | None = None, k_rep=None):
@@ -308,6 +324,53 @@ def chai_prefill_attention(q, k_rep, v, membership, reps, scale: float, causal: 
 def chai_prefill_attention_simt(q, k_rep, v, membership, reps, scale: float, causal: bool = True, out=None,
                                 workspace=None):
     return _prefill("chai_prefill_attention_simt", q, k_rep, v, membership, reps, scale, causal, out, workspace)
+
+
+def chai_decode_attention_qkv(q, k_rep, v_rep, membership, reps, scale: float, T: int | None = None, seq_lens=None,
+                              out=None, workspace=None):
+    """CHAI-QKV decode: q [B,H,D], k_rep / v_rep [B,k,T_cap,D] -> out [B,H,D] (a member's row = its cluster's)."""
+    _dev(q, k_rep, v_rep, membership, reps, seq_lens, out, workspace)
+    B, H, D = q.shape
+    k, T_cap = k_rep.shape[1], k_rep.shape[2]
+    T = T_cap if T is None else T
+    dt = _dt(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(int(load().chai_decode_qkv_workspace_bytes(B, H, k, T, D, dt)), q.device)
+    _check(load().chai_decode_attention_qkv(_ptr(q), _ptr(k_rep), _ptr(v_rep), _ptr(membership), _ptr(reps),
+                                            _ptr(seq_lens), _ptr(out), B, H, k, T, T_cap, D, scale, dt, _ptr(workspace),
+                                            workspace.numel(), _stream()))
+    return out
+
+
+def chai_prefill_attention_qkv(q, k_rep, v_rep, membership, reps, scale: float, causal: bool = True, q_start: int = 0,
+                               out=None, workspace=None):
+    """CHAI-QKV prefill: q [B,H,T,D], k_rep / v_rep [B,k,T,D] -> out [B,H,T,D]."""
+    _dev(q, k_rep, v_rep, membership, reps, out, workspace)
+    B, H, T, D = q.shape
+    k = k_rep.shape[1]
+    dt = _dt(q)
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(int(load().chai_prefill_qkv_workspace_bytes(B, H, k, T, D, dt)), q.device)
+    _check(load().chai_prefill_attention_qkv(_ptr(q), _ptr(k_rep), _ptr(v_rep), _ptr(membership), _ptr(reps), _ptr(out),
+                                             B, H, k, T, int(q_start), D, scale, int(bool(causal)), dt, _ptr(workspace),
+                                             workspace.numel(), _stream()))
+    return out
+
+
+def chai_broadcast_membership(membership_static, reps_static, B: int):
+    """One membership [H] / reps [k] for every request -> ([B,H], [B,k]) int32 (CHAI-static)."""
+    _dev(membership_static, reps_static)
+    H, k = membership_static.numel(), reps_static.numel()
+    dev = membership_static.device
+    membership = torch.empty((B, H), device=dev, dtype=torch.int32)
+    reps = torch.empty((B, k), device=dev, dtype=torch.int32)
+    _check(load().chai_broadcast_membership(_ptr(membership_static), _ptr(reps_static), _ptr(membership), _ptr(reps), B,
+                                            H, k, _stream()))
+    return membership, reps
 
 
 def chai_device_status(workspace) -> int:

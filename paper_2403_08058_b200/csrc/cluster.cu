@@ -195,6 +195,52 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
     }
 }
 
+// Representative of each cluster = the member nearest to the cluster's mean (an alternative to "lowest
+// member"; ties go to the lowest head index).  One CTA per request; fp64 with the same explicitly rounded
+// operations and summation orders as the clustering itself, so the choice is reproducible bit for bit.
+// Shared memory: X [H,F], C [k,F], dist [H] doubles; a [H], count [k] ints.
+__global__ void __launch_bounds__(256)
+select_reps_kernel(const float* __restrict__ features, const int32_t* __restrict__ membership, int H, int F, int k,
+                   int32_t* __restrict__ reps) {
+    extern __shared__ double sh_sel[];
+    double* X = sh_sel;
+    double* C = X + (size_t)H * F;
+    double* dist = C + (size_t)k * F;
+    int* a = reinterpret_cast<int*>(dist + H);
+    int* count = a + H;
+    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+    for (int i = tid; i < H * F; i += nt) X[i] = (double)features[(size_t)b * H * F + i];
+    for (int h = tid; h < H; h += nt) {
+        const int c = membership[(size_t)b * H + h];
+        a[h] = (c >= 0 && c < k) ? c : -1;  // heads with an invalid cluster id belong nowhere
+    }
+    __syncthreads();
+    for (int c = tid; c < k; c += nt) {
+        int n = 0;
+        for (int h = 0; h < H; ++h) n += (a[h] == c);
+        count[c] = n;
+    }
+    __syncthreads();
+    for (int p = tid; p < k * F; p += nt) {
+        const int c = p / F, f = p % F;
+        if (count[c] == 0) continue;
+        double s = 0.0;
+        for (int h = 0; h < H; ++h)
+            if (a[h] == c) s = __dadd_rn(s, X[(size_t)h * F + f]);
+        C[(size_t)c * F + f] = __ddiv_rn(s, (double)count[c]);
+    }
+    __syncthreads();
+    for (int h = tid; h < H; h += nt)
+        if (a[h] >= 0) dist[h] = sqdist(X + (size_t)h * F, C + (size_t)a[h] * F, F);
+    __syncthreads();
+    for (int c = tid; c < k; c += nt) {
+        int best = -1;
+        for (int h = 0; h < H; ++h)
+            if (a[h] == c && (best < 0 || dist[h] < dist[best])) best = h;
+        reps[(size_t)b * k + c] = best;  // -1 for an empty cluster
+    }
+}
+
 static size_t kmeans_smem_bytes(int H, int F, int k) {
     return sizeof(double) * ((size_t)H * F + (size_t)k * F + (size_t)H * k) + sizeof(int) * (2 * (size_t)H + 2 * (size_t)k);
 }
@@ -246,6 +292,23 @@ int chai_cluster_heads(const float* features, int B, int H, int F, int k, int ma
     kmeans_kernel<<<B, 256, smem, s>>>(features, H, F, k, max_iter, (unsigned long long)seed, membership, reps,
                                        k_eff, inertia);
     CHAI_LAUNCH_CHECK("kmeans_kernel launch");
+    return CHAI_OK;
+}
+
+int chai_select_representatives(const float* features, const int32_t* membership, int B, int H, int F, int k,
+                                int32_t* reps, void* stream) {
+    using namespace chai;
+    CHAI_REQUIRE(features && membership && reps, CHAI_ERR_INVALID_ARG, "chai_select_representatives: null pointer");
+    CHAI_REQUIRE(B > 0 && H > 0 && F > 0 && k >= 1 && k <= H, CHAI_ERR_INVALID_ARG,
+                 "chai_select_representatives: need B, H, F > 0 and 1 <= k <= H");
+    const size_t smem = sizeof(double) * ((size_t)H * F + (size_t)k * F + (size_t)H) + sizeof(int) * ((size_t)H + k);
+    CHAI_REQUIRE(H <= 1024 && smem <= 200 * 1024, CHAI_ERR_UNSUPPORTED,
+                 "chai_select_representatives: problem needs %zu bytes of shared memory (limit 204800)", smem);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaFuncSetAttribute(select_reps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e, "select_reps_kernel shared-memory opt-in");
+    select_reps_kernel<<<B, 256, smem, s>>>(features, membership, H, F, k, reps);
+    CHAI_LAUNCH_CHECK("select_reps_kernel launch");
     return CHAI_OK;
 }
 

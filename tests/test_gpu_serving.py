@@ -157,3 +157,91 @@ def test_prefill_from_q_start(fn_name, T, q_start):
     ref = orc.cha_attention(q, kr, v, mem, reps, scale, True)
     assert (got[:, :, :q_start] == 7.0).all()
     assert_parity(got[:, :, q_start:], ref[:, :, q_start:], "bf16", f"{fn_name} T {T} q_start {q_start}")
+
+
+# ---- variants: CHAI-QKV and CHAI-static ---------------------------------------------------------------
+
+@pytest.mark.parametrize("cfg,ragged", [(1, False), (2, False), (2, True)])
+def test_decode_qkv(cfg, ragged):
+    B, H, k, T_cap = 4, 12, 3, 300
+    case = ragged_case(cfg, 31, B, H, k, T_cap)
+    reps = case["reps"]
+    v_rep = torch.stack([case["v"][b, reps[b].long()] for b in range(B)]).contiguous()
+    lens = [300, 1, 129, 77] if ragged else [T_cap] * B
+    seq = torch.tensor(lens, dtype=torch.int32, device=DEV) if ragged else None
+    out = chai.chai_decode_attention_qkv(case["q"].to(DEV), case["k_rep"].to(DEV), v_rep.to(DEV),
+                                         case["membership"].to(DEV), reps.to(DEV), case["scale"], seq_lens=seq)
+    got = out.float().cpu().numpy()
+    ref = np.zeros_like(got, dtype=np.float64)
+    for b, n in enumerate(lens):
+        ref[b] = orc.cha_attention_qkv(case["q"][b:b + 1], case["k_rep"][b:b + 1, :, :n], v_rep[b:b + 1, :, :n],
+                                       case["membership"][b:b + 1], reps[b:b + 1], case["scale"], False)[0]
+    assert_parity(got, ref, case["dtype"], f"QKV decode cfg {cfg} ragged {ragged}")
+    mem = case["membership"]
+    for b in range(B):
+        for h in range(H):
+            assert np.array_equal(got[b, h], got[b, int(reps[b, int(mem[b, h])])])   # a member's row IS its representative's
+
+
+@pytest.mark.parametrize("T,q_start,dtype", [(300, 0, "bf16"), (300, 5, "bf16"), (200, 0, "f32")])
+def test_prefill_qkv(T, q_start, dtype):
+    B, H, k, D = 2, 8, 3, 128
+    r = synth.batch_partitions(B, H, k, "uneven", T, 80, q_start)
+    g = torch.Generator().manual_seed(T)
+    td = synth.TORCH_DTYPE[dtype]
+    q = (torch.randn(B, H, T, D, generator=g) * 2.0).to(td)
+    kr = (torch.randn(B, k, T, D, generator=g) * 0.5).to(td)
+    vr = (torch.randn(B, k, T, D, generator=g) * 0.5).to(td)
+    mem, reps = torch.as_tensor(r[0]), torch.as_tensor(r[1])
+    scale = 1.0 / np.sqrt(D)
+    out = torch.full((B, H, T, D), 7.0, dtype=td, device=DEV)
+    chai.chai_prefill_attention_qkv(q.to(DEV), kr.to(DEV), vr.to(DEV), mem.to(DEV), reps.to(DEV), scale, True, q_start,
+                                    out=out)
+    got = out.float().cpu().numpy()
+    ref = orc.cha_attention_qkv(q, kr, vr, mem, reps, scale, True)
+    assert (got[:, :, :q_start] == 7.0).all()
+    assert_parity(got[:, :, q_start:], ref[:, :, q_start:], dtype, f"QKV prefill T {T} q_start {q_start} {dtype}")
+
+
+def test_qkv_bad_membership_is_reported():
+    B, H, k, T = 1, 6, 2, 64
+    case = ragged_case(2, 5, B, H, k, T)
+    v_rep = torch.stack([case["v"][b, case["reps"][b].long()] for b in range(B)]).contiguous()
+    mem = case["membership"].clone()
+    hbad = [h for h in range(H) if h not in case["reps"][0].tolist()][0]
+    mem[0, hbad] = 9
+    ws = chai.new_workspace(int(chai.load().chai_decode_qkv_workspace_bytes(B, H, k, T, 128, chai.CHAI_BF16)), DEV)
+    out = chai.chai_decode_attention_qkv(case["q"].to(DEV), case["k_rep"].to(DEV), v_rep.to(DEV), mem.to(DEV),
+                                         case["reps"].to(DEV), case["scale"], workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_ERR_BAD_MEMBERSHIP
+    assert not out[0, hbad].float().abs().sum().item()
+
+
+def test_static_membership_broadcast_equals_per_request_arrays():
+    B, H, k, T = 3, 8, 4, 200
+    case = ragged_case(2, 8, B, H, k, T)
+    m0, r0 = case["membership"][0].contiguous(), case["reps"][0].contiguous()
+    mem, reps = chai.chai_broadcast_membership(m0.to(DEV), r0.to(DEV), B)
+    assert mem.cpu().tolist() == [m0.tolist()] * B and reps.cpu().tolist() == [r0.tolist()] * B
+    k_rep = torch.stack([case["k_full"][b, r0.long()] for b in range(B)]).contiguous()
+    out = chai.chai_decode_attention(case["q"].to(DEV), k_rep.to(DEV), case["v"].to(DEV), mem, reps, case["scale"])
+    ref = orc.cha_attention(case["q"], k_rep, case["v"], mem.cpu(), reps.cpu(), case["scale"], False)
+    assert_parity(out.float().cpu().numpy(), ref, "bf16", "static membership")
+
+
+def test_select_representatives_matches_oracle():
+    B, H, F, k = 3, 40, 25, 6
+    feats, planted, _ = synth.blob_features(B, H, F, k, seed=2)
+    feats = torch.as_tensor(feats, dtype=torch.float32)
+    mem, _, _, _ = chai.chai_cluster_heads(feats.to(DEV), k, 20, 1)
+    got = chai.chai_select_representatives(feats.to(DEV), mem, k).cpu().numpy()
+    want = orc.closest_representatives(feats.numpy(), mem.cpu().numpy(), k)
+    assert np.array_equal(got, want)
+    m = mem.cpu().numpy()
+    for b in range(B):
+        for c in range(k):
+            assert got[b, c] >= c and m[b, got[b, c]] == c           # a member of its own cluster
+    # exact ties (duplicated heads) and an empty cluster
+    f2 = torch.tensor([[[0.0], [1.0], [10.0], [4.0], [3.0]]])
+    m2 = torch.tensor([[0, 1, 0, 0, 1]], dtype=torch.int32)
+    assert chai.chai_select_representatives(f2.to(DEV), m2.to(DEV), 3).cpu().tolist() == [[3, 1, -1]]

@@ -340,3 +340,26 @@ def test_inplace_compaction_definition():
         for c in range(3):
             if reps[b, c] >= 0:
                 assert np.array_equal(got[b, c], k_full[b, reps[b, c], :6])
+
+
+def test_qkv_variant_member_rows_equal_the_representatives_plain_attention():
+    """In CHAI-QKV a member's output is the representative's own single-head attention output."""
+    rng = np.random.default_rng(15)
+    B, H, k, T, D = 2, 6, 3, 9, 8
+    membership = np.array([[0, 1, 0, 2, 1, 2], [0, 0, 1, 1, 2, 2]], dtype=np.int32)
+    reps = np.array([[0, 1, 3], [0, 2, 4]], dtype=np.int32)
+    q = rng.normal(size=(B, H, T, D))
+    k_rep = rng.normal(size=(B, k, T, D))
+    v_rep = rng.normal(size=(B, k, T, D))
+    scale = 0.4
+    got = orc.cha_attention_qkv(q, k_rep, v_rep, membership, reps, scale, True)
+    for b in range(B):
+        for h in range(H):
+            c = membership[b, h]
+            r = reps[b, c]
+            s = scale * q[b, r] @ k_rep[b, c].T
+            s = np.where(np.tril(np.ones((T, T), bool)), s, -np.inf)
+            p = np.exp(s - s.max(axis=1, keepdims=True))
+            p /= p.sum(axis=1, keepdims=True)
+            assert np.allclose(got[b, h], p @ v_rep[b, c], rtol=1e-12, atol=1e-13)
+            assert np.array_equal(got[b, h], got[b, r])

@@ -181,3 +181,29 @@ def test_flow_features_then_kmeans_recovers_planted_prompt_clusters():
         f32 = f.astype(np.float32)
         r = orc.kmeans(f32, case["k"], 20, 0)
         assert np.array_equal(r["membership"], case["planted"]), seed
+
+
+def test_closest_representatives_hand_cases():
+    """Medoid-like choice checked on points whose answer is visible by eye."""
+    # cluster 0 = heads {0, 2, 3} at x = 0, 10, 4 (mean 14/3 = 4.67 -> head 3); cluster 1 = heads {1, 4} at 1 and 3:
+    # both 1 away from the mean 2 -> tie -> lowest index (head 1)
+    feats = np.array([[[0.0], [1.0], [10.0], [4.0], [3.0]]])
+    mem = np.array([[0, 1, 0, 0, 1]], dtype=np.int32)
+    assert orc.closest_representatives(feats, mem, 3).tolist() == [[3, 1, -1]]
+    # a singleton is its own representative; identical members -> lowest index
+    feats = np.array([[[2.0, 2.0], [5.0, 5.0], [5.0, 5.0], [9.0, 1.0]]])
+    mem = np.array([[0, 1, 1, 2]], dtype=np.int32)
+    assert orc.closest_representatives(feats, mem, 3).tolist() == [[0, 1, 3]]
+    # brute force against numpy on random blobs
+    rng = np.random.default_rng(3)
+    x = rng.normal(size=(2, 12, 7))
+    mem = rng.integers(0, 4, size=(2, 12)).astype(np.int32)
+    got = orc.closest_representatives(x, mem, 4)
+    for b in range(2):
+        for c in range(4):
+            idx = np.where(mem[b] == c)[0]
+            if len(idx) == 0:
+                assert got[b, c] == -1
+                continue
+            d = ((x[b, idx] - x[b, idx].mean(axis=0)) ** 2).sum(axis=1)
+            assert got[b, c] == idx[np.argmin(d)]
