@@ -90,6 +90,18 @@ int chai_cluster_heads(const float* features, int B, int H, int F, int k, int ma
                        int32_t* membership, int32_t* reps, int32_t* k_eff, double* inertia, void* stream);
 
 /*
+ * Offline choice of the number of clusters (Section 3.2, Fig. 8: the clustering error is plotted against the
+ * number of clusters and the count is taken where the curve flattens; the paper reads the plot by eye).
+ * Runs chai_cluster_heads' k-means for every k = 1..k_max on every request at once (one CTA per (request, k))
+ * and returns the error curve; optionally picks the knee: with k scaled to x in [0,1] and the error to y in
+ * [0,1], the k farthest below the line from (0,1) to (1,0), ties to the smaller k (a flat curve gives 1).
+ *   features [B,H,F] fp32 -> inertia_curve [B,k_max] fp64 (entry k-1 = inertia with k clusters),
+ *   k_pick [B] int32 or NULL.  Same seed / max_iter meaning and size limits as chai_cluster_heads.
+ */
+int chai_cluster_sweep(const float* features, int B, int H, int F, int k_max, int max_iter, uint64_t seed,
+                       double* inertia_curve, int32_t* k_pick, void* stream);
+
+/*
  * Alternative choice of representatives: for every cluster the member whose feature vector is nearest
  * (squared Euclidean distance, fp64) to the mean of the cluster's members; ties go to the lowest head index
  * (the paper does not say which member stands for a cluster; chai_cluster_heads takes the lowest member).

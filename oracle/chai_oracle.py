@@ -247,3 +247,33 @@ def closest_representatives(features, membership, k: int) -> np.ndarray:
                     best, best_d = h, d
             reps[b, c] = best
     return reps
+
+
+def knee_of_curve(e) -> int:
+    """Knee of a decreasing error curve e[0..n-1] (entry i = error with i + 1 clusters): with the cluster count
+    scaled to x in [0,1] and the error to y in [0,1], the count farthest below the line from (0,1) to (1,0),
+    i.e. the maximiser of 1 - x - y; ties to the smaller count; a flat curve gives 1."""
+    e = np.asarray(e, dtype=np.float64)
+    n = len(e)
+    lo, hi = float(e.min()), float(e.max())
+    if n < 2 or not hi > lo:
+        return 1
+    best, best_v = 1, None
+    for i in range(n):
+        x = float(i) / float(n - 1)
+        y = (float(e[i]) - lo) / (hi - lo)
+        v = (1.0 - x) - y
+        if best_v is None or v > best_v:
+            best, best_v = i + 1, v
+    return best
+
+
+def cluster_sweep(features, k_max: int, max_iter: int = 20, seed: int = 0):
+    """Clustering error for every k = 1..k_max (Section 3.2) and the knee of each curve.
+    features [B,H,F] -> (curve [B,k_max] float64, knee [B] int32)."""
+    x = _f64(features)
+    B = x.shape[0]
+    curve = np.empty((B, k_max), dtype=np.float64)
+    for k in range(1, k_max + 1):
+        curve[:, k - 1] = kmeans(x, k, max_iter, seed)["inertia"]
+    return curve, np.array([knee_of_curve(curve[b]) for b in range(B)], dtype=np.int32)

@@ -28,7 +28,7 @@ EXPORTS = [
     "chai_decode_attention_ragged", "chai_append_kv", "chai_compact_k_cache_inplace",
     "chai_prefill_attention_from", "chai_prefill_attention_simt_from",
     "chai_decode_qkv_workspace_bytes", "chai_decode_attention_qkv", "chai_prefill_qkv_workspace_bytes",
-    "chai_prefill_attention_qkv", "chai_broadcast_membership", "chai_select_representatives",
+    "chai_prefill_attention_qkv", "chai_broadcast_membership", "chai_select_representatives", "chai_cluster_sweep",
 ]
 DECODE_STATIC_SCRATCH_BYTES = 8 << 20   # CHAI_DECODE_STATIC_SCRATCH_BYTES
 
@@ -63,6 +63,7 @@ def load() -> ctypes.CDLL:
     lib.chai_prefill_attention_qkv.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
     lib.chai_broadcast_membership.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp]
     lib.chai_select_representatives.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
+    lib.chai_cluster_sweep.argtypes = [vp, ci, ci, ci, ci, ci, ctypes.c_uint64, vp, vp, vp]
     for name in ("chai_decode_workspace_bytes", "chai_prefill_workspace_bytes", "chai_decode_qkv_workspace_bytes",
                  "chai_prefill_qkv_workspace_bytes"):
         getattr(lib, name).argtypes = [ci, ci, ci, ci, ci, ci]
@@ -153,6 +154,18 @@ def chai_cluster_heads(features, k: int, max_iter: int = 20, seed: int = 0, want
     _check(load().chai_cluster_heads(_ptr(features), B, H, F, k, max_iter, seed, _ptr(membership), _ptr(reps),
                                      _ptr(k_eff), _ptr(inertia), _stream()))
     return membership, reps, k_eff, inertia
+
+
+def chai_cluster_sweep(features, k_max: int, max_iter: int = 20, seed: int = 0):
+    """features [B,H,F] fp32 -> (inertia curve [B,k_max] f64, knee [B] int32): k-means for every k = 1..k_max."""
+    _dev(features)
+    if features.dtype != torch.float32:
+        raise TypeError("features must be float32")
+    B, H, F = features.shape
+    curve = torch.empty((B, k_max), device=features.device, dtype=torch.float64)
+    pick = torch.empty((B,), device=features.device, dtype=torch.int32)
+    _check(load().chai_cluster_sweep(_ptr(features), B, H, F, k_max, max_iter, seed, _ptr(curve), _ptr(pick), _stream()))
+    return curve, pick
 
 
 def chai_select_representatives(features, membership, k: int):

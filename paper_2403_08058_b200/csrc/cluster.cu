@@ -51,10 +51,15 @@ __device__ __forceinline__ double sqdist(const double* x, const double* y, int F
 }
 
 // One CTA per request.  Shared memory: X [H,F], C [k,F], dist [H,k] doubles; a, prev, count ints.
-__global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ features, int H, int F, int k,
+// Sweep mode (k_arg = 0, grid (B, k_max)): CTA (b, j) clusters request b with k = j + 1 and writes only the
+// inertia, to inertia[b * k_max + j]; the other outputs are not written.
+__global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ features, int H, int F, int k_arg,
                                                      int max_iter, unsigned long long seed,
                                                      int32_t* __restrict__ membership, int32_t* __restrict__ reps,
                                                      int32_t* __restrict__ k_eff, double* __restrict__ inertia) {
+    const bool sweep = k_arg == 0;
+    const int k = sweep ? (int)blockIdx.y + 1 : k_arg;
+    if (sweep) inertia += (size_t)blockIdx.x * gridDim.y + blockIdx.y - blockIdx.x;  // so that inertia[b] below is the curve entry
     extern __shared__ double smem_d[];
     double* X = smem_d;
     double* C = X + (size_t)H * F;
@@ -147,23 +152,23 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
     if (tid == 0) {
         for (int c = 0; c < k; ++c) {
             newid[c] = -1;
-            reps[(size_t)b * k + c] = -1;
+            if (!sweep) reps[(size_t)b * k + c] = -1;
         }
         int next = 0;
         for (int h = 0; h < H; ++h) {
             if (newid[a[h]] < 0) {
                 newid[a[h]] = next;
-                reps[(size_t)b * k + next] = h;
+                if (!sweep) reps[(size_t)b * k + next] = h;
                 ++next;
             }
         }
-        k_eff[b] = next;
+        if (!sweep) k_eff[b] = next;
         s_ncentres = next;
     }
     __syncthreads();
     for (int h = tid; h < H; h += nt) {
         a[h] = newid[a[h]];
-        membership[(size_t)b * H + h] = a[h];
+        if (!sweep) membership[(size_t)b * H + h] = a[h];
     }
     if (inertia == nullptr) return;
     __syncthreads();
@@ -241,6 +246,38 @@ select_reps_kernel(const float* __restrict__ features, const int32_t* __restrict
     }
 }
 
+// Knee of a clustering-error curve e(1..n) (Section 3.2 / Fig. 8: the number of clusters is read off where
+// the error stops falling quickly; the paper does it by eye).  Rule: scale k to x in [0,1] and the error to
+// y in [0,1] (y = 1 at the largest error, 0 at the smallest); the knee is the k that lies farthest below the
+// straight line from (0,1) to (1,0), i.e. maximises 1 - x - y; ties go to the smaller k.  One thread per request.
+__global__ void knee_kernel(const double* __restrict__ curve, int B, int n, int32_t* __restrict__ k_pick) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const double* e = curve + (size_t)b * n;
+    double lo = e[0], hi = e[0];
+    for (int i = 1; i < n; ++i) {
+        lo = e[i] < lo ? e[i] : lo;
+        hi = e[i] > hi ? e[i] : hi;
+    }
+    int best = 1;
+    if (n > 1 && hi > lo) {
+        const double span = __dsub_rn(hi, lo);
+        double best_v = 0.0;
+        bool have = false;
+        for (int i = 0; i < n; ++i) {
+            const double x = __ddiv_rn((double)i, (double)(n - 1));
+            const double y = __ddiv_rn(__dsub_rn(e[i], lo), span);
+            const double v = __dsub_rn(__dsub_rn(1.0, x), y);
+            if (!have || v > best_v) {
+                best_v = v;
+                best = i + 1;
+                have = true;
+            }
+        }
+    }
+    k_pick[b] = best;
+}
+
 static size_t kmeans_smem_bytes(int H, int F, int k) {
     return sizeof(double) * ((size_t)H * F + (size_t)k * F + (size_t)H * k) + sizeof(int) * (2 * (size_t)H + 2 * (size_t)k);
 }
@@ -309,6 +346,29 @@ int chai_select_representatives(const float* features, const int32_t* membership
     if (e != cudaSuccess) return cuda_fail(e, "select_reps_kernel shared-memory opt-in");
     select_reps_kernel<<<B, 256, smem, s>>>(features, membership, H, F, k, reps);
     CHAI_LAUNCH_CHECK("select_reps_kernel launch");
+    return CHAI_OK;
+}
+
+int chai_cluster_sweep(const float* features, int B, int H, int F, int k_max, int max_iter, uint64_t seed,
+                       double* inertia_curve, int32_t* k_pick, void* stream) {
+    using namespace chai;
+    CHAI_REQUIRE(features && inertia_curve, CHAI_ERR_INVALID_ARG, "chai_cluster_sweep: null pointer");
+    CHAI_REQUIRE(B > 0 && H > 0 && F > 0 && max_iter > 0, CHAI_ERR_INVALID_ARG, "chai_cluster_sweep: sizes must be positive");
+    CHAI_REQUIRE(k_max >= 1 && k_max <= H, CHAI_ERR_INVALID_ARG, "chai_cluster_sweep: need 1 <= k_max <= H (k_max=%d, H=%d)",
+                 k_max, H);
+    const size_t smem = kmeans_smem_bytes(H, F, k_max);
+    CHAI_REQUIRE(H <= 1024 && B <= 65535 && smem <= 200 * 1024, CHAI_ERR_UNSUPPORTED,
+                 "chai_cluster_sweep: problem needs %zu bytes of shared memory (limit 204800)", smem);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaFuncSetAttribute(kmeans_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return cuda_fail(e, "kmeans_kernel shared-memory opt-in");
+    kmeans_kernel<<<dim3(B, k_max), 256, smem, s>>>(features, H, F, 0, max_iter, (unsigned long long)seed, nullptr,
+                                                    nullptr, nullptr, inertia_curve);
+    CHAI_LAUNCH_CHECK("kmeans_kernel (sweep) launch");
+    if (k_pick != nullptr) {
+        knee_kernel<<<(B + 127) / 128, 128, 0, s>>>(inertia_curve, B, k_max, k_pick);
+        CHAI_LAUNCH_CHECK("knee_kernel launch");
+    }
     return CHAI_OK;
 }
 

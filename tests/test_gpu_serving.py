@@ -245,3 +245,25 @@ def test_select_representatives_matches_oracle():
     f2 = torch.tensor([[[0.0], [1.0], [10.0], [4.0], [3.0]]])
     m2 = torch.tensor([[0, 1, 0, 0, 1]], dtype=torch.int32)
     assert chai.chai_select_representatives(f2.to(DEV), m2.to(DEV), 3).cpu().tolist() == [[3, 1, -1]]
+
+
+@pytest.mark.parametrize("k_true,H,F", [(4, 32, 25), (8, 32, 25), (13, 52, 64)])
+def test_cluster_sweep_matches_oracle_and_finds_the_planted_count(k_true, H, F):
+    feats, _, _ = synth.blob_features(3, H, F, k_true, seed=k_true + 1, noise=0.05)
+    curve, knee = chai.chai_cluster_sweep(torch.as_tensor(feats).to(DEV), H, 20, 0)
+    ref_curve, ref_knee = orc.cluster_sweep(feats, H, 20, 0)
+    got = curve.cpu().numpy()
+    assert np.allclose(got, ref_curve, rtol=1e-12, atol=1e-18)
+    assert knee.cpu().tolist() == ref_knee.tolist() == [k_true] * 3
+    # column k-1 of the sweep is what a single clustering call with k clusters reports
+    _, _, _, inertia = chai.chai_cluster_heads(torch.as_tensor(feats).to(DEV), k_true, 20, 0)
+    assert np.array_equal(inertia.cpu().numpy(), got[:, k_true - 1])
+
+
+def test_cluster_sweep_on_unstructured_features():
+    rng = np.random.default_rng(9)
+    feats = rng.normal(size=(2, 24, 10)).astype(np.float32)
+    curve, knee = chai.chai_cluster_sweep(torch.as_tensor(feats).to(DEV), 24, 20, 3)
+    ref_curve, ref_knee = orc.cluster_sweep(feats, 24, 20, 3)
+    assert np.allclose(curve.cpu().numpy(), ref_curve, rtol=1e-12, atol=1e-18)
+    assert knee.cpu().tolist() == ref_knee.tolist()

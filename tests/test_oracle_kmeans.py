@@ -207,3 +207,25 @@ def test_closest_representatives_hand_cases():
                 continue
             d = ((x[b, idx] - x[b, idx].mean(axis=0)) ** 2).sum(axis=1)
             assert got[b, c] == idx[np.argmin(d)]
+
+
+def test_knee_rule_on_hand_made_curves():
+    assert orc.knee_of_curve([10.0, 10.0, 10.0]) == 1                      # flat
+    assert orc.knee_of_curve([7.0]) == 1
+    # falls linearly to zero at k = 4 of 10, flat afterwards: the corner is the knee
+    assert orc.knee_of_curve([9.0, 6.0, 3.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0]) == 4
+    # a straight line has no knee: every point is on the chord, the smallest k wins the tie
+    assert orc.knee_of_curve([4.0, 3.0, 2.0, 1.0, 0.0]) == 1
+    # convex curve 1/k on 1..8: maximise 1 - (k-1)/7 - (1/k - 1/8)/(7/8) -> k = 3 (0.476 vs 0.449 at k = 2, 0.429 at k = 4)
+    assert orc.knee_of_curve([1.0 / k for k in range(1, 9)]) == 3
+
+
+def test_cluster_sweep_recovers_the_planted_count_and_is_monotone_enough():
+    for k_true, H in [(4, 32), (8, 32), (6, 24)]:
+        feats, planted, _ = synth.blob_features(2, H, 25, k_true, seed=k_true, noise=0.05)
+        curve, knee = orc.cluster_sweep(feats, H, 20, 0)
+        assert curve.shape == (2, H)
+        assert knee.tolist() == [k_true, k_true]
+        assert np.all(curve[:, -1] <= 1e-20)                 # k = H: every head its own cluster
+        # with the planted count the error is at the noise floor, far below one cluster less
+        assert np.all(curve[:, k_true - 1] < 0.2 * curve[:, k_true - 2])
