@@ -365,6 +365,47 @@ def bench_serving(device, peaks, iters=20, warmup=3):
             "l2": "flushed by a 256 MB write before every timed call"}
 
 
+def bench_fp8(device, peaks, iters=20, warmup=3):
+    """Decode on e4m3 caches at workload 2's layer shape for k = 8 and k = 32: the layer calls run back to back over
+    eight different cache sets (1.3 - 2.2 GB, larger than L2), as in the main decode number."""
+    w = synth.WORKLOADS[2]
+    B, H, T, D = w.B, w.H, w.T, w.D
+    res = {}
+    for k in (8, 32):
+        sets = []
+        for i in range(8):
+            c = synth.decode_layer(2, i, 2, device=device, B=B, H=H, T=T, k=k)
+            k8, ks = chai.chai_quantize_cache_fp8(c["k_rep"])
+            v8, vs = chai.chai_quantize_cache_fp8(c["v"])
+            sets.append((c["q"], k8, v8, ks, vs, c["membership"], c["reps"], c["scale"]))
+            del c
+        ws = chai.new_workspace(int(chai.load().chai_decode_fp8_workspace_bytes(B, H, k, T, D)), device)
+        out = torch.empty_like(sets[0][0])
+
+        def step():
+            for (q, k8, v8, ks, vs, mem, reps, scale) in sets:
+                chai.chai_decode_attention_fp8(q, k8, v8, ks, vs, mem, reps, scale, out=out, workspace=ws)
+
+        for _ in range(warmup):
+            step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(iters):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / (iters * len(sets))
+        nbytes = (k + H) * B * T * D * 1 + (k + H) * B * D * 2 + 4 * B * (H + k) * 2
+        gbs = nbytes / (us * 1e-6) / 1e9
+        res[f"k{k}"] = {"us_per_layer": us, "algorithmic_mb": nbytes / 1e6, "gbs": gbs,
+                        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
+                                     "frac": gbs / peaks["hbm"], "peak_source": peaks["source"], "traffic": None}}
+        del sets
+    res["workload"] = "config2 layer shape (B 16, H 32, T 2048, D 128), e4m3 caches + per-plane scales, bf16 q/out"
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -459,6 +500,7 @@ def main():
             line["prefill"] = bench_prefill(device, peaks)
             line["compaction"] = bench_compaction(device, peaks)
             line["serving"] = bench_serving(device, peaks)
+            line["fp8_decode"] = bench_fp8(device, peaks)
             line["cpu_baseline"] = cpu_baseline_decode(args.workload, 0)
         print(json.dumps(line))
     ranks.close()

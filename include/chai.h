@@ -54,7 +54,7 @@ typedef enum {
     CHAI_ERR_CACHE_FULL = 7      /* device status word only: chai_append_kv found seq_lens[b] outside [0, T_cap) */
 } chai_status_t;
 
-typedef enum { CHAI_F32 = 0, CHAI_BF16 = 1 } chai_dtype_t;
+typedef enum { CHAI_F32 = 0, CHAI_BF16 = 1, CHAI_FP8_E4M3 = 2 /* caches of chai_decode_attention_fp8 only */ } chai_dtype_t;
 
 /* size of the built-in scratch array used by chai_decode_attention_static */
 #define CHAI_DECODE_STATIC_SCRATCH_BYTES (8u << 20)
@@ -283,6 +283,32 @@ int chai_prefill_attention_qkv(const void* q, const void* k_rep, const void* v_r
  */
 int chai_broadcast_membership(const int32_t* membership_static, const int32_t* reps_static, int32_t* membership,
                               int32_t* reps, int B, int H, int k, void* stream);
+
+/*
+ * fp8 caches (the paper treats head clustering as orthogonal to quantisation; one byte per cached element
+ * halves the decode step's bytes once more).  Format: e4m3 (4 exponent bits, bias 7, 3 mantissa bits, no
+ * infinities, largest finite value 448), one fp32 scale per cache plane; a stored byte stands for
+ * decode(byte) * scale.
+ *
+ * chai_quantize_cache_fp8: src [n_planes,T_cap,D] bf16 -> dst [n_planes,T_cap,D] bytes + scales [n_planes].
+ *   Per plane: scale = max|x| over rows [0,T) divided by 448 in fp32 (1 if the plane is all zero); each element
+ *   is x / scale (fp32 division) rounded to the nearest e4m3 value, ties to even, saturating.  Rows >= T are not
+ *   touched.  Works for K_rep (n_planes = B*k) and V (n_planes = B*H) alike.
+ *
+ * chai_decode_attention_fp8: the decode step of chai_decode_attention / _ragged on such caches.
+ *   q, out [B,H,D] bf16; k_rep, v: e4m3 bytes; k_scale [B,k], v_scale [B,H] fp32 (device);
+ *   seq_lens NULL or [B] device; k_batch_stride in elements (= bytes), 0 for dense.
+ *   out[b][h] = v_scale[b][h] * sum_t softmax_t(scale * k_scale[b][c] * q[b][r] . k8[b][c][t]) * v8[b][h][t]
+ *   with fp32 accumulation.  Workspace: chai_decode_fp8_workspace_bytes.  Runs on the persistent kernel only;
+ *   CHAI_ERR_UNSUPPORTED on a device without cooperative launch.
+ */
+int chai_quantize_cache_fp8(const void* src, void* dst, float* scales, int n_planes, int T, int T_cap, int D,
+                            void* stream);
+size_t chai_decode_fp8_workspace_bytes(int B, int H, int k, int T, int D);
+int chai_decode_attention_fp8(const void* q, const void* k_rep, const void* v, const float* k_scale, const float* v_scale,
+                              const int32_t* membership, const int32_t* reps, const int32_t* seq_lens, void* out, int B,
+                              int H, int k, int T, int T_cap, int D, size_t k_batch_stride, float scale, void* workspace,
+                              size_t workspace_bytes, void* stream);
 
 /* Blocking read of the status word a decode/prefill call left in `workspace`
  * (synchronises `stream`).  *status_out receives a chai_status_t. */

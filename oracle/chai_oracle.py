@@ -277,3 +277,58 @@ def cluster_sweep(features, k_max: int, max_iter: int = 20, seed: int = 0):
     for k in range(1, k_max + 1):
         curve[:, k - 1] = kmeans(x, k, max_iter, seed)["inertia"]
     return curve, np.array([knee_of_curve(curve[b]) for b in range(B)], dtype=np.int32)
+
+
+# ---- fp8 (e4m3) caches: the number format written out, and the decode step on dequantised values ---------
+
+def e4m3_values() -> np.ndarray:
+    """The 256 numbers an e4m3 byte stands for: sign bit, 4 exponent bits (bias 7), 3 mantissa bits; exponent
+    field 0 is subnormal (m/8 * 2^-6); there are no infinities and only exponent 15 with mantissa 7 is NaN."""
+    out = np.empty(256, dtype=np.float64)
+    for byte in range(256):
+        sign = -1.0 if byte & 0x80 else 1.0
+        e, m = (byte >> 3) & 0xF, byte & 0x7
+        if e == 15 and m == 7:
+            out[byte] = np.nan
+        elif e == 0:
+            out[byte] = sign * (m / 8.0) * 2.0 ** -6
+        else:
+            out[byte] = sign * (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return out
+
+
+def quantize_cache_fp8(cache_f32: np.ndarray, T: int):
+    """cache [planes..., T_cap, D] (values exactly representable in float32, e.g. widened bf16) ->
+    (bytes uint8 same shape, scales float32 [planes...]).  Per plane: scale = float32(max|x| over rows [0,T)) /
+    float32(448) in float32 (1 if the plane is zero); element = float32(x) / scale in float32, rounded to the
+    nearest e4m3 value, ties to the even mantissa, saturated to +-448.  Rows >= T are left zero."""
+    x = np.asarray(cache_f32, dtype=np.float32)
+    lead = x.shape[:-2]
+    flat = x.reshape((-1,) + x.shape[-2:])
+    vals = e4m3_values()
+    pos = vals[:127]                      # bytes 0..126: the finite non-negative values in ascending order
+    q = np.zeros(flat.shape, dtype=np.uint8)
+    scales = np.empty(flat.shape[0], dtype=np.float32)
+    for p in range(flat.shape[0]):
+        amax = np.float32(np.max(np.abs(flat[p, :T]))) if T > 0 else np.float32(0)
+        scale = np.float32(amax / np.float32(448.0)) if amax > 0 else np.float32(1.0)
+        scales[p] = scale
+        y = (flat[p, :T] / scale).astype(np.float32).astype(np.float64)
+        mag = np.minimum(np.abs(y), 448.0)
+        hi = np.searchsorted(pos, mag, side="left")          # first value >= mag
+        hi = np.minimum(hi, 126)
+        lo = np.maximum(hi - 1, 0)
+        d_hi, d_lo = pos[hi] - mag, mag - pos[lo]
+        take_lo = (d_lo < d_hi) | ((d_lo == d_hi) & (lo % 2 == 0))   # ties: even mantissa = even byte
+        code = np.where(take_lo, lo, hi).astype(np.uint8)
+        code = np.where(pos[hi] == mag, hi, code).astype(np.uint8)
+        q[p, :T] = code | np.where(np.signbit(y), 0x80, 0).astype(np.uint8)
+    return q.reshape(x.shape), scales.reshape(lead)
+
+
+def decode_attention_fp8(q, k8, v8, k_scale, v_scale, membership, reps, seq_lens, scale: float) -> np.ndarray:
+    """The ragged decode definition on the numbers the fp8 caches stand for: byte -> e4m3 value * plane scale."""
+    vals = e4m3_values()
+    k_rep = vals[np.asarray(k8)] * np.asarray(k_scale, dtype=np.float64)[:, :, None, None]
+    v = vals[np.asarray(v8)] * np.asarray(v_scale, dtype=np.float64)[:, :, None, None]
+    return decode_attention_ragged(q, k_rep, v, membership, reps, seq_lens, scale)

@@ -12,7 +12,7 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(ROOT, "build", "chai")
 LIB = os.path.join(PKG, "libchai.so")
 SOURCES = ["api.cu", "cluster.cu", "compact.cu", "decode.cu", "decode_persist.cu", "prefill_simt.cu", "prefill_tc.cu",
-           "serving.cu", "variants.cu"]
+           "serving.cu", "variants.cu", "fp8.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

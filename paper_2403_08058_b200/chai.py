@@ -29,6 +29,7 @@ EXPORTS = [
     "chai_prefill_attention_from", "chai_prefill_attention_simt_from",
     "chai_decode_qkv_workspace_bytes", "chai_decode_attention_qkv", "chai_prefill_qkv_workspace_bytes",
     "chai_prefill_attention_qkv", "chai_broadcast_membership", "chai_select_representatives", "chai_cluster_sweep",
+    "chai_quantize_cache_fp8", "chai_decode_fp8_workspace_bytes", "chai_decode_attention_fp8",
 ]
 DECODE_STATIC_SCRATCH_BYTES = 8 << 20   # CHAI_DECODE_STATIC_SCRATCH_BYTES
 
@@ -63,6 +64,10 @@ def load() -> ctypes.CDLL:
     lib.chai_prefill_attention_qkv.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
     lib.chai_broadcast_membership.argtypes = [vp, vp, vp, vp, ci, ci, ci, vp]
     lib.chai_select_representatives.argtypes = [vp, vp, ci, ci, ci, ci, vp, vp]
+    lib.chai_quantize_cache_fp8.argtypes = [vp, vp, vp, ci, ci, ci, ci, vp]
+    lib.chai_decode_fp8_workspace_bytes.argtypes = [ci, ci, ci, ci, ci]
+    lib.chai_decode_fp8_workspace_bytes.restype = sz
+    lib.chai_decode_attention_fp8.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, sz, cf, vp, sz, vp]
     lib.chai_cluster_sweep.argtypes = [vp, ci, ci, ci, ci, ci, ctypes.c_uint64, vp, vp, vp]
     for name in ("chai_decode_workspace_bytes", "chai_prefill_workspace_bytes", "chai_decode_qkv_workspace_bytes",
                  "chai_prefill_qkv_workspace_bytes"):
@@ -384,6 +389,37 @@ def chai_broadcast_membership(membership_static, reps_static, B: int):
     _check(load().chai_broadcast_membership(_ptr(membership_static), _ptr(reps_static), _ptr(membership), _ptr(reps), B,
                                             H, k, _stream()))
     return membership, reps
+
+
+def chai_quantize_cache_fp8(cache, T: int | None = None):
+    """cache [B,P,T_cap,D] bf16 -> (bytes [B,P,T_cap,D] uint8 in e4m3, scales [B,P] fp32); rows [0,T) are converted."""
+    _dev(cache)
+    if cache.dtype != torch.bfloat16:
+        raise TypeError("the cache must be bfloat16")
+    B, P, T_cap, D = cache.shape
+    T = T_cap if T is None else T
+    q8 = torch.zeros((B, P, T_cap, D), device=cache.device, dtype=torch.uint8)
+    scales = torch.empty((B, P), device=cache.device, dtype=torch.float32)
+    _check(load().chai_quantize_cache_fp8(_ptr(cache), _ptr(q8), _ptr(scales), B * P, T, T_cap, D, _stream()))
+    return q8, scales
+
+
+def chai_decode_attention_fp8(q, k_rep8, v8, k_scale, v_scale, membership, reps, scale: float, T: int | None = None,
+                              seq_lens=None, out=None, workspace=None):
+    """Decode on e4m3 caches: q [B,H,D] bf16, k_rep8 [B,k|H,T_cap,D] uint8, v8 [B,H,T_cap,D] uint8, scales fp32."""
+    _dev(q, k_rep8, v8, k_scale, v_scale, membership, reps, seq_lens, out, workspace)
+    B, H, D = q.shape
+    k, T_cap = reps.shape[1], v8.shape[2]
+    T = T_cap if T is None else T
+    stride = k_rep8.shape[1] * T_cap * D
+    if out is None:
+        out = torch.empty_like(q)
+    if workspace is None:
+        workspace = new_workspace(int(load().chai_decode_fp8_workspace_bytes(B, H, k, T, D)), q.device)
+    _check(load().chai_decode_attention_fp8(_ptr(q), _ptr(k_rep8), _ptr(v8), _ptr(k_scale), _ptr(v_scale),
+                                            _ptr(membership), _ptr(reps), _ptr(seq_lens), _ptr(out), B, H, k, T, T_cap, D,
+                                            stride, scale, _ptr(workspace), workspace.numel(), _stream()))
+    return out
 
 
 def chai_device_status(workspace) -> int:

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp8.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stdio.h>
@@ -25,7 +26,7 @@ int cuda_fail(cudaError_t e, const char* what);  // records the text, returns CH
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-inline size_t elem_size(int dtype) { return dtype == CHAI_BF16 ? 2 : 4; }
+inline size_t elem_size(int dtype) { return dtype == CHAI_BF16 ? 2 : (dtype == CHAI_FP8_E4M3 ? 1 : 4); }
 
 #define CHAI_REQUIRE(cond, code, ...)            \
     do {                                         \
@@ -79,6 +80,30 @@ struct Vec16<__nv_bfloat16> {
         f[5] = __uint_as_float(r.z & 0xffff0000u);
         f[6] = __uint_as_float(r.w << 16);
         f[7] = __uint_as_float(r.w & 0xffff0000u);
+    }
+};
+
+// One byte per element: fp8 e4m3 (4 exponent bits, bias 7, 3 mantissa bits, no infinities) as stored by
+// chai_quantize_cache_fp8; the value it stands for is the decoded number times the plane's scale.
+struct Fp8E4M3 {
+    unsigned char bits;
+};
+template <>
+struct Vec16<Fp8E4M3> {
+    static constexpr int N = 16;
+    __device__ __forceinline__ static void unpack(const uint4& r, float* f) {
+        const unsigned w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __half2_raw lo = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(w[i] & 0xffffu), __NV_E4M3);
+            const __half2_raw hi = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(w[i] >> 16), __NV_E4M3);
+            const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&lo));
+            const float2 b = __half22float2(*reinterpret_cast<const __half2*>(&hi));
+            f[4 * i + 0] = a.x;
+            f[4 * i + 1] = a.y;
+            f[4 * i + 2] = b.x;
+            f[4 * i + 3] = b.y;
+        }
     }
 };
 

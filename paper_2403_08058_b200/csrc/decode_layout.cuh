@@ -9,7 +9,9 @@ constexpr int kDecThreads = 256;
 constexpr int kDecWarps = kDecThreads / 32;
 constexpr int kStepsK = 8;   // independent 16-byte loads per thread in flight, score kernel
 constexpr int kStepsV = 16;  // rows per thread in a value chunk (two batches of 8 loads)
-constexpr int kTileBytes = 32768;  // persistent kernel: one ring slot = TR cache rows
+constexpr int kTileBytes = 32768;     // persistent kernel: one ring slot = TR cache rows ...
+constexpr int kTileBytesFp8 = 16384;  // ... of half the size for one-byte elements (same number of elements per tile)
+inline int decode_tile_bytes(int dtype) { return dtype == CHAI_FP8_E4M3 ? kTileBytesFp8 : kTileBytes; }
 
 struct DecodeLayout {
     int CK, CV, nK, nV;  // split kernels: rows per key / value chunk and chunks per plane
@@ -29,7 +31,7 @@ inline bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLa
     L->CV = rps * kStepsV;
     L->nK = (T + L->CK - 1) / L->CK;
     L->nV = (T + L->CV - 1) / L->CV;
-    L->TR = kTileBytes / (D * es);
+    L->TR = decode_tile_bytes(dtype) / (D * es);
     // the persistent kernel deals key work tile by tile and value work in items of 2 tiles
     const int pk = (T + L->TR - 1) / L->TR, pv = (T + 2 * L->TR - 1) / (2 * L->TR);
     L->capK = pk > L->nK ? pk : L->nK;
@@ -61,6 +63,7 @@ constexpr int kDecodeNotLaunched = -1;
 int launch_decode_persistent(const void* q, const void* k_rep, const void* v, const int32_t* membership,
                              const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T,
                              int T_cap, int D, size_t k_batch_stride, float scale, int dtype, char* ws,
-                             const DecodeLayout& L, cudaStream_t s);
+                             const DecodeLayout& L, cudaStream_t s, const float* k_scale = nullptr,
+                             const float* v_scale = nullptr);  // scales: fp8 caches only (dtype CHAI_FP8_E4M3)
 
 }  // namespace chai

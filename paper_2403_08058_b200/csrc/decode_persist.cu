@@ -33,9 +33,19 @@
 namespace chai {
 namespace pd {
 
-constexpr int CONSUMER_WARPS = 8;
-constexpr int THREADS = CONSUMER_WARPS * 32 + 32;
-constexpr int STAGES = 6;                  // 192 KB of cache rows in flight per SM
+// Shape of the pipeline per cache element type: W consumer warps (+ 1 producer warp), a ring of STAGES slots
+// of TILE bytes.  A slot is held while its tile is in flight AND while a warp works on it, so at most STAGES
+// warps are busy at once.  For one-byte elements the per-element work (conversion, fused multiply-adds) is what
+// limits the kernel, not the bytes: tiles keep the element count of the two-byte case (half the bytes), and more
+// slots and more warps work side by side.
+template <typename T>
+struct Cfg {
+    static constexpr int W = 8, STAGES = 6, TILE = kTileBytes;      // 192 KB of cache rows in flight per SM
+};
+template <>
+struct Cfg<Fp8E4M3> {
+    static constexpr int W = 12, STAGES = 12, TILE = kTileBytesFp8;  // 192 KB in 12 slots, 12 consumer warps
+};
 constexpr int MAX_IV = 4;                  // tiles per value item
 constexpr int ITEM_SLOTS = 8;              // value items whose tile partials may be open in one CTA
 constexpr int TABLE_CAP = 2048;            // heads whose cluster id is cached in shared memory
@@ -48,8 +58,9 @@ struct TileMeta {
     int islot;     // shared-memory slot of the item's tile partials
 };
 
+template <int STAGES, int TILE>
 struct Smem {
-    alignas(128) unsigned char ring[STAGES][kTileBytes];
+    alignas(128) unsigned char ring[STAGES][TILE];
     alignas(16) float part[ITEM_SLOTS][MAX_IV][128];  // per-tile partial sums of open items
     float lpart[ITEM_SLOTS][MAX_IV];
     alignas(8) unsigned long long full[STAGES];
@@ -69,6 +80,8 @@ struct Params {
     const void* v;
     const int32_t* membership;
     const int32_t* reps;
+    const float* k_scale;        // fp8 caches: scale of each representative key plane [B,k] / value plane [B,H]
+    const float* v_scale;
     const int32_t* seq_lens;     // per-request context length, or null (all T)
     size_t k_batch_bytes;        // bytes between two requests' representative planes in k_rep
     void* out;
@@ -189,6 +202,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 
 template <typename T, int D>
 struct Geom {
+    static constexpr int kTileBytes = Cfg<T>::TILE;
     static constexpr int EPV = 16 / (int)sizeof(T);   // elements per 16-byte vector
     static constexpr int ROW_BYTES = D * (int)sizeof(T);
     static constexpr int TR = kTileBytes / ROW_BYTES;  // rows per tile
@@ -200,25 +214,27 @@ struct Geom {
 };
 
 struct Ring {
-    uint32_t full0, empty0, data0;
+    uint32_t full0, empty0, data0, tile_bytes;
     __device__ __forceinline__ uint32_t full(int slot) const { return full0 + 8 * slot; }
     __device__ __forceinline__ uint32_t empty(int slot) const { return empty0 + 8 * slot; }
-    __device__ __forceinline__ uint32_t data(int slot) const { return data0 + kTileBytes * slot; }
+    __device__ __forceinline__ uint32_t data(int slot) const { return data0 + tile_bytes * slot; }
 };
 
 // RAGGED = false is the equal-length, dense-cache case: per-request lengths, the K batch stride and the
 // skipping of tiles beyond a request's end compile away (the streaming loops are sensitive to every
 // instruction on the producer thread and in the per-tile consumer chain).
-template <typename T, int D, bool RAGGED>
-__global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Params P) {
+// T = element type of the caches, TQ = element type of the queries and the output (they differ for fp8 caches).
+template <typename T, typename TQ, int D, bool RAGGED>
+__global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kernel(const Params P) {
     using G = Geom<T, D>;
-    constexpr int W = CONSUMER_WARPS;
+    constexpr int W = Cfg<T>::W, STAGES = Cfg<T>::STAGES, THREADS = W * 32 + 32;
+    using SmemT = Smem<STAGES, Cfg<T>::TILE>;
     extern __shared__ unsigned char smem_raw[];
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    SmemT& sm = *reinterpret_cast<SmemT*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, ncta = gridDim.x;
     volatile int* abort_flag = &sm.abort_flag;
-    const Ring ring{smem_u32(&sm.full[0]), smem_u32(&sm.empty[0]), smem_u32(&sm.ring[0][0])};
+    const Ring ring{smem_u32(&sm.full[0]), smem_u32(&sm.empty[0]), smem_u32(&sm.ring[0][0]), (uint32_t)Cfg<T>::TILE};
     const int B = P.B, H = P.H, k = P.k, T_len = P.T;
     const bool use_table = B * H <= TABLE_CAP;
     const int tp = (T_len + G::TR - 1) / G::TR;          // tiles per cache plane
@@ -384,9 +400,13 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
 #pragma unroll
             for (int e = 0; e < G::EPV; ++e) qf[e] = 0.f;
             if (live) {
-                const uint4 qv = *reinterpret_cast<const uint4*>(static_cast<const T*>(P.q) + ((size_t)b * H + rep) * D + part * G::EPV);
-                Vec16<T>::unpack(qv, qf);
+                // the EPV query elements that face this lane's 16-byte slice of a key row
+                const TQ* qsrc = static_cast<const TQ*>(P.q) + ((size_t)b * H + rep) * D + part * G::EPV;
+#pragma unroll
+                for (int x = 0; x < G::EPV / Vec16<TQ>::N; ++x)
+                    Vec16<TQ>::unpack(*reinterpret_cast<const uint4*>(qsrc + x * Vec16<TQ>::N), qf + x * Vec16<TQ>::N);
             }
+            const float kscale = P.k_scale ? P.scale * __ldg(P.k_scale + plane) : P.scale;  // fp8 keys carry a scale per plane
             const int slot = n % STAGES;
             if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag) &&
                                                      mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
@@ -427,7 +447,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                             v[x] = keep + __shfl_xor_sync(0xffffffffu, send, o);
                         }
                     }
-                    const float sc = v[0] * P.scale;
+                    const float sc = v[0] * kscale;
                     const int row = (bt * G::LPR + part) * G::RPW + sub;
                     if (row < rows) {  // rows past the end of a ragged last tile hold stale bytes
                         srow[row] = sc;
@@ -460,7 +480,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
             }
         }
         // ---- phase V: tiles of claimed items ----
-        T* outp = static_cast<T*>(P.out);
+        TQ* outp = static_cast<TQ*>(P.out);
         for (int n = n_issued + ((warp - n_issued) % W + W) % W;; n += W) {  // this warp's next position
             const int slot = n % STAGES;
             if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag) &&
@@ -547,7 +567,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                 // unresolved head: zero output, flagged after the status reset (ordered by the layer's first flag)
                 ok = flags_wait(P.flags, 1, P.token, lane, abort_flag);
                 if (ok && lane == 0) flag_bad_membership(P.hdr, b, h);
-                for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<T>(0.f);
+                for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<TQ>(0.f);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(ring.empty(slot));  // the tile's bytes are no longer needed
@@ -612,8 +632,9 @@ __global__ void __launch_bounds__(THREADS, 1) decode_persistent_kernel(const Par
                     ll += __ldcg(&P.lpart[(size_t)head * P.nVi + i]);
                 }
 #pragma unroll
+                const float vscale = P.v_scale ? __ldg(P.v_scale + head) : 1.f;  // fp8 values carry a scale per plane
                 for (int e = 0; e < DPL; ++e)  // (an empty context has no probabilities: the output is zero)
-                    outp[(size_t)head * D + lane * DPL + e] = from_float<T>(ll > 0.f ? o[e] / ll : 0.f);
+                    outp[(size_t)head * D + lane * DPL + e] = from_float<TQ>(ll > 0.f ? o[e] / ll * vscale : 0.f);
             }
         }
     }
@@ -638,24 +659,25 @@ static DeviceInfo& device_info(int dev) {
     return d;
 }
 
-template <typename T, int D, bool RAGGED>
+template <typename T, typename TQ, int D, bool RAGGED>
 static int launch(const Params& P0, int ncta, int dev, cudaStream_t s) {
     Params P = P0;
-    const size_t smem = sizeof(Smem) + 128;
-    static bool configured_dev[64] = {};
+    constexpr int THREADS = Cfg<T>::W * 32 + 32;
+    const size_t smem = sizeof(Smem<Cfg<T>::STAGES, Cfg<T>::TILE>) + 128;
+    static bool configured_dev[64] = {};  // (one flag array per instantiation)
     bool& configured = configured_dev[dev & 63];
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(decode_persistent_kernel<T, D, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(decode_persistent_kernel<T, TQ, D, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel shared-memory opt-in");
         int per_sm = 0;
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_persistent_kernel<T, D, RAGGED>, THREADS, smem);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_persistent_kernel<T, TQ, D, RAGGED>, THREADS, smem);
         if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel occupancy query");
         if (per_sm < 1) return kDecodeNotLaunched;
         configured = true;
     }
     void* args[] = {&P};
     // cooperative launch: value tiles wait for flags set by other CTAs, so all CTAs must be resident at once
-    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_persistent_kernel<T, D, RAGGED>), dim3(ncta),
+    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_persistent_kernel<T, TQ, D, RAGGED>), dim3(ncta),
                                                 dim3(THREADS), args, smem, s);
     if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel launch");
     return CHAI_OK;
@@ -666,7 +688,7 @@ static int launch(const Params& P0, int ncta, int dev, cudaStream_t s) {
 int launch_decode_persistent(const void* q, const void* k_rep, const void* v, const int32_t* membership,
                              const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T,
                              int T_cap, int D, size_t k_batch_stride, float scale, int dtype, char* ws,
-                             const DecodeLayout& L, cudaStream_t s) {
+                             const DecodeLayout& L, cudaStream_t s, const float* k_scale, const float* v_scale) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return kDecodeNotLaunched;
     const pd::DeviceInfo& info = pd::device_info(dev);
@@ -676,6 +698,8 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     pd::Params P;
     P.q = q; P.k_rep = k_rep; P.v = v; P.membership = membership; P.reps = reps; P.out = out;
     P.seq_lens = seq_lens;
+    P.k_scale = k_scale;
+    P.v_scale = v_scale;
     P.k_batch_bytes = k_batch_stride * elem_size(dtype);
     P.hdr = reinterpret_cast<WsHeader*>(ws);
     P.counters = reinterpret_cast<int*>(ws + L.off_counters);
@@ -698,12 +722,17 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     P.scale = scale;
     if (tiles > L.capK || P.nVi > L.capV || (long long)B * H * P.nVi > 0x7fffffffll) return kDecodeNotLaunched;
     const bool ragged = seq_lens != nullptr || k_batch_stride != (size_t)k * T_cap * D;
-    if (dtype == CHAI_BF16) {
-        if (D == 128) return ragged ? pd::launch<__nv_bfloat16, 128, true>(P, ncta, dev, s) : pd::launch<__nv_bfloat16, 128, false>(P, ncta, dev, s);
-        return ragged ? pd::launch<__nv_bfloat16, 64, true>(P, ncta, dev, s) : pd::launch<__nv_bfloat16, 64, false>(P, ncta, dev, s);
+    using bf16 = __nv_bfloat16;
+    if (dtype == CHAI_FP8_E4M3) {  // fp8 caches, bf16 queries and output
+        if (D == 128) return ragged ? pd::launch<Fp8E4M3, bf16, 128, true>(P, ncta, dev, s) : pd::launch<Fp8E4M3, bf16, 128, false>(P, ncta, dev, s);
+        return ragged ? pd::launch<Fp8E4M3, bf16, 64, true>(P, ncta, dev, s) : pd::launch<Fp8E4M3, bf16, 64, false>(P, ncta, dev, s);
     }
-    if (D == 128) return ragged ? pd::launch<float, 128, true>(P, ncta, dev, s) : pd::launch<float, 128, false>(P, ncta, dev, s);
-    return ragged ? pd::launch<float, 64, true>(P, ncta, dev, s) : pd::launch<float, 64, false>(P, ncta, dev, s);
+    if (dtype == CHAI_BF16) {
+        if (D == 128) return ragged ? pd::launch<bf16, bf16, 128, true>(P, ncta, dev, s) : pd::launch<bf16, bf16, 128, false>(P, ncta, dev, s);
+        return ragged ? pd::launch<bf16, bf16, 64, true>(P, ncta, dev, s) : pd::launch<bf16, bf16, 64, false>(P, ncta, dev, s);
+    }
+    if (D == 128) return ragged ? pd::launch<float, float, 128, true>(P, ncta, dev, s) : pd::launch<float, float, 128, false>(P, ncta, dev, s);
+    return ragged ? pd::launch<float, float, 64, true>(P, ncta, dev, s) : pd::launch<float, float, 64, false>(P, ncta, dev, s);
 }
 
 }  // namespace chai

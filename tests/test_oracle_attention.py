@@ -363,3 +363,27 @@ def test_qkv_variant_member_rows_equal_the_representatives_plain_attention():
             p /= p.sum(axis=1, keepdims=True)
             assert np.allclose(got[b, h], p @ v_rep[b, c], rtol=1e-12, atol=1e-13)
             assert np.array_equal(got[b, h], got[b, r])
+
+
+def test_e4m3_table_and_quantiser():
+    vals = orc.e4m3_values()
+    assert vals[0] == 0.0 and vals[0x38] == 1.0 and vals[0x7E] == 448.0 and vals[0x01] == 2.0 ** -9
+    assert vals[0x08] == 2.0 ** -6 and vals[0x40] == 2.0 and vals[0xB8] == -1.0 and np.isnan(vals[0x7F])
+    finite = vals[:127]
+    assert np.all(np.diff(finite) > 0)                       # bytes 0..126 ascend
+    # a plane whose largest magnitude is 448 has scale 1: representable values map to themselves, midpoints to even
+    x = np.zeros((1, 4, 8), dtype=np.float32)
+    x[0, 0] = [448.0, -1.0, 1.0625, 1.1875, 0.0, 1e-4, -448.0, 17.0]
+    q, s = orc.quantize_cache_fp8(x, 4)
+    assert s.tolist() == [1.0]
+    got = vals[q[0, 0]]
+    # 1.0625 is halfway between 1.0 (mantissa 0) and 1.125 (mantissa 1) -> 1.0; 1.1875 between 1.125 and 1.25 -> 1.25;
+    # 1e-4 is below half the smallest subnormal (2^-10) -> 0; 17 lies halfway between 16 and 18 -> 16 (even mantissa)
+    assert got.tolist() == [448.0, -1.0, 1.0, 1.25, 0.0, 0.0, -448.0, 16.0]
+    # scale: absmax / 448; rows beyond T do not count and stay zero
+    y = np.zeros((2, 3, 2), dtype=np.float32)
+    y[0, :2] = [[2.0, -4.0], [1.0, 0.5]]
+    y[0, 2] = [100.0, 100.0]
+    q, s = orc.quantize_cache_fp8(y, 2)
+    assert s[0] == np.float32(4.0) / np.float32(448.0) and s[1] == 1.0
+    assert np.allclose(vals[q[0, :2]] * s[0], y[0, :2], rtol=2 ** -4) and not q[0, 2].any() and not q[1].any()
