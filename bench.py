@@ -415,6 +415,8 @@ def main():
     ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4])
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers (not a bench result)")
     ap.add_argument("--skip-extras", action="store_true", help="only the decode step (no prefill/compaction/CPU legs)")
+    ap.add_argument("--only", default="", choices=["", "prefill", "compaction", "serving", "fp8"],
+                    help="profiling aid: run just this leg and print its object (not the bench line)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -439,6 +441,11 @@ def main():
         torch.cuda.synchronize()
 
     peaks = load_peaks()
+    if args.only:
+        leg = {"prefill": bench_prefill, "compaction": bench_compaction, "serving": bench_serving, "fp8": bench_fp8}[args.only]
+        print(json.dumps({"leg": args.only, "result": leg(device, peaks)}))
+        ranks.close()
+        return
     wl = DecodeWorkload(args.workload, device, layers=args.layers)
     w = wl.w
     for _ in range(args.warmup):
