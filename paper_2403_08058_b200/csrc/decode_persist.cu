@@ -483,11 +483,15 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
         TQ* outp = static_cast<TQ*>(P.out);
         for (int n = n_issued + ((warp - n_issued) % W + W) % W;; n += W) {  // this warp's next position
             const int slot = n % STAGES;
-            if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag) &&
-                                                     mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
+            // The tile's description is in place as soon as the slot's tag says so, before its bytes have
+            // arrived: the probabilities of the tile (scores and maxima from L2, exponentials) are formed while
+            // the bulk copy is still in flight, and the barrier is only waited for when the bytes are needed.
+            if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag));
             if (!ok) break;
+            __threadfence_block();  // the description was written before the tag: read it after the tag
             const TileMeta m = sm.meta[slot];
             if (m.item < 0) {  // end marker
+                ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
                 __syncwarp();
                 if (lane == 0) mbar_arrive(ring.empty(slot));
                 break;
@@ -502,6 +506,8 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
 #pragma unroll
             for (int e = 0; e < G::EPV; ++e) acc[e] = 0.f;
             float lsum = 0.f;
+            float pv[G::PV];
+            bool have_p = false;
             if (live) {
                 const size_t plane = (size_t)b * k + c;
                 // all scores of the plane must exist; once seen, remembered per CTA (planes complete in order, so
@@ -516,7 +522,6 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                     float mx = -INFINITY;
                     for (int x = lane, nx = tiles_of(b); x < nx; x += 32) mx = fmaxf(mx, __ldcg(&P.cmax[plane * tp + x]));
                     const float* srow = P.scores + plane * T_len + (size_t)tile * G::TR;
-                    float pv[G::PV];
 #pragma unroll
                     for (int u = 0; u < G::PV; ++u) {
                         const int r = u * 32 + lane;
@@ -529,6 +534,18 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                         pv[u] = pv[u] == -INFINITY ? 0.f : expf(pv[u] - mx);
                         lsum += pv[u];
                     }
+                    have_p = true;
+                }
+            } else if (chunk == 0 && m.t == 0) {
+                // unresolved head: zero output, flagged after the status reset (ordered by the layer's first flag)
+                ok = flags_wait(P.flags, 1, P.token, lane, abort_flag);
+                if (ok && lane == 0) flag_bad_membership(P.hdr, b, h);
+                for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<TQ>(0.f);
+            }
+            // now the tile's bytes
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
+            if (ok && have_p) {
+                {
                     const unsigned char* data = sm.ring[slot];
                     if (rows == G::TR) {
 #pragma unroll
@@ -563,11 +580,6 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                         }
                     }
                 }
-            } else if (chunk == 0 && m.t == 0) {
-                // unresolved head: zero output, flagged after the status reset (ordered by the layer's first flag)
-                ok = flags_wait(P.flags, 1, P.token, lane, abort_flag);
-                if (ok && lane == 0) flag_bad_membership(P.hdr, b, h);
-                for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<TQ>(0.f);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(ring.empty(slot));  // the tile's bytes are no longer needed
