@@ -72,6 +72,7 @@ struct Smem {
     int table[TABLE_CAP];
     unsigned ready[TABLE_CAP / 32];  // bit p: every key tile of plane p is known to carry this launch's token
     int abort_flag;
+    int next_pos;               // next ring position a consumer warp may take
 };
 
 struct Params {
@@ -255,6 +256,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
         }
         for (int i = 0; i < TABLE_CAP / 32; ++i) sm.ready[i] = 0;
         sm.abort_flag = 0;
+        sm.next_pos = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -325,9 +327,9 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             {
                 int plane = cta / tp, tile = cta % tp;
                 const int dplane = ncta / tp, dtile = ncta % tp;
-                const TileMeta m{0, 0, 0, 0};
                 constexpr bool plain = !RAGGED;
                 for (int t = 0; t < nkt && ok; ++t) {
+                    const TileMeta m{(int)(cta + (long long)t * ncta), -1, 0, 0};  // key tile: global tile id, t = -1
                     if constexpr (plain) {  // equal lengths, dense cache: no per-tile division on this (single) thread
                         ok = issue(kc + ((size_t)plane * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
                                    (uint32_t)tile_rows(0, tile) * G::ROW_BYTES, m);
@@ -378,21 +380,33 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
         // ------------------------------ consumers: every warp works alone ------------------------------
         const int sub = lane / G::LPR, part = lane % G::LPR;
         bool ok = true;
-        // this warp owns ring positions warp, warp + W, ...; the key tiles of this CTA take positions in the
-        // order of their ids, those beyond their request's length take none
-        constexpr bool ragged = RAGGED;
-        int n_issued = ragged ? 0 : nkt;
-        // ---- phase K: one tile = TR scores and their maximum ----
-        for (int t_idx = ragged ? 0 : warp; t_idx < nkt; t_idx += ragged ? 1 : W) {
-            const long long g = (long long)cta + (long long)t_idx * ncta;
+        // Ring positions are taken in order by whichever warp is free (a warp that is held up -- an item or head
+        // to combine, a ticket to fetch -- does not keep a filled slot waiting).  What a position holds is in
+        // its description: a key tile (t < 0, item = global tile id), a value tile, or an end marker.
+        TQ* outp = static_cast<TQ*>(P.out);
+        for (;;) {
+            int n = 0;
+            if (lane == 0) n = atomicAdd(&sm.next_pos, 1);
+            n = __shfl_sync(0xffffffffu, n, 0);
+            const int slot = n % STAGES;
+            // The description is in place as soon as the slot's tag says so, before the tile's bytes have
+            // arrived: whatever does not need the bytes (the query row of a key tile; scores, maxima and the
+            // probabilities of a value tile) is fetched and formed while the bulk copy is still in flight.
+            if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag));
+            if (!ok) break;
+            __threadfence_block();  // the description was written before the tag: read it after the tag
+            const TileMeta m = sm.meta[slot];
+            if (m.item < 0) {  // end marker
+                ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(ring.empty(slot));
+                break;
+            }
+          if (m.t < 0) {
+            // ---- key tile: TR scores and their maximum ----
+            const long long g = m.item;
             const int plane = (int)(g / tp), tile = (int)(g % tp);
             const int b = plane / k;
-            int n = t_idx;  // ring position of this tile
-            if constexpr (ragged) {
-                if (tile >= tiles_of(b)) continue;
-                if ((n_issued++ % W) != warp) continue;
-                n = n_issued - 1;
-            }
             const int rows = tile_rows(b, tile);
             const int rep = P.reps[plane];
             const bool live = rep >= 0 && rep < H;  // unused cluster slot: the tile is drained, nothing computed
@@ -407,9 +421,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                     Vec16<TQ>::unpack(*reinterpret_cast<const uint4*>(qsrc + x * Vec16<TQ>::N), qf + x * Vec16<TQ>::N);
             }
             const float kscale = P.k_scale ? P.scale * __ldg(P.k_scale + plane) : P.scale;  // fp8 keys carry a scale per plane
-            const int slot = n % STAGES;
-            if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag) &&
-                                                     mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
+            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
             if (ok && live && rows == 0) {  // tile beyond this request's length: no scores, neutral maximum
                 if (lane == 0) P.cmax[(size_t)plane * tp + tile] = -INFINITY;
             } else if (ok && live) {
@@ -478,24 +490,10 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 if (lane == 0)
                     asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(P.flags + (size_t)plane * tp + tile), "l"(P.token) : "memory");
             }
-        }
-        // ---- phase V: tiles of claimed items ----
-        TQ* outp = static_cast<TQ*>(P.out);
-        for (int n = n_issued + ((warp - n_issued) % W + W) % W;; n += W) {  // this warp's next position
-            const int slot = n % STAGES;
-            // The tile's description is in place as soon as the slot's tag says so, before its bytes have
-            // arrived: the probabilities of the tile (scores and maxima from L2, exponentials) are formed while
-            // the bulk copy is still in flight, and the barrier is only waited for when the bytes are needed.
-            if (ok) ok = __all_sync(0xffffffffu, word_wait(&sm.seq[slot], n, abort_flag));
             if (!ok) break;
-            __threadfence_block();  // the description was written before the tag: read it after the tag
-            const TileMeta m = sm.meta[slot];
-            if (m.item < 0) {  // end marker
-                ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
-                __syncwarp();
-                if (lane == 0) mbar_arrive(ring.empty(slot));
-                break;
-            }
+            continue;
+          }
+            // ---- value tile of a claimed item ----
             const int head = m.item / P.nVi, chunk = m.item % P.nVi;
             const int b = head / H, h = head % H;
             const int tile = chunk * P.IV + m.t;
@@ -732,7 +730,9 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     P.IV = tiles < pd::MAX_IV ? tiles : pd::MAX_IV;
     P.nVi = (tiles + P.IV - 1) / P.IV;
     P.scale = scale;
-    if (tiles > L.capK || P.nVi > L.capV || (long long)B * H * P.nVi > 0x7fffffffll) return kDecodeNotLaunched;
+    if (tiles > L.capK || P.nVi > L.capV || (long long)B * H * P.nVi > 0x7fffffffll ||
+        (long long)B * k * tiles > 0x7fffffffll)  // item and key-tile ids travel as ints
+        return kDecodeNotLaunched;
     const bool ragged = seq_lens != nullptr || k_batch_stride != (size_t)k * T_cap * D;
     using bf16 = __nv_bfloat16;
     if (dtype == CHAI_FP8_E4M3) {  // fp8 caches, bf16 queries and output
