@@ -1,10 +1,11 @@
 // Clustered decode attention, persistent streaming kernel (Fig. 3(b), Section 3.4).
 //
-// One CTA per SM (cooperative launch, for co-residency only).  Warp 8 is the producer: it streams cache
-// rows, 32 KB tile by tile, into a shared-memory ring with bulk async copies that complete on
-// mbarriers, and runs ahead of the consumers by the depth of the ring, so HBM stays busy while a
-// consumer does the serial part of a tile.  Warps 0..7 consume, each on its own: ring position n
-// belongs to warp n mod 8, nothing is synchronised across the warps of a CTA except item completion.
+// One CTA per SM (cooperative launch, for co-residency only).  The last warp is the producer: it streams
+// cache rows, tile by tile, into a shared-memory ring with bulk async copies that complete on mbarriers, and
+// runs ahead of the consumers by the depth of the ring, so HBM stays busy while a consumer does the serial
+// part of a tile.  The other warps consume, each on its own: a free warp takes the next ring position (an
+// atomic counter in shared memory), reads what the position holds from the slot's description and works on
+// it; nothing else is synchronised across the warps of a CTA except item completion.
 //
 //   phase K   unit = one key tile (TR rows of one cluster's K_rep), dealt round-robin over CTAs: scaled
 //             scores s_t -> workspace (fp32, stays in L2), the tile's maximum, then the tile's flag word
