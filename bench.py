@@ -415,6 +415,7 @@ def main():
     ap.add_argument("--workload", type=int, default=2, choices=[2, 3, 4])
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers (not a bench result)")
     ap.add_argument("--skip-extras", action="store_true", help="only the decode step (no prefill/compaction/CPU legs)")
+    ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a replayed CUDA graph")
     ap.add_argument("--only", default="", choices=["", "prefill", "compaction", "serving", "fp8"],
                     help="profiling aid: run just this leg and print its object (not the bench line)")
     args = ap.parse_args()
@@ -450,9 +451,28 @@ def main():
     w = wl.w
     for _ in range(args.warmup):
         wl.step()
+    # The decode step is launch-bound between its 32..64 layer calls, so it is captured once into a CUDA graph
+    # and replayed (what a serving loop does); the eager launch loop is timed as well and reported beside it.
+    graph = None
+    if not args.no_graph:
+        try:
+            torch.cuda.synchronize()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                wl.step()
+            torch.cuda.current_stream().wait_stream(side)
+            for _ in range(args.warmup):
+                graph.replay()
+        except Exception as e:  # capture not possible here: time the eager loop only
+            print(f"bench.py: CUDA graph capture failed ({e!r}); timing eager launches", file=sys.stderr)
+            graph = None
+    timed_step = graph.replay if graph is not None else wl.step
     # 1) device-resident timing: exactly K steps, two events
     with ClockSampler(local_rank) as clk:
-        ms_total = time_region(wl.step, args.steps, sync_all)
+        ms_total = time_region(timed_step, args.steps, sync_all)
+        ms_eager = time_region(wl.step, args.steps, sync_all) if graph is not None else ms_total
         # 2) same K steps again with an event after every layer call: per-launch durations for the roofline
         events = [[torch.cuda.Event(enable_timing=True) for _ in range(w.layers + 1)] for _ in range(args.steps)]
         sync_all()
@@ -466,14 +486,16 @@ def main():
         wl.step_host()
     ms_e2e = time_region(wl.step_host, args.steps, sync_all)
 
-    ms_total, ms_e2e = ranks.max_over_ranks([ms_total, ms_e2e])
+    ms_total, ms_e2e, ms_eager = ranks.max_over_ranks([ms_total, ms_e2e, ms_eager])
     ms_step = ms_total / args.steps
     value = replicas.whole_job_throughput(ranks, wl.bytes_per_step / 1e9, ms_step * 1e-3)["value"]
     e2e_value = replicas.whole_job_throughput(ranks, wl.bytes_per_step / 1e9, ms_e2e / args.steps * 1e-3)["value"]
 
     if rank == 0:
-        per_launch_ms = float(layer_ms.mean())
+        # average launch duration over the timed region itself (K steps x layers launches, gaps included)
+        per_launch_ms = ms_step / w.layers
         achieved = float(np.mean(wl.bytes_per_layer)) / (per_launch_ms * 1e-3) / 1e9
+        eager_value = wl.bytes_per_step / 1e9 / (ms_eager / args.steps * 1e-3) * world
         by_k = {}
         for c, col in zip(wl.layers, layer_ms.T):
             by_k.setdefault(c["k"], []).append(float(np.median(col)) * 1e3)
@@ -485,7 +507,10 @@ def main():
                        "k_per_layer": [c["k"] for c in wl.layers], "partition": w.partition,
                        "algorithmic_gb_per_step": wl.bytes_per_step / 1e9,
                        "l2": "inputs larger than L2: every layer has its own >=168 MiB caches, 12+ GB per step",
+                       "launch": ("one CUDA graph of the step's layer calls, replayed" if graph is not None else "eager launches"),
                        "multi_gpu": "independent replicas, no data-path collective"},
+            "eager": {"value": eager_value, "unit": UNIT, "ms_per_step": ms_eager / args.steps,
+                      "note": "the same K steps launched call by call from the host"},
             "gpu_launches": wl.launches_per_step * args.steps,
             "roofline": {"bound": "hbm", "kernel": "decode_persistent_kernel (one launch per layer call)",
                          "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
@@ -494,6 +519,7 @@ def main():
                          # layers (profiles/decode_persistent_kernel_workload2.md), scaled to the mean launch here
                          "traffic": 1.02 * float(np.mean(wl.bytes_per_layer)), "traffic_unit": "bytes per launch",
                          "us_per_layer_by_k": {str(k): statistics.median(v) for k, v in sorted(by_k.items())},
+                         "us_per_layer_by_k_note": "eager launches with an event after every layer call",
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "e2e": {"value": e2e_value, "unit": UNIT, "us_per_step": ms_e2e / args.steps * 1e3,
                     "h2d_bytes_per_step": w.layers * w.B * w.H * w.D * wl.es,

@@ -74,6 +74,7 @@ struct Smem {
     unsigned ready[TABLE_CAP / 32];  // bit p: every key tile of plane p is known to carry this launch's token
     int abort_flag;
     int next_pos;               // next ring position a consumer warp may take
+    unsigned epoch;             // launch count of this workspace, read once at start
 };
 
 struct Params {
@@ -244,6 +245,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
     const int nkt = n_ktiles > cta ? (int)((n_ktiles - cta + ncta - 1) / ncta) : 0;  // this CTA's share
     const int n_items = B * H * P.nVi;                   // value items of the layer
     int* work_counter = &P.hdr->pad[0];
+    int* launch_epoch = &P.hdr->pad[8];
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -258,6 +260,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
         for (int i = 0; i < TABLE_CAP / 32; ++i) sm.ready[i] = 0;
         sm.abort_flag = 0;
         sm.next_pos = 0;
+        sm.epoch = *reinterpret_cast<volatile unsigned*>(&P.hdr->pad[8]);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -268,6 +271,11 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
         }
     }
     __syncthreads();
+    // Token of this launch: the workspace's launch count (bumped once per launch, below) in the high word, a
+    // host-side value in the low word.  It differs from the token of every earlier launch on this workspace --
+    // also when the launch is a replay of a captured graph, whose kernel arguments never change -- so flag
+    // words left by earlier launches cannot look ready.
+    const unsigned long long token = ((unsigned long long)sm.epoch << 32) | (P.token & 0xffffffffull);
     auto cluster_of = [&](int b, int h) -> int {
         if (use_table) return sm.table[b * H + h];
         int c, r;
@@ -350,7 +358,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             }
             // ---- value items, claimed one at a time; the next claim is in flight while this item streams ----
             // (the work counter is reset by the owner of the layer's first key tile before that tile's flag)
-            if (ok) ok = flag_wait_one(P.flags, P.token, abort_flag);
+            if (ok) ok = flag_wait_one(P.flags, token, abort_flag);
             int n_open = 0;  // items this CTA has opened (item slots are handed out round-robin)
             int next = ok ? atomicAdd(work_counter, 1) : n_items;
             while (ok && next < n_items) {
@@ -373,6 +381,9 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                                (uint32_t)tile_rows(b_item, tile) * G::ROW_BYTES, m);
                 }
             }
+            // The claim that comes back with the largest id is the last one of the launch: every CTA has started
+            // (and read the launch count) by then, so the count can move on for the next launch.
+            if (ok && next == n_items + ncta - 1) atomicAdd(launch_epoch, 1);
             // ---- one end marker per consumer warp ----
             const TileMeta end{-1, 0, 0, 0};
             for (int w = 0; w < W && ok; ++w) ok = issue(nullptr, 0, end);
@@ -489,7 +500,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 }
                 __syncwarp();
                 if (lane == 0)
-                    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(P.flags + (size_t)plane * tp + tile), "l"(P.token) : "memory");
+                    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(P.flags + (size_t)plane * tp + tile), "l"(token) : "memory");
             }
             if (!ok) break;
             continue;
@@ -513,7 +524,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 // after the first tiles of phase V this is a shared-memory bit test)
                 const bool cached = plane < TABLE_CAP && ((*reinterpret_cast<volatile unsigned*>(&sm.ready[plane >> 5]) >> (plane & 31)) & 1u);
                 if (!cached) {
-                    ok = flags_wait(P.flags + plane * tp, tiles_of(b), P.token, lane, abort_flag);
+                    ok = flags_wait(P.flags + plane * tp, tiles_of(b), token, lane, abort_flag);
                     if (ok && lane == 0 && plane < TABLE_CAP) atomicOr(&sm.ready[plane >> 5], 1u << (plane & 31));
                 }
                 if (ok && rows > 0) {  // (the only tile of an empty request has no rows: it just passes the ticket on,
@@ -537,7 +548,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 }
             } else if (chunk == 0 && m.t == 0) {
                 // unresolved head: zero output, flagged after the status reset (ordered by the layer's first flag)
-                ok = flags_wait(P.flags, 1, P.token, lane, abort_flag);
+                ok = flags_wait(P.flags, 1, token, lane, abort_flag);
                 if (ok && lane == 0) flag_bad_membership(P.hdr, b, h);
                 for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<TQ>(0.f);
             }
