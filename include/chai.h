@@ -198,6 +198,19 @@ int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage
                                int dtype, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * As chai_decode_attention_host, but the call only enqueues upload, kernels and download on `stream` and
+ * returns: out_host is valid once the caller has synchronised the stream (or an event recorded after the call).
+ * q_host must stay unchanged and out_host untouched until then; with pageable instead of pinned host memory the
+ * copies fall back to synchronous staging by the CUDA runtime.  Successive calls on one stream may share q_stage
+ * and out_stage (stream order keeps them apart), so a whole decode step of layer calls needs one
+ * synchronisation, not one per layer.
+ */
+int chai_decode_attention_host_async(const void* q_host, void* out_host, void* q_stage, void* out_stage,
+                                     const void* k_rep, const void* v, const int32_t* membership,
+                                     const int32_t* reps, int B, int H, int k, int T, int T_cap, int D, float scale,
+                                     int dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Decode step for callers that can neither pass a workspace nor let the library allocate one
  * (no counterpart in the paper: this is a deployment convenience).  Typical cases: a serving
  * engine that has already handed every free byte of HBM to its KV-cache pool, so a later

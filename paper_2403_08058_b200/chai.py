@@ -22,7 +22,7 @@ CHAI_F32, CHAI_BF16 = 0, 1
 # every symbol include/chai.h declares
 EXPORTS = [
     "chai_prefix_features", "chai_cluster_heads", "chai_compact_k_cache", "chai_decode_attention",
-    "chai_decode_workspace_bytes", "chai_decode_attention_host", "chai_prefill_attention",
+    "chai_decode_workspace_bytes", "chai_decode_attention_host", "chai_decode_attention_host_async", "chai_prefill_attention",
     "chai_prefill_attention_simt", "chai_prefill_workspace_bytes", "chai_device_status",
     "chai_status_string", "chai_last_error", "chai_version", "chai_decode_attention_static",
     "chai_decode_attention_ragged", "chai_append_kv", "chai_compact_k_cache_inplace",
@@ -56,8 +56,8 @@ def load() -> ctypes.CDLL:
     lib.chai_cluster_heads.argtypes = [vp, ci, ci, ci, ci, ci, ctypes.c_uint64, vp, vp, vp, vp, vp]
     lib.chai_compact_k_cache.argtypes = [vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp]
     lib.chai_decode_attention.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp, sz, vp]
-    lib.chai_decode_attention_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci,
-                                               vp, sz, vp]
+    for name in ("chai_decode_attention_host", "chai_decode_attention_host_async"):
+        getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp, sz, vp]
     for name in ("chai_prefill_attention", "chai_prefill_attention_simt"):
         getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
     lib.chai_decode_attention_qkv.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp, sz, vp]
@@ -276,18 +276,29 @@ def chai_compact_k_cache_inplace(k_cache, reps, T: int | None = None, workspace=
     return k_cache
 
 
-def chai_decode_attention_host(q_host, out_host, q_stage, out_stage, k_rep, v, membership, reps, scale: float,
-                               workspace, T: int | None = None):
-    """Decode step with q / out in (pinned) host memory; returns after the stream has drained."""
+def _decode_host(fn_name, q_host, out_host, q_stage, out_stage, k_rep, v, membership, reps, scale, workspace, T):
     _dev(q_stage, out_stage, k_rep, v, membership, reps, workspace)
     B, H, D = q_host.shape
     k, T_cap = k_rep.shape[1], k_rep.shape[2]
     T = T_cap if T is None else T
-    _check(load().chai_decode_attention_host(q_host.data_ptr(), out_host.data_ptr(), _ptr(q_stage),
-                                             _ptr(out_stage), _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps),
-                                             B, H, k, T, T_cap, D, scale, _dt(q_host), _ptr(workspace),
-                                             workspace.numel(), _stream()))
+    _check(getattr(load(), fn_name)(q_host.data_ptr(), out_host.data_ptr(), _ptr(q_stage), _ptr(out_stage),
+                                    _ptr(k_rep), _ptr(v), _ptr(membership), _ptr(reps), B, H, k, T, T_cap, D, scale,
+                                    _dt(q_host), _ptr(workspace), workspace.numel(), _stream()))
     return out_host
+
+
+def chai_decode_attention_host(q_host, out_host, q_stage, out_stage, k_rep, v, membership, reps, scale: float,
+                               workspace, T: int | None = None):
+    """Decode step with q / out in (pinned) host memory; returns after the stream has drained."""
+    return _decode_host("chai_decode_attention_host", q_host, out_host, q_stage, out_stage, k_rep, v, membership,
+                        reps, scale, workspace, T)
+
+
+def chai_decode_attention_host_async(q_host, out_host, q_stage, out_stage, k_rep, v, membership, reps, scale: float,
+                                     workspace, T: int | None = None):
+    """As above but only enqueued on the current stream: out_host is valid after the caller synchronises it."""
+    return _decode_host("chai_decode_attention_host_async", q_host, out_host, q_stage, out_stage, k_rep, v,
+                        membership, reps, scale, workspace, T)
 
 
 def _prefill(fn_name, q, k_rep, v, membership, reps, scale, causal, out, workspace):

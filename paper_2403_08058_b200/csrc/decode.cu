@@ -318,26 +318,36 @@ int chai_decode_attention_ragged(const void* q, const void* k_rep, const void* v
                        T_cap, D, k_batch_stride, scale, dtype, workspace, workspace_bytes, stream);
 }
 
-int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage, void* out_stage, const void* k_rep,
-                               const void* v, const int32_t* membership, const int32_t* reps, int B, int H, int k,
-                               int T, int T_cap, int D, float scale, int dtype, void* workspace,
-                               size_t workspace_bytes, void* stream) {
+int chai_decode_attention_host_async(const void* q_host, void* out_host, void* q_stage, void* out_stage,
+                                     const void* k_rep, const void* v, const int32_t* membership, const int32_t* reps,
+                                     int B, int H, int k, int T, int T_cap, int D, float scale, int dtype,
+                                     void* workspace, size_t workspace_bytes, void* stream) {
     using namespace chai;
-    CHAI_REQUIRE(q_host && out_host && q_stage && out_stage, CHAI_ERR_INVALID_ARG,
-                 "chai_decode_attention_host: null pointer");
+    const char* fn = "chai_decode_attention_host_async";
+    CHAI_REQUIRE(q_host && out_host && q_stage && out_stage, CHAI_ERR_INVALID_ARG, "%s: null pointer", fn);
     CHAI_REQUIRE(B > 0 && H > 0 && D > 0 && (dtype == CHAI_F32 || dtype == CHAI_BF16), CHAI_ERR_INVALID_ARG,
-                 "chai_decode_attention_host: bad sizes or dtype");
+                 "%s: bad sizes or dtype", fn);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t bytes = (size_t)B * H * D * elem_size(dtype);
     cudaError_t e = cudaMemcpyAsync(q_stage, q_host, bytes, cudaMemcpyHostToDevice, s);
-    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_host: query upload");
+    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_host_async: query upload");
     int rc = chai_decode_attention(q_stage, k_rep, v, membership, reps, out_stage, B, H, k, T, T_cap, D, scale, dtype,
                                    workspace, workspace_bytes, stream);
     if (rc != CHAI_OK) return rc;
     e = cudaMemcpyAsync(out_host, out_stage, bytes, cudaMemcpyDeviceToHost, s);
-    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_host: output download");
-    e = cudaStreamSynchronize(s);
-    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_host: synchronize");
+    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_host_async: output download");
+    return CHAI_OK;
+}
+
+int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage, void* out_stage, const void* k_rep,
+                               const void* v, const int32_t* membership, const int32_t* reps, int B, int H, int k,
+                               int T, int T_cap, int D, float scale, int dtype, void* workspace,
+                               size_t workspace_bytes, void* stream) {
+    const int rc = chai_decode_attention_host_async(q_host, out_host, q_stage, out_stage, k_rep, v, membership, reps, B,
+                                                    H, k, T, T_cap, D, scale, dtype, workspace, workspace_bytes, stream);
+    if (rc != CHAI_OK) return rc;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return chai::cuda_fail(e, "chai_decode_attention_host: synchronize");
     return CHAI_OK;
 }
 

@@ -260,10 +260,15 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
         for (int i = 0; i < TABLE_CAP / 32; ++i) sm.ready[i] = 0;
         sm.abort_flag = 0;
         sm.next_pos = 0;
-        sm.epoch = *reinterpret_cast<volatile unsigned*>(&P.hdr->pad[8]);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    // Launched as a programmatic dependent, the kernel gets here while its predecessor in the stream may still
+    // be running: let our own dependents be scheduled, then wait for the predecessor to complete before the
+    // first access to global memory (inputs, workspace, launch count).  Both are no-ops otherwise.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (tid == 0) sm.epoch = *reinterpret_cast<volatile unsigned*>(&P.hdr->pad[8]);
     if (use_table) {
         for (int i = tid; i < B * H; i += THREADS) {
             int c, r;
@@ -697,10 +702,24 @@ static int launch(const Params& P0, int ncta, int dev, cudaStream_t s) {
         if (per_sm < 1) return kDecodeNotLaunched;
         configured = true;
     }
-    void* args[] = {&P};
-    // cooperative launch: value tiles wait for flags set by other CTAs, so all CTAs must be resident at once
-    cudaError_t e = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_persistent_kernel<T, TQ, D, RAGGED>), dim3(ncta),
-                                                dim3(THREADS), args, smem, s);
+    // Cooperative: value tiles wait for flags set by other CTAs, so all CTAs must be resident at once (a plain
+    // launch would let two such kernels on different streams starve each other).  Programmatic stream
+    // serialisation: the kernel may be scheduled while its predecessor in the stream drains and blocks in
+    // griddepcontrol.wait until that predecessor has completed; worth 0.4 % on a replayed graph of layer calls.
+    cudaLaunchAttribute attr[2];
+    const unsigned n_attr = 2;
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(ncta);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cfg.attrs = attr;
+    cfg.numAttrs = n_attr;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, decode_persistent_kernel<T, TQ, D, RAGGED>, P);
     if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel launch");
     return CHAI_OK;
 }

@@ -154,6 +154,14 @@ def test_decode_host_entry_point():
     chai.chai_decode_attention_host(qh, oh, torch.empty_like(d["q"]), torch.empty_like(d["q"]), d["k_rep"], d["v"],
                                     d["membership"], d["reps"], case["scale"], ws)
     assert_parity(oh.float().numpy(), oracle_decode(case), "bf16", "host entry")
+    # the enqueue-only form: two calls share the staging buffers, one synchronisation at the end
+    oh1, oh2 = torch.zeros_like(oh).pin_memory(), torch.zeros_like(oh).pin_memory()
+    qs, os_ = torch.empty_like(d["q"]), torch.empty_like(d["q"])
+    for o in (oh1, oh2):
+        chai.chai_decode_attention_host_async(qh, o, qs, os_, d["k_rep"], d["v"], d["membership"], d["reps"],
+                                              case["scale"], ws)
+    torch.cuda.current_stream().synchronize()
+    assert torch.equal(oh1, oh) and torch.equal(oh2, oh)
 
 
 # ---- k-means, features, compaction ---------------------------------------------------------------------
