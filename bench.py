@@ -431,6 +431,21 @@ def bench_fp8(device, peaks, iters=20, warmup=3):
                         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s",
                                      "frac": gbs / peaks["hbm"], "peak_source": peaks["source"], "traffic": None}}
         del sets
+    # the quantiser on one layer's value cache (read twice: maximum, then conversion; written once in bytes)
+    caches = [synth.decode_layer(2, i, 2, device=device, B=B, H=H, T=T, k=8)["v"] for i in range(4)]
+    for c in caches[:2]:
+        chai.chai_quantize_cache_fp8(c)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for c in caches:
+        q8, sc = chai.chai_quantize_cache_fp8(c)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / len(caches)
+    qbytes = caches[0].numel() * (2 + 2 + 1)
+    res["quantize_v_cache"] = {"us": us, "algorithmic_mb": qbytes / 1e6, "gbs": qbytes / (us * 1e-6) / 1e9,
+                               "note": "includes the binding's zero-fill of the byte buffer"}
     res["workload"] = "config2 layer shape (B 16, H 32, T 2048, D 128), e4m3 caches + per-plane scales, bf16 q/out"
     return res
 

@@ -10,21 +10,48 @@ namespace chai {
 
 constexpr float kE4M3Max = 448.f;  // largest finite e4m3 value
 
-// absmax per plane over rows [0,T): positive floats order like their bit patterns, so an integer atomicMax does it
+// absmax per plane over rows [0,T): positive floats order like their bit patterns, so an integer atomicMax does it.
+// VEC: 16-byte loads of 8 elements (the host checks alignment and that the row count allows it).
+template <bool VEC>
 __global__ void __launch_bounds__(256)
 fp8_absmax_kernel(const __nv_bfloat16* __restrict__ src, int* __restrict__ absmax_bits, int T, int T_cap, int D) {
     const int plane = blockIdx.y;
     const size_t n = (size_t)T * D;
     const __nv_bfloat16* p = src + (size_t)plane * T_cap * D;
+    const size_t first = (size_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
     float m = 0.f;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
-        m = fmaxf(m, fabsf(__bfloat162float(p[i])));
+    if constexpr (VEC) {
+        const uint4* p4 = reinterpret_cast<const uint4*>(p);
+        const size_t n4 = n / 8;
+        for (size_t i = first; i < n4; i += 4 * stride) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i + u * stride < n4) v[u] = __ldg(p4 + i + u * stride); else v[u] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    m = fmaxf(m, fabsf(__uint_as_float(w[e] << 16)));
+                    m = fmaxf(m, fabsf(__uint_as_float(w[e] & 0xffff0000u)));
+                }
+            }
+        }
+    } else {
+        for (size_t i = first; i < n; i += stride) m = fmaxf(m, fabsf(__bfloat162float(p[i])));
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     if ((threadIdx.x & 31) == 0 && m > 0.f) atomicMax(absmax_bits + plane, __float_as_int(m));
 }
 
+__device__ __forceinline__ unsigned quant1(float x, float scale) {
+    return (unsigned)__nv_cvt_float_to_fp8(__fdiv_rn(x, scale), __NV_SATFINITE, __NV_E4M3);
+}
+
 // q = round-to-nearest-even e4m3 of (x / scale), scale = absmax / 448 in fp32 (1 for an all-zero plane)
+template <bool VEC>
 __global__ void __launch_bounds__(256)
 fp8_quantize_kernel(const __nv_bfloat16* __restrict__ src, unsigned char* __restrict__ dst,
                     const int* __restrict__ absmax_bits, int T, int T_cap, int D) {
@@ -34,8 +61,35 @@ fp8_quantize_kernel(const __nv_bfloat16* __restrict__ src, unsigned char* __rest
     const size_t n = (size_t)T * D;
     const __nv_bfloat16* p = src + (size_t)plane * T_cap * D;
     unsigned char* q = dst + (size_t)plane * T_cap * D;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
-        q[i] = (unsigned char)__nv_cvt_float_to_fp8(__fdiv_rn(__bfloat162float(p[i]), scale), __NV_SATFINITE, __NV_E4M3);
+    const size_t first = (size_t)blockIdx.x * blockDim.x + threadIdx.x, stride = (size_t)gridDim.x * blockDim.x;
+    if constexpr (VEC) {
+        const uint4* p4 = reinterpret_cast<const uint4*>(p);
+        uint2* q2 = reinterpret_cast<uint2*>(q);
+        const size_t n4 = n / 8;
+        for (size_t i = first; i < n4; i += 4 * stride) {
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (i + u * stride < n4) v[u] = __ldg(p4 + i + u * stride);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (i + u * stride >= n4) break;
+                const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                unsigned b[8];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    b[2 * e] = quant1(__uint_as_float(w[e] << 16), scale);
+                    b[2 * e + 1] = quant1(__uint_as_float(w[e] & 0xffff0000u), scale);
+                }
+                uint2 o;
+                o.x = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+                o.y = b[4] | (b[5] << 8) | (b[6] << 16) | (b[7] << 24);
+                q2[i + u * stride] = o;
+            }
+        }
+    } else {
+        for (size_t i = first; i < n; i += stride) q[i] = (unsigned char)quant1(__bfloat162float(p[i]), scale);
+    }
 }
 
 __global__ void fp8_scales_kernel(int* __restrict__ absmax_bits_to_scale, int n) {
@@ -59,14 +113,21 @@ int chai_quantize_cache_fp8(const void* src, void* dst, float* scales, int n_pla
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemsetAsync(scales, 0, sizeof(float) * (size_t)n_planes, s);
     if (e != cudaSuccess) return cuda_fail(e, "chai_quantize_cache_fp8: clearing the scales");
+    // 16-byte loads need every plane to start on a 16-byte boundary and hold a multiple of 8 elements
+    const bool vec = ((size_t)T * D) % 8 == 0 && ((size_t)T_cap * D) % 16 == 0 && aligned16(src) && aligned16(dst);
     const size_t n = (size_t)T * D;
-    unsigned chunks = (unsigned)((n + 256 * 16 - 1) / (256 * 16));
+    const size_t per_cta = vec ? 256 * 8 * 4 : 256 * 16;
+    unsigned chunks = (unsigned)((n + per_cta - 1) / per_cta);
     chunks = chunks < 1 ? 1 : (chunks > 64 ? 64 : chunks);
     int* bits = reinterpret_cast<int*>(scales);
-    fp8_absmax_kernel<<<dim3(chunks, n_planes), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(src), bits, T, T_cap, D);
+    const dim3 grid(chunks, n_planes);
+    const __nv_bfloat16* sp = static_cast<const __nv_bfloat16*>(src);
+    unsigned char* dp = static_cast<unsigned char*>(dst);
+    if (vec) fp8_absmax_kernel<true><<<grid, 256, 0, s>>>(sp, bits, T, T_cap, D);
+    else fp8_absmax_kernel<false><<<grid, 256, 0, s>>>(sp, bits, T, T_cap, D);
     CHAI_LAUNCH_CHECK("fp8_absmax_kernel launch");
-    fp8_quantize_kernel<<<dim3(chunks, n_planes), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(src),
-                                                              static_cast<unsigned char*>(dst), bits, T, T_cap, D);
+    if (vec) fp8_quantize_kernel<true><<<grid, 256, 0, s>>>(sp, dp, bits, T, T_cap, D);
+    else fp8_quantize_kernel<false><<<grid, 256, 0, s>>>(sp, dp, bits, T, T_cap, D);
     CHAI_LAUNCH_CHECK("fp8_quantize_kernel launch");
     fp8_scales_kernel<<<(n_planes + 255) / 256, 256, 0, s>>>(bits, n_planes);
     CHAI_LAUNCH_CHECK("fp8_scales_kernel launch");

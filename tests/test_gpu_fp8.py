@@ -21,10 +21,11 @@ def case_for(seed, B, H, k, T_cap, D=128):
     return c
 
 
-@pytest.mark.parametrize("T,T_cap", [(300, 300), (100, 256), (1, 8)])
-def test_quantiser_bit_exact(T, T_cap):
+# D = 128: 16-byte vector path; D = 12 with odd sizes: element-wise path; (2100, 2100): more than one pass per thread
+@pytest.mark.parametrize("T,T_cap,D", [(300, 300, 128), (100, 256, 128), (1, 8, 128), (2100, 2100, 128), (33, 35, 12)])
+def test_quantiser_bit_exact(T, T_cap, D):
     g = torch.Generator().manual_seed(T)
-    x = (torch.randn(2, 5, T_cap, 128, generator=g) * torch.tensor([0.01, 0.5, 1.0, 30.0, 0.0])[None, :, None, None])
+    x = (torch.randn(2, 5, T_cap, D, generator=g) * torch.tensor([0.01, 0.5, 1.0, 30.0, 0.0])[None, :, None, None])
     x = x.to(torch.bfloat16)
     x[0, 1, 0, :8] = torch.tensor([1.0625, 1.1875, 17.0, -17.0, 2.0 ** -12, 0.0, -0.0, 3.0]).to(torch.bfloat16)
     q8, scales = chai.chai_quantize_cache_fp8(x.to(DEV), T)
