@@ -59,6 +59,9 @@ prefill_plan_kernel(const int32_t* __restrict__ membership, const int32_t* __res
     // a kernel launched as a programmatic dependent may start its own set-up now; it still waits for this
     // grid to finish (griddepcontrol.wait) before it reads anything written here
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // launched as a programmatic dependent itself, the planner may be here while its predecessor still runs
+    // (and still uses the workspace): wait for it before the first access to global memory
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (b == 0)
         for (int i = tid; i < 60; i += nt) hdr->pad[i] = 0;
     for (int h = tid; h < H; h += nt) mem[h] = membership[(size_t)b * H + h];

@@ -164,7 +164,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // Everything above is independent of the planning kernel, which may still be running (the launch is
-    // programmatically dependent); its results are read only after this point.
+    // programmatically dependent); its results are read only after this point.  Our own dependents (the
+    // planner of a following prefill call) may be placed as soon as SMs free up; they wait for this grid's end.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 0) {
         if (blockIdx.x == 0 && counter_slot == 0) publish_plan_status(hdr, bad, B_total);
