@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
                                                      int max_iter, unsigned long long seed,
                                                      int32_t* __restrict__ membership, int32_t* __restrict__ reps,
                                                      int32_t* __restrict__ k_eff, double* __restrict__ inertia) {
+    dependent_grid_sync();
     const bool sweep = k_arg == 0;
     const int k = sweep ? (int)blockIdx.y + 1 : k_arg;
     if (sweep) inertia += (size_t)blockIdx.x * gridDim.y + blockIdx.y - blockIdx.x;  // so that inertia[b] below is the curve entry
@@ -68,7 +69,7 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
     int* prev = a + H;
     int* count = prev + H;
     int* newid = count + k;
-    __shared__ int s_far, s_ncentres, s_same;
+    __shared__ int s_ncentres, s_same;
 
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const float* xin = features + (size_t)b * H * F;
@@ -83,25 +84,40 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
     double* dmin = dist;
     for (int h = tid; h < H; h += nt) dmin[h] = sqdist(X + (size_t)h * F, C, F);
     __syncthreads();
-    for (int n = 1; n < k; ++n) {
-        if (tid == 0) {
-            int far = 0;
-            for (int h = 1; h < H; ++h)
-                if (dmin[h] > dmin[far]) far = h;
-            s_far = dmin[far] == 0.0 ? -1 : far;
+    // The traversal is a chain of k - 1 dependent steps (farthest head, then every head's distance to it), so
+    // one warp walks it without block-wide barriers: lane l owns heads l, l + 32, ... and their dmin entries.
+    if (tid < 32) {
+        const int lane = tid;
+        int ncent = 1;
+        for (int n = 1; n < k; ++n) {
+            double bd = -1.0;  // farthest head so far: largest dmin, lowest index on ties
+            int bh = 0x7fffffff;
+            for (int h = lane; h < H; h += 32) {
+                const double d = dmin[h];
+                if (d > bd) {
+                    bd = d;
+                    bh = h;
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const double od = __shfl_xor_sync(0xffffffffu, bd, o);
+                const int oh = __shfl_xor_sync(0xffffffffu, bh, o);
+                if (od > bd || (od == bd && oh < bh)) {
+                    bd = od;
+                    bh = oh;
+                }
+            }
+            if (bd == 0.0) break;  // fewer than k distinct points (warp-uniform)
+            const double* xf = X + (size_t)bh * F;
+            for (int f = lane; f < F; f += 32) C[(size_t)n * F + f] = xf[f];
+            for (int h = lane; h < H; h += 32) {
+                const double d = sqdist(X + (size_t)h * F, xf, F);
+                if (d < dmin[h]) dmin[h] = d;
+            }
+            ncent = n + 1;
         }
-        __syncthreads();
-        const int far = s_far;
-        if (far < 0) break;  // uniform: every thread reads the same shared value
-        double* cn = C + (size_t)n * F;
-        for (int f = tid; f < F; f += nt) cn[f] = X[(size_t)far * F + f];
-        if (tid == 0) s_ncentres = n + 1;
-        __syncthreads();
-        for (int h = tid; h < H; h += nt) {
-            double d = sqdist(X + (size_t)h * F, cn, F);
-            if (d < dmin[h]) dmin[h] = d;
-        }
-        __syncthreads();
+        if (lane == 0) s_ncentres = ncent;
     }
     __syncthreads();
     const int nc = s_ncentres;
@@ -189,13 +205,17 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
         C[(size_t)c * F + f] = __ddiv_rn(s, (double)count[c]);
     }
     __syncthreads();
-    for (int h = tid; h < H; h += nt) dist[h] = sqdist(X + (size_t)h * F, C + (size_t)a[h] * F, F);
+    // heads in (cluster, head) order: that is the order of the sum below
+    for (int h = tid; h < H; h += nt) {
+        dist[h] = sqdist(X + (size_t)h * F, C + (size_t)a[h] * F, F);
+        int rank = 0;
+        for (int h2 = 0; h2 < H; ++h2) rank += (a[h2] < a[h] || (a[h2] == a[h] && h2 < h)) ? 1 : 0;
+        prev[rank] = h;
+    }
     __syncthreads();
     if (tid == 0) {
         double total = 0.0;
-        for (int c = 0; c < ke; ++c)
-            for (int h = 0; h < H; ++h)
-                if (a[h] == c) total = __dadd_rn(total, dist[h]);
+        for (int i = 0; i < H; ++i) total = __dadd_rn(total, dist[prev[i]]);
         inertia[b] = total;
     }
 }
@@ -326,9 +346,8 @@ int chai_cluster_heads(const float* features, int B, int H, int F, int k, int ma
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaFuncSetAttribute(kmeans_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e, "kmeans_kernel shared-memory opt-in");
-    kmeans_kernel<<<B, 256, smem, s>>>(features, H, F, k, max_iter, (unsigned long long)seed, membership, reps,
-                                       k_eff, inertia);
-    CHAI_LAUNCH_CHECK("kmeans_kernel launch");
+    CHAI_LAUNCH_DEPENDENT("kmeans_kernel launch", kmeans_kernel, dim3(B), dim3(256), smem, s, features, H, F, k, max_iter,
+                          (unsigned long long)seed, membership, reps, k_eff, inertia);
     return CHAI_OK;
 }
 

@@ -14,6 +14,7 @@ __global__ void __launch_bounds__(256)
 append_kv_kernel(const uint4* __restrict__ k_new, const uint4* __restrict__ v_new, uint4* __restrict__ k_rep,
                  uint4* __restrict__ v, const int32_t* __restrict__ reps, int32_t* __restrict__ seq_lens,
                  WsHeader* __restrict__ hdr, int H, int k, int T_cap, int vec_per_row, size_t k_batch_vecs, int advance) {
+    dependent_grid_sync();
     const int b = blockIdx.x, tid = threadIdx.x;
     const int pos = seq_lens[b];
     __syncthreads();  // every thread holds the position before thread 0 may advance it
@@ -102,6 +103,7 @@ compact_inplace_kernel(uint4* __restrict__ k_cache, const int32_t* __restrict__ 
 }
 
 __global__ void reset_status_kernel(WsHeader* hdr) {
+    dependent_grid_sync();
     hdr->status = CHAI_OK;
     hdr->bad_b = -1;
     hdr->bad_h = -1;
@@ -130,14 +132,13 @@ int chai_append_kv(const void* k_new, const void* v_new, void* k_rep, void* v, c
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsHeader* hdr = static_cast<WsHeader*>(workspace);
     if (hdr != nullptr) {
-        reset_status_kernel<<<1, 1, 0, s>>>(hdr);
-        CHAI_LAUNCH_CHECK("chai_append_kv: status reset");
+        CHAI_LAUNCH_DEPENDENT("chai_append_kv: status reset", reset_status_kernel, dim3(1), dim3(1), 0, s, hdr);
     }
     const int vec_per_row = (int)(D * es / 16);
-    append_kv_kernel<<<B, 256, 0, s>>>(static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new),
-                                       static_cast<uint4*>(k_rep), static_cast<uint4*>(v), reps, seq_lens, hdr, H, k,
-                                       T_cap, vec_per_row, k_batch_stride * es / 16, advance);
-    CHAI_LAUNCH_CHECK("append_kv_kernel launch");
+    CHAI_LAUNCH_DEPENDENT("append_kv_kernel launch", append_kv_kernel, dim3(B), dim3(256), 0, s,
+                          static_cast<const uint4*>(k_new), static_cast<const uint4*>(v_new), static_cast<uint4*>(k_rep),
+                          static_cast<uint4*>(v), reps, seq_lens, hdr, H, k, T_cap, vec_per_row,
+                          (size_t)(k_batch_stride * es / 16), advance);
     return CHAI_OK;
 }
 
@@ -156,8 +157,7 @@ int chai_compact_k_cache_inplace(void* k_cache, const int32_t* reps, int B, int 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     WsHeader* hdr = static_cast<WsHeader*>(workspace);
     if (hdr != nullptr) {
-        reset_status_kernel<<<1, 1, 0, s>>>(hdr);
-        CHAI_LAUNCH_CHECK("chai_compact_k_cache_inplace: status reset");
+        CHAI_LAUNCH_DEPENDENT("chai_compact_k_cache_inplace: status reset", reset_status_kernel, dim3(1), dim3(1), 0, s, hdr);
     }
     const int vec_per_row = (int)(D * elem_size(dtype) / 16);
     const size_t n_vecs = (size_t)T * vec_per_row;

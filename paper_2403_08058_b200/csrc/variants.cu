@@ -11,18 +11,15 @@
 
 namespace chai {
 
-// identity maps for the inner k-head problem: membership[b][c] = c, reps[b][c] = c
-__global__ void identity_maps_kernel(int32_t* __restrict__ ident, int n, int k) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) ident[i] = i % k;
-}
-
 // rows of `rows_per_head` * vec_per_row 16-byte vectors per head.
-// gather:  dst[b][c] = src[b][reps[b][c]]   (zero for an unused slot)
+// gather:  dst[b][c] = src[b][reps[b][c]]   (zero for an unused slot); also writes the identity maps of the
+// inner k-head problem: membership[b][c] = c, reps[b][c] = c
 __global__ void __launch_bounds__(256)
-gather_rep_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const int32_t* __restrict__ reps, int H,
-                       int k, size_t vecs_per_head) {
+gather_rep_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const int32_t* __restrict__ reps,
+                       int32_t* __restrict__ ident, int H, int k, size_t vecs_per_head) {
+    dependent_grid_sync();
     const int c = blockIdx.y, b = blockIdx.z;
+    if (blockIdx.x == 0 && threadIdx.x == 0) ident[(size_t)b * k + c] = c;
     const int r = reps[(size_t)b * k + c];
     const bool live = r >= 0 && r < H;
     const uint4* s = src + ((size_t)b * H + (live ? r : 0)) * vecs_per_head;
@@ -123,11 +120,8 @@ int chai_decode_attention_qkv(const void* q, const void* k_rep, const void* v_re
     char* ws = static_cast<char*>(workspace);
     int32_t* ident = reinterpret_cast<int32_t*>(ws + L.off_ident);
     const size_t vecs = (size_t)D * elem_size(dtype) / 16;
-    identity_maps_kernel<<<(B * k + 255) / 256, 256, 0, s>>>(ident, B * k, k);
-    CHAI_LAUNCH_CHECK("identity_maps_kernel launch");
-    gather_rep_rows_kernel<<<dim3(1, k, B), 32, 0, s>>>(static_cast<const uint4*>(q), reinterpret_cast<uint4*>(ws + L.off_q),
-                                                       reps, H, k, vecs);
-    CHAI_LAUNCH_CHECK("gather_rep_rows_kernel launch");
+    CHAI_LAUNCH_DEPENDENT("gather_rep_rows_kernel launch", gather_rep_rows_kernel, dim3(1, k, B), dim3(32), 0, s,
+                          static_cast<const uint4*>(q), reinterpret_cast<uint4*>(ws + L.off_q), reps, ident, H, k, vecs);
     int rc;
     if (seq_lens != nullptr)
         rc = chai_decode_attention_ragged(ws + L.off_q, k_rep, v_rep, ident, ident, seq_lens, ws + L.off_out, B, k, k, T,
@@ -173,10 +167,8 @@ int chai_prefill_attention_qkv(const void* q, const void* k_rep, const void* v_r
     int32_t* ident = reinterpret_cast<int32_t*>(ws + L.off_ident);
     const size_t row_vecs = (size_t)D * elem_size(dtype) / 16;
     const size_t vecs = (size_t)T * row_vecs;
-    identity_maps_kernel<<<(B * k + 255) / 256, 256, 0, s>>>(ident, B * k, k);
-    CHAI_LAUNCH_CHECK("identity_maps_kernel launch");
     gather_rep_rows_kernel<<<dim3(blocks_for(vecs), k, B), 256, 0, s>>>(
-        static_cast<const uint4*>(q), reinterpret_cast<uint4*>(ws + L.off_q), reps, H, k, vecs);
+        static_cast<const uint4*>(q), reinterpret_cast<uint4*>(ws + L.off_q), reps, ident, H, k, vecs);
     CHAI_LAUNCH_CHECK("gather_rep_rows_kernel launch");
     const int rc = chai_prefill_attention_from(ws + L.off_q, k_rep, v_rep, ident, ident, ws + L.off_out, B, k, k, T, q_start,
                                                D, scale, causal, dtype, ws, inner, stream);
