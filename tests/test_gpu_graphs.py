@@ -68,3 +68,54 @@ def test_prefill_graph_replay():
         torch.cuda.synchronize()
         ref = orc.cha_attention(q.cpu(), kr.cpu(), v.cpu(), mem.cpu(), reps.cpu(), scale, True)
         assert_parity(out.float().cpu().numpy(), ref, "bf16", f"prefill graph replay {it}")
+
+
+def test_whole_flow_in_one_graph():
+    """Features, clustering, compaction, prefill, append and a decode step captured as one graph: the kernels
+    that are launched as programmatic dependents of one another keep their order inside a graph, and a replay on
+    new inputs gives bit for bit what the same calls give eagerly."""
+    case = synth.prefill_case(seed=4, B=2, T=300, peaked=4.0)
+    k = case["k"]
+    q, kf, v = (case[n].to(DEV).clone() for n in ("q_full", "k_full", "v"))
+    B, H, T, D = q.shape
+    T_cap = T + 8
+    v_cache = torch.zeros(B, H, T_cap, D, dtype=v.dtype, device=DEV)
+    k_cache = torch.zeros(B, k, T_cap, D, dtype=v.dtype, device=DEV)
+    k_new = torch.randn(B, H, D, device=DEV).to(torch.bfloat16)
+    v_new = torch.randn(B, H, D, device=DEV).to(torch.bfloat16)
+    q_step = torch.randn(B, H, D, device=DEV).to(torch.bfloat16)
+    res = {}
+
+    def flow():
+        feats = chai.chai_prefix_features(q, kf, 5, case["scale"])
+        mem, reps, _, _ = chai.chai_cluster_heads(feats, k, 20, 0)
+        k_rep = chai.chai_compact_k_cache(kf, reps)
+        res["out"] = chai.chai_prefill_attention(q, k_rep, v, mem, reps, case["scale"])
+        v_cache[:, :, :T].copy_(v)
+        k_cache[:, :, :T].copy_(k_rep)
+        lens = torch.full((B,), T, dtype=torch.int32, device=DEV)
+        chai.chai_append_kv(k_new, v_new, k_cache, v_cache, reps, lens)
+        res["dec"] = chai.chai_decode_attention_ragged(q_step, k_cache, v_cache, mem, reps, lens, case["scale"], T + 1)
+        res["mem"] = mem
+
+    flow()                                          # eager warm-up
+    torch.cuda.synchronize()
+    g = capture(flow)
+    graph_res = dict(res)
+    gen = torch.Generator().manual_seed(9)
+    for it in range(3):
+        other = synth.prefill_case(seed=10 + it, B=2, T=300, peaked=4.0)
+        q.copy_(other["q_full"]); kf.copy_(other["k_full"]); v.copy_(other["v"])
+        q_step.copy_((torch.randn(B, H, D, generator=gen)).to(torch.bfloat16))
+        g.replay()
+        torch.cuda.synchronize()
+        got = {n: graph_res[n].clone() for n in ("out", "dec", "mem")}
+        flow()                                      # the same calls, eagerly, on the same inputs
+        torch.cuda.synchronize()
+        for n in ("out", "dec", "mem"):
+            assert torch.equal(got[n], res[n]), f"replay {it}: {n} differs from the eager result"
+        km = orc.kmeans(orc.prefix_features(other["q_full"], other["k_full"], 5, case["scale"]).astype(np.float32), k, 20, 0)
+        assert np.array_equal(got["mem"].cpu().numpy(), km["membership"])
+        k_rep_ref = torch.stack([other["k_full"][b][torch.as_tensor(km["reps"][b]).long()] for b in range(B)])
+        ref = orc.cha_attention(other["q_full"], k_rep_ref, other["v"], km["membership"], km["reps"], case["scale"], True)
+        assert_parity(got["out"].float().cpu().numpy(), ref, "bf16", f"flow graph replay {it}")
