@@ -547,10 +547,11 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "us_per_step": ms_step * 1e3, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16 storage, fp32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": w.name + (" (TRUNCATED for profiling)" if args.layers else ""), "layers": w.layers, "B": w.B, "H": w.H, "D": w.D, "T": w.T,
                        "k_per_layer": [c["k"] for c in wl.layers], "partition": w.partition,
                        "algorithmic_gb_per_step": wl.bytes_per_step / 1e9,
+                       "arithmetic": "bf16 caches, queries and outputs; fp32 scores, softmax and accumulation",
                        "l2": "inputs larger than L2: every layer has its own >=168 MiB caches, 12+ GB per step",
                        "launch": ("one CUDA graph of the step's layer calls, replayed" if graph is not None else "eager launches"),
                        "multi_gpu": "independent replicas, no data-path collective"},
