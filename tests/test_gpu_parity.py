@@ -106,6 +106,27 @@ def test_decode_full_size_layers():
         torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("B,H,k,T", [(2, 8, 3, 100003),     # long context: hundreds of tiles per plane, ragged tail
+                                      (1500, 4, 2, 40),        # many short requests: far more heads than the head table holds
+                                      (1, 1, 1, 1)])           # the smallest problem there is
+def test_decode_extreme_shapes(B, H, k, T):
+    case = synth.decode_layer(2, layer=1, seed=5, device=DEV, B=B, H=H, T=T, k=k, with_k_full=False, peaked=4.0)
+    ws = chai.new_workspace(chai.chai_decode_workspace_bytes(B, H, k, T, 128, chai.CHAI_BF16), DEV)
+    out = chai.chai_decode_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"],
+                                     case["scale"], workspace=ws)
+    out2 = chai.chai_decode_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"],
+                                      case["scale"], workspace=ws)
+    torch.cuda.synchronize()
+    assert chai.chai_device_status(ws) == chai.CHAI_OK
+    assert torch.equal(out, out2)
+    got = out.float().cpu().numpy()
+    step = max(1, B // 6)                                      # every request when B is small, a spread of them otherwise
+    for b in list(range(0, B, step)) + [B - 1]:
+        sl = {n: case[n][b:b + 1].cpu() for n in ("q", "k_rep", "v", "membership", "reps")}
+        ref = orc.cha_attention(sl["q"], sl["k_rep"], sl["v"], sl["membership"], sl["reps"], case["scale"], causal=False)
+        assert_parity(got[b:b + 1], ref, "bf16", f"B {B} H {H} k {k} T {T} request {b}")
+
+
 def test_decode_bad_membership_is_reported_not_faulted():
     case = synth.decode_layer(2, seed=1, B=2, H=8, T=200, k=4)
     ref = oracle_decode(case)
@@ -363,6 +384,25 @@ def test_prefill_full_size_sampled_rows():
     assert_parity(out[:, :, :192].float().cpu().numpy(), head, "bf16", "first rows")
     tail = orc.cha_attention(q[:, :, T - 64:], kr, v, mem, reps, case["scale"], True)
     assert_parity(out[:, :, T - 64:].float().cpu().numpy(), tail, "bf16", "last rows")
+
+
+def test_prefill_long_prompt_sampled_rows():
+    """A prompt of 40 query tiles plus a ragged one: first rows, rows around a tile boundary in the middle, last rows."""
+    B, H, k, T, D = 1, 6, 2, 5003, 128
+    r = synth.batch_partitions(B, H, k, "uneven", 3, 77, T)
+    gen = torch.Generator().manual_seed(11)
+    q = (torch.randn(B, H, T, D, generator=gen) * 2.0).to(torch.bfloat16)
+    kr = (torch.randn(B, k, T, D, generator=gen) * 0.5).to(torch.bfloat16)
+    v = (torch.randn(B, H, T, D, generator=gen) * 0.5).to(torch.bfloat16)
+    mem, reps = torch.as_tensor(r[0]), torch.as_tensor(r[1])
+    scale = 1.0 / np.sqrt(D)
+    out = chai.chai_prefill_attention(q.to(DEV), kr.to(DEV), v.to(DEV), mem.to(DEV), reps.to(DEV), scale)
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy()
+    for lo, hi in ((0, 70), (2530, 2600), (T - 45, T)):
+        # rows [lo, hi) see keys [0, hi): the oracle runs on that prefix and its last hi - lo rows are compared
+        ref = orc.cha_attention(q[:, :, :hi], kr[:, :, :hi], v[:, :, :hi], mem, reps, scale, True)
+        assert_parity(got[:, :, lo:hi], ref[:, :, lo:hi], "bf16", f"long prompt rows {lo}..{hi}")
 
 
 def test_prefill_flow_features_kmeans_compaction_attention():
