@@ -381,7 +381,23 @@ def bench_serving(device, peaks, iters=20, warmup=3):
     v_new = torch.randn((B, H, D), device=device).to(torch.bfloat16)
     ms_a = timed(lambda: chai.chai_append_kv(k_new, v_new, cache, c["v"], c["reps"], seq, advance=False))
     gbs_d, gbs_c = bytes_d / (ms_d * 1e-3) / 1e9, bytes_c / (ms_c * 1e-3) / 1e9
+    # one request with a 128k-token context (k = 8): 1.3 GB per layer call, timed the same way
+    del c, cache
+    torch.cuda.empty_cache()
+    TL = 131072
+    cl = synth.decode_layer(2, 1, 3, device=device, B=1, H=H, T=TL, k=k, with_k_full=False)
+    wsl = chai.new_workspace(chai.chai_decode_workspace_bytes(1, H, k, TL, D, chai.CHAI_BF16), device)
+    outl = torch.empty_like(cl["q"])
+    ms_l = timed(lambda: chai.chai_decode_attention(cl["q"], cl["k_rep"], cl["v"], cl["membership"], cl["reps"], cl["scale"],
+                                                    out=outl, workspace=wsl))
+    bytes_l = decode_bytes(1, H, k, TL, D, es)
+    gbs_l = bytes_l / (ms_l * 1e-3) / 1e9
+    long_ctx = {"workload": "B 1, H 32, k 8, T 131072, bf16", "us": ms_l * 1e3, "algorithmic_mb": bytes_l / 1e6, "gbs": gbs_l,
+                "roofline": {"bound": "hbm", "achieved": gbs_l, "peak": peaks["hbm"], "unit": "GB/s",
+                             "frac": gbs_l / peaks["hbm"], "peak_source": peaks["source"], "traffic": None}}
+    del cl
     return {"workload": "config2 layer shape, k=8, lengths uniform in [T/4, T), K cache compacted in place",
+            "long_context_decode": long_ctx,
             "seq_lens": [int(x) for x in lens],
             "full_length_same_timing": {"us": ms_f * 1e3, "algorithmic_mb": bytes_f / 1e6, "gbs": bytes_f / (ms_f * 1e-3) / 1e9},
             "ragged_decode": {"us": ms_d * 1e3, "algorithmic_mb": bytes_d / 1e6, "gbs": gbs_d,

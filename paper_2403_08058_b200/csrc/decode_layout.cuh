@@ -17,10 +17,12 @@ struct DecodeLayout {
     int CK, CV, nK, nV;  // split kernels: rows per key / value chunk and chunks per plane
     int TR;              // persistent kernel: rows per 16 KB tile
     int capK, capV;      // entries per plane reserved for chunk maxima / partials (either implementation)
-    size_t off_counters, off_flags, off_scores, off_cmax, off_lpart, off_opart, total;
+    size_t off_counters, off_flags, off_scores, off_cmax, off_pmax, off_lpart, off_opart, total;
 };
 
-// off_flags: one 64-bit word per key tile (B * k * capK): carries the launch token once the tile's scores exist
+// off_flags: 64-bit words of the persistent kernel: [0] carries the launch token once the layer's first key tile
+// is done (status and work counter are reset by then); [2 + p] carries it once every key tile of plane p is
+// done and off_pmax[p] holds the plane's largest score; [2 + B*k + p] counts plane p's finished key tiles.
 
 inline bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLayout* L) {
     const int es = (int)elem_size(dtype);
@@ -40,11 +42,13 @@ inline bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLa
     L->off_counters = off;
     off = round_up(off + sizeof(int) * (size_t)B * H, 256);
     L->off_flags = off;
-    off = round_up(off + sizeof(unsigned long long) * (size_t)B * k * L->capK, 256);
+    off = round_up(off + sizeof(unsigned long long) * (2 * (size_t)B * k + 2), 256);
     L->off_scores = off;
     off = round_up(off + sizeof(float) * (size_t)B * k * T, 256);
     L->off_cmax = off;
     off = round_up(off + sizeof(float) * (size_t)B * k * L->capK, 256);
+    L->off_pmax = off;
+    off = round_up(off + sizeof(float) * (size_t)B * k, 256);
     L->off_lpart = off;
     off = round_up(off + sizeof(float) * (size_t)B * H * L->capV, 256);
     L->off_opart = off;

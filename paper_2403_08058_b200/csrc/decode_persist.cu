@@ -8,12 +8,14 @@
 // it; nothing else is synchronised across the warps of a CTA except item completion.
 //
 //   phase K   unit = one key tile (TR rows of one cluster's K_rep), dealt round-robin over CTAs: scaled
-//             scores s_t -> workspace (fp32, stays in L2), the tile's maximum, then the tile's flag word
-//             is set to this launch's token.  Every K_rep row is read exactly once.
+//             scores s_t -> workspace (fp32, stays in L2), the tile's maximum, then an arrival on the plane's
+//             tile counter; the warp whose arrival completes a plane reduces the tile maxima to the plane's
+//             largest score and sets the plane's flag word to this launch's token.  Every K_rep row is read
+//             exactly once.
 //   phase V   unit = item (request, head, run of IV value tiles), claimed by the producers from an atomic
 //             counter, so fast SMs take more.  A tile waits (almost never in practice: planes complete in
-//             request order) until all flags of its cluster's plane carry the token, takes the plane's
-//             global maximum, forms p_t = exp(s_t - max) and reduces its rows; the warp that finishes an
+//             request order) until the flag of its cluster's plane carries the token, takes the plane's
+//             largest score, forms p_t = exp(s_t - max) and reduces its rows; the warp that finishes an
 //             item's last tile adds the tile partials in tile order and publishes (sum p_t V_t, sum p_t);
 //             the warp that completes a head's last item (atomic ticket, nobody waits) adds the item
 //             partials in chunk order and writes out = sum / l.
@@ -90,7 +92,10 @@ struct Params {
     void* out;
     WsHeader* hdr;
     int* counters;               // tickets, one per head
-    unsigned long long* flags;   // one word per key tile
+    unsigned long long* flags;   // [0]: the layer's first key tile is done
+    unsigned long long* pflag;   // per key plane: all its tiles are done and pmax holds its largest score
+    unsigned long long* pcnt;    // per key plane: finished tiles of this launch (launch tag in the upper bits)
+    float* pmax;
     unsigned long long token;    // value unique to this launch (never seen in the flags before)
     float* scores;
     float* cmax;
@@ -170,6 +175,23 @@ __device__ __forceinline__ bool flag_wait_one(const unsigned long long* flag, un
         }
         __nanosleep(100);
     }
+}
+// A key tile of a plane is done: returns how many of the plane's tiles are done now, this one included.  The
+// counter word holds a tag of the launch (40 bits of its token) above a 24-bit count, so whatever an earlier
+// launch or the allocator left there is recognised and replaced by the first arriver; after that every arrival
+// is one atomic add.  The adds are acquire-release: the arriver that completes the plane has all the other
+// tiles' scores and maxima visible.
+__device__ __forceinline__ unsigned long long plane_peek(const unsigned long long* cnt) {
+    unsigned long long cur;  // (issued early, while the tile's bytes are still on their way)
+    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(cur) : "l"(cnt) : "memory");
+    return cur;
+}
+__device__ __forceinline__ unsigned plane_arrive(unsigned long long* cnt, unsigned long long token, unsigned long long cur) {
+    const unsigned long long tag = (token ^ (token >> 24)) << 24;  // epoch and host counter both reach the upper 40 bits
+    if ((cur >> 24) != (tag >> 24)) atomicCAS(cnt, cur, tag);  // stale word: one arriver installs this launch's tag
+    unsigned long long prev;
+    asm volatile("atom.acq_rel.gpu.global.add.u64 %0, [%1], 1;" : "=l"(prev) : "l"(cnt) : "memory");
+    return (unsigned)(prev & 0xffffffull) + 1u;
 }
 // ... and by a whole warp for `n` consecutive flags.
 __device__ __forceinline__ bool flags_wait(const unsigned long long* flags, int n, unsigned long long token, int lane,
@@ -438,6 +460,8 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                     Vec16<TQ>::unpack(*reinterpret_cast<const uint4*>(qsrc + x * Vec16<TQ>::N), qf + x * Vec16<TQ>::N);
             }
             const float kscale = P.k_scale ? P.scale * __ldg(P.k_scale + plane) : P.scale;  // fp8 keys carry a scale per plane
+            unsigned long long cnt_seen = 0;
+            if (lane == 0) cnt_seen = plane_peek(P.pcnt + plane);
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
             if (ok && live && rows == 0) {  // tile beyond this request's length: no scores, neutral maximum
                 if (lane == 0) P.cmax[(size_t)plane * tp + tile] = -INFINITY;
@@ -497,15 +521,43 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                     *work_counter = 0;
                 }
                 // the warp that owns tile 0 of a plane also clears the tickets of the plane's heads: every value
-                // tile of those heads waits for all of the plane's flags, this tile's included
+                // tile of those heads waits until all of the plane's tiles are done, this one included
                 if (tile == 0 && live) {
                     const int c = plane % k;
                     for (int h = lane; h < H; h += 32)
                         if (cluster_of(b, h) == c) P.counters[(size_t)b * H + h] = 0;
                 }
                 __syncwarp();
-                if (lane == 0)
-                    asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(P.flags + (size_t)plane * tp + tile), "l"(token) : "memory");
+                unsigned done = 0;
+                if (lane == 0) {
+                    if (g == 0) asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(P.flags), "l"(token) : "memory");
+                    done = plane_arrive(P.pcnt + plane, token, cnt_seen);
+                }
+                done = __shfl_sync(0xffffffffu, done, 0);
+                if (done == (unsigned)tiles_of(b)) {
+                    // the plane's last tile: every tile's scores and maximum are visible (acquire in the arrival);
+                    // reduce the tile maxima to the plane's largest score and publish the plane
+                    const float* cm = P.cmax + (size_t)plane * tp;
+                    const int nx = tiles_of(b);
+                    float mx = -INFINITY;
+                    if (live) {
+                        int x = lane;
+                        for (; x + 7 * 32 < nx; x += 8 * 32) {
+                            float t8[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) t8[u] = __ldcg(cm + x + u * 32);
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) mx = fmaxf(mx, t8[u]);
+                        }
+                        for (; x < nx; x += 32) mx = fmaxf(mx, __ldcg(cm + x));
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                    }
+                    if (lane == 0) {
+                        P.pmax[plane] = mx;
+                        asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(P.pflag + plane), "l"(token) : "memory");
+                    }
+                }
             }
             if (!ok) break;
             continue;
@@ -529,21 +581,18 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 // after the first tiles of phase V this is a shared-memory bit test)
                 const bool cached = plane < TABLE_CAP && ((*reinterpret_cast<volatile unsigned*>(&sm.ready[plane >> 5]) >> (plane & 31)) & 1u);
                 if (!cached) {
-                    ok = flags_wait(P.flags + plane * tp, tiles_of(b), token, lane, abort_flag);
+                    ok = flags_wait(P.pflag + plane, 1, token, lane, abort_flag);
                     if (ok && lane == 0 && plane < TABLE_CAP) atomicOr(&sm.ready[plane >> 5], 1u << (plane & 31));
                 }
                 if (ok && rows > 0) {  // (the only tile of an empty request has no rows: it just passes the ticket on,
                                        //  which the flag wait above has ordered after the ticket's reset)
-                    float mx = -INFINITY;
-                    for (int x = lane, nx = tiles_of(b); x < nx; x += 32) mx = fmaxf(mx, __ldcg(&P.cmax[plane * tp + x]));
+                    const float mx = __ldcg(P.pmax + plane);  // the plane's largest score
                     const float* srow = P.scores + plane * T_len + (size_t)tile * G::TR;
 #pragma unroll
                     for (int u = 0; u < G::PV; ++u) {
                         const int r = u * 32 + lane;
                         pv[u] = r < rows ? __ldcg(&srow[r]) : -INFINITY;
                     }
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
 #pragma unroll
                     for (int u = 0; u < G::PV; ++u) {
                         pv[u] = pv[u] == -INFINITY ? 0.f : expf(pv[u] - mx);
@@ -652,11 +701,28 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) o[e] = 0.f;
                 float ll = 0.f;
-                for (int i = 0; i < n_chunks; ++i) {
-                    const float* src = P.opart + ((size_t)head * P.nVi + i) * D + lane * DPL;
+                const float* src = P.opart + (size_t)head * P.nVi * D + lane * DPL;
+                const float* lsrc = P.lpart + (size_t)head * P.nVi;
+                int i = 0;
+                for (; i + 8 <= n_chunks; i += 8) {  // long contexts: eight chunks' loads in flight, added in chunk order
+                    float t8[8][DPL], l8[8];
 #pragma unroll
-                    for (int e = 0; e < DPL; ++e) o[e] += __ldcg(src + e);
-                    ll += __ldcg(&P.lpart[(size_t)head * P.nVi + i]);
+                    for (int u = 0; u < 8; ++u) {
+#pragma unroll
+                        for (int e = 0; e < DPL; ++e) t8[u][e] = __ldcg(src + (size_t)(i + u) * D + e);
+                        l8[u] = __ldcg(lsrc + i + u);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+#pragma unroll
+                        for (int e = 0; e < DPL; ++e) o[e] += t8[u][e];
+                        ll += l8[u];
+                    }
+                }
+                for (; i < n_chunks; ++i) {
+#pragma unroll
+                    for (int e = 0; e < DPL; ++e) o[e] += __ldcg(src + (size_t)i * D + e);
+                    ll += __ldcg(lsrc + i);
                 }
 #pragma unroll
                 const float vscale = P.v_scale ? __ldg(P.v_scale + head) : 1.f;  // fp8 values carry a scale per plane
@@ -745,6 +811,9 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     P.hdr = reinterpret_cast<WsHeader*>(ws);
     P.counters = reinterpret_cast<int*>(ws + L.off_counters);
     P.flags = reinterpret_cast<unsigned long long*>(ws + L.off_flags);
+    P.pflag = P.flags + 2;
+    P.pcnt = P.flags + 2 + (size_t)B * k;
+    P.pmax = reinterpret_cast<float*>(ws + L.off_pmax);
     P.scores = reinterpret_cast<float*>(ws + L.off_scores);
     P.cmax = reinterpret_cast<float*>(ws + L.off_cmax);
     P.lpart = reinterpret_cast<float*>(ws + L.off_lpart);
