@@ -158,8 +158,9 @@ int prefill_check_args(const char* fn, const void* q, const void* k_rep, const v
     CHAI_REQUIRE(dtype == CHAI_F32 || dtype == CHAI_BF16, CHAI_ERR_UNSUPPORTED, "%s: unknown dtype %d", fn, dtype);
     CHAI_REQUIRE(D == 64 || D == 128, CHAI_ERR_UNSUPPORTED, "%s: head_dim %d (64 or 128 supported)", fn, D);
     CHAI_REQUIRE(H <= 65535 && B <= 65535, CHAI_ERR_UNSUPPORTED, "%s: H and B must be <= 65535", fn);
-    CHAI_REQUIRE((size_t)(2 * k + 2 * H + 4) * sizeof(int) + sizeof(GroupEntry) * (size_t)H <= 48 * 1024, CHAI_ERR_UNSUPPORTED,
-                 "%s: too many heads for the planner", fn);
+    CHAI_REQUIRE(prefill_plan_smem(H, k) <= 48 * 1024, CHAI_ERR_UNSUPPORTED,
+                 "%s: too many heads and clusters for the planner (H=%d, k=%d need %zu bytes of shared memory, limit 49152)",
+                 fn, H, k, prefill_plan_smem(H, k));
     const PrefillLayout L = prefill_layout(B, H);
     CHAI_REQUIRE(workspace_bytes >= L.total, CHAI_ERR_WORKSPACE, "%s: workspace has %zu bytes, %zu needed", fn,
                  workspace_bytes, L.total);
@@ -169,7 +170,7 @@ int prefill_check_args(const char* fn, const void* q, const void* k_rep, const v
 int prefill_run_plan(const int32_t* membership, const int32_t* reps, int B, int H, int k, int gmax, char* ws,
                      cudaStream_t s) {
     const PrefillLayout L = prefill_layout(B, H);
-    const size_t smem = sizeof(int) * (size_t)((2 * k + 2 * H + 3) & ~3) + sizeof(GroupEntry) * (size_t)H;
+    const size_t smem = prefill_plan_smem(H, k);
     // Launched as a programmatic dependent: when the kernel before it on the stream lets its dependents go
     // early (the tensor-core prefill kernel does), the planner's CTAs are placed while that kernel drains and
     // wait inside griddepcontrol.wait for it to complete, which hides the launch latency between
