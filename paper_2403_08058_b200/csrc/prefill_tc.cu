@@ -415,18 +415,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar.s_free());  // the scores are in registers: the next S = Q K^T may overwrite the buffer
+                // Columns the row may not see (beyond the diagonal, beyond T) become -inf here, in registers:
+                // they then lose every maximum and give probability 0, and the arithmetic below is the same
+                // for every tile.
+                if (!full_tile) {
+#pragma unroll
+                    for (int i = 0; i < 64; ++i)
+                        if (i >= vis) r[i] = 0xff800000u;
+                }
                 // own half-row maximum (eight independent chains)
                 float mxa[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) mxa[c] = -INFINITY;
-                if (full_tile) {
 #pragma unroll
-                    for (int i = 0; i < 64; i += 2) mxa[(i >> 1) & 7] = max3(mxa[(i >> 1) & 7], __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 64; ++i)
-                        if (i < vis) mxa[i & 7] = fmaxf(mxa[i & 7], __uint_as_float(r[i]));
-                }
+                for (int i = 0; i < 64; i += 2) mxa[(i >> 1) & 7] = max3(mxa[(i >> 1) & 7], __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
                 // The two threads of a row must agree on one reference.  Each rounds its half-row maximum up to
                 // bf16 and publishes it (slots alternate with the tile's parity); both take the larger of the two
                 // rounded values, a reference slightly above the true maximum being as good.
@@ -449,23 +451,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     }
                     return true;
                 };
-                // probabilities, rounded to bf16, two per 32-bit column: the layout of an A operand in tensor
-                // memory.  Score columns 64 h + c map to column 32 h + c / 2 of the tile's P buffer.
-                float ls0 = 0.f, ls1 = 0.f, ls2 = 0.f, ls3 = 0.f;
-                // P buffer kt & 1 was last read by the P V of tile kt - 2 (long complete as a rule)
-                if (kt >= 2) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done(sb), ((kt >> 1) & 1) ^ 1, abort_flag));
-                    if (!ok) break;
-                    tc_fence_after();
-                }
-                // After an item's first tile the reference hardly ever moves, so a full tile is computed
-                // against the current reference at once, without waiting for the partner's maximum, and goes
-                // to tensor memory in chunks of 16 probabilities as they are ready; the meeting follows the
-                // arithmetic, and only if some row's reference did move is the tile computed and stored again.
-                const bool speculate = j > 0 && full_tile;
-                bool redo = !speculate;
-                if (speculate) {
-                    const float m_ref = m_used == -INFINITY ? 0.f : m_used;
+                // probabilities against reference m, rounded to bf16, two per 32-bit column: the layout of an A
+                // operand in tensor memory (score columns 64 h + c map to column 32 h + c / 2 of the tile's P
+                // buffer); they leave in chunks of 16 as they are ready.  Returns the row's partial sum.
+                auto emit = [&](float m) -> float {
+                    const float m_ref = m == -INFINITY ? 0.f : m;
                     const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m_ref, -m_ref);
                     uint64_t acc01 = 0ull, acc23 = 0ull;  // two packed pairs of partial row sums
 #pragma unroll
@@ -486,33 +476,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         }
                         tc_st8(p_st + c * 8, packed);
                     }
-                    unpack2(add2(acc01, acc23), ls0, ls1);
+                    float s0, s1;
+                    unpack2(add2(acc01, acc23), s0, s1);
+                    return s0 + s1;
+                };
+                // P buffer kt & 1 was last read by the P V of tile kt - 2 (long complete as a rule)
+                if (kt >= 2) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done(sb), ((kt >> 1) & 1) ^ 1, abort_flag));
+                    if (!ok) break;
+                    tc_fence_after();
                 }
+                // After an item's first tile the reference hardly ever moves, so the tile is computed against
+                // the current reference at once, without waiting for the partner's maximum; the meeting follows
+                // the arithmetic, and only if some row's reference did move is the tile computed and stored again.
+                const bool speculate = j > 0;
+                float ls = 0.f;
+                if (speculate) ls = emit(m_used);
                 ok = meet();
                 if (!ok) break;
-                if (speculate) redo = __any_sync(0xffffffffu, m_new != m_used);
-                if (redo) {
-                    const float m_ref = m_new == -INFINITY ? 0.f : m_new;
-                    ls0 = ls1 = ls2 = ls3 = 0.f;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t packed[8];
-#pragma unroll
-                        for (int u = 0; u < 16; u += 2) {
-                            const int i = c * 16 + u;
-                            float p0 = fast_exp2(fmaf(__uint_as_float(r[i]), scale_log2, -m_ref));
-                            float p1 = fast_exp2(fmaf(__uint_as_float(r[i + 1]), scale_log2, -m_ref));
-                            if (i >= vis) p0 = 0.f;
-                            if (i + 1 >= vis) p1 = 0.f;
-                            ls0 += p0;
-                            ls1 += p1;
-                            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
-                            packed[u >> 1] = *reinterpret_cast<uint32_t*>(&pk);
-                        }
-                        tc_st8(p_st + c * 8, packed);
-                    }
-                }
-                l_run = l_run * corr + ((ls0 + ls1) + (ls2 + ls3));
+                if (!speculate || __any_sync(0xffffffffu, m_new != m_used)) ls = emit(m_new);
+                l_run = l_run * corr + ls;
                 m_used = m_new;
                 // Rescaling touches the O accumulators, so the previous tile's P V must be complete first; a warp
                 // whose rows all keep their reference (the usual case after the first tiles) has nothing to wait
