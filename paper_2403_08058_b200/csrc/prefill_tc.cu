@@ -281,7 +281,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // streams goes through an mbarrier, and tcgen05.commit tracks the issuing thread's own MMAs, so the
         // streams need no program order between them.  Each warp walks its loop as a whole, which keeps the
         // control flow and the descriptor arithmetic warp-uniform; one elected lane issues.
-        constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc(true);
+        constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc(true), IDESC_PV2 = make_idesc_n(true, 2 * HD);
         auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
         auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_polling(b, parity, abort_flag)); };
         const bool qk_role = warp == 1;
@@ -334,6 +334,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (!ok) break;
                     const uint32_t p_addr = tmem_base + P_COL0 + ts * 64;  // P buffer of this tile
                     const bool reuse = j == 0 && qi > 0;  // the accumulators still hold the previous item's output
+                    if (n_members == G && G == 2 && !reuse) {
+                        // Both members at once: their V tiles lie side by side in shared memory (four 64-column
+                        // blocks at one stride) and so do their accumulators in tensor memory, so one N = 256
+                        // instruction per 16 keys does the work of two N = 128 ones and reads P once.
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint32_t d = tmem_base + O_COL0;
+                            const uint32_t vb = v_lo + (ts * G) * (TILE_BYTES >> 4);
+#pragma unroll
+                            for (int s = 0; s < BN / 16; ++s)
+                                tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV2, (j > 0 || s > 0) ? 1u : 0u);
+                            tc_commit(bar.pv_done(ts));
+                        }
+                        __syncwarp();
+                        continue;
+                    }
 #pragma unroll
                     for (int g = 0; g < G; ++g) {
                         if (g >= n_members) break;
