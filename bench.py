@@ -436,6 +436,70 @@ def bench_serving(device, peaks, iters=20, warmup=3):
             "l2": "flushed by a 256 MB write before every timed call"}
 
 
+def bench_config1(device, iters=200, warmup=10):
+    """Configuration 1 (fp32, B 1, H 32, k 8, T 256, D 128; 5 MB, L2 resident): a latency point, microseconds only.
+    The decode call and the clustering of its [1,32,64] features, back to back on one stream; beside them the
+    oracle on one host thread."""
+    c = synth.decode_layer(1, 0, 0, device=device, with_k_full=False)
+    ws = chai.new_workspace(chai.chai_decode_workspace_bytes(c["B"], c["H"], c["k"], c["T"], c["D"], chai.CHAI_F32), device)
+    out = torch.empty_like(c["q"])
+    feats_np, _, _ = synth.blob_features(B=1, H=32, F=64, k=8, seed=0)
+    feats = torch.as_tensor(feats_np, device=device)
+    dec = lambda: chai.chai_decode_attention(c["q"], c["k_rep"], c["v"], c["membership"], c["reps"], c["scale"], out=out,
+                                             workspace=ws)
+    km = lambda: chai.chai_cluster_heads(feats, 8, 20, 0, want_inertia=False)
+    res = {"workload": "config1: fp32, B 1, H 32, k 8, T 256, D 128 (L2 resident); features [1,32,64]"}
+    for name, fn in (("decode", dec), ("cluster_heads", km)):
+        for _ in range(warmup):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(iters):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        res[name + "_us_eager"] = e0.elapsed_time(e1) * 1e3 / iters
+        # the same 20 calls captured in a CUDA graph: what the GPU needs without the host's share
+        g = torch.cuda.CUDAGraph()
+        st = torch.cuda.Stream()
+        st.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.graph(g, stream=st):
+            for _ in range(20):
+                fn()
+        g.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(10):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        res[name + "_us_graph"] = e0.elapsed_time(e1) * 1e3 / 200
+    res["note"] = ("eager: calls enqueued back to back from Python (launch and binding latency); graph: 20 calls per "
+                   "captured graph, replayed")
+    from oracle import chai_oracle as orc
+    cpu = {n: c[n].cpu() for n in ("q", "k_rep", "v", "membership", "reps")}
+    # one host thread for the oracle: the OpenMP runtime is told so from here (the oracle itself is left as it is)
+    threads_before, gomp = orc.num_threads(), None
+    try:
+        import ctypes
+        gomp = ctypes.CDLL("libgomp.so.1")
+        gomp.omp_set_num_threads(1)
+    except OSError:
+        gomp = None
+    orc.cha_attention(cpu["q"], cpu["k_rep"], cpu["v"], cpu["membership"], cpu["reps"], c["scale"], False)
+    t0 = time.perf_counter()
+    n = 0
+    while time.perf_counter() - t0 < 0.5:
+        orc.cha_attention(cpu["q"], cpu["k_rep"], cpu["v"], cpu["membership"], cpu["reps"], c["scale"], False)
+        n += 1
+    res["oracle_decode_us"] = (time.perf_counter() - t0) * 1e6 / n
+    res["oracle_threads"] = orc.num_threads()
+    if gomp is not None:
+        gomp.omp_set_num_threads(threads_before)
+    return res
+
+
 def bench_fp8(device, peaks, iters=20, warmup=3):
     """Decode on e4m3 caches at workload 2's layer shape for k = 8 and k = 32: the layer calls run back to back over
     eight different cache sets (1.3 - 2.2 GB, larger than L2), as in the main decode number."""
@@ -502,7 +566,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers (not a bench result)")
     ap.add_argument("--skip-extras", action="store_true", help="only the decode step (no prefill/compaction/CPU legs)")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a replayed CUDA graph")
-    ap.add_argument("--only", default="", choices=["", "prefill", "compaction", "serving", "fp8"],
+    ap.add_argument("--only", default="", choices=["", "prefill", "compaction", "serving", "fp8", "config1"],
                     help="profiling aid: run just this leg and print its object (not the bench line)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
@@ -529,7 +593,8 @@ def main():
 
     peaks = load_peaks()
     if args.only:
-        leg = {"prefill": bench_prefill, "compaction": bench_compaction, "serving": bench_serving, "fp8": bench_fp8}[args.only]
+        leg = {"prefill": bench_prefill, "compaction": bench_compaction, "serving": bench_serving, "fp8": bench_fp8,
+               "config1": lambda d, p: bench_config1(d)}[args.only]
         print(json.dumps({"leg": args.only, "result": leg(device, peaks)}))
         ranks.close()
         return
@@ -628,6 +693,7 @@ def main():
             line["compaction"] = bench_compaction(device, peaks)
             line["serving"] = bench_serving(device, peaks)
             line["fp8_decode"] = bench_fp8(device, peaks)
+            line["config1"] = bench_config1(device)
             line["cpu_baseline"] = cpu_baseline_decode(args.workload, 0)
         print(json.dumps(line))
     ranks.close()

@@ -41,12 +41,48 @@ __global__ void prefix_features_kernel(const T* __restrict__ q_full, const T* __
 }
 
 // ---- k-means (Section 3.5; objective of Section 3.2) ------------------------------------------------
+// Squared distance, summed in ascending f in one chain (the order the result is defined with).  Only the
+// additions depend on one another: the loads, differences and squares of eight elements are issued ahead of
+// the chain, which is what the time of the whole kernel hangs on.
 __device__ __forceinline__ double sqdist(const double* x, const double* y, int F) {
     double s = 0.0;
-    for (int f = 0; f < F; ++f) {
-        double d = __dsub_rn(x[f], y[f]);
+    int f = 0;
+    for (; f + 8 <= F; f += 8) {
+        double q[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const double d = __dsub_rn(x[f + u], y[f + u]);
+            q[u] = __dmul_rn(d, d);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s = __dadd_rn(s, q[u]);
+    }
+    for (; f < F; ++f) {
+        const double d = __dsub_rn(x[f], y[f]);
         s = __dadd_rn(s, __dmul_rn(d, d));
     }
+    return s;
+}
+
+// Sum over the members of cluster c of feature f, ascending h (the order the mean is defined with); the
+// loads run ahead of the chain of additions.
+__device__ __forceinline__ double member_sum(const double* X, const int* a, int c, int f, int H, int F) {
+    double s = 0.0;
+    int h = 0;
+    for (; h + 8 <= H; h += 8) {
+        double v[8];
+        bool in[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            in[u] = a[h + u] == c;
+            v[u] = X[(size_t)(h + u) * F + f];
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (in[u]) s = __dadd_rn(s, v[u]);
+    }
+    for (; h < H; ++h)
+        if (a[h] == c) s = __dadd_rn(s, X[(size_t)h * F + f]);
     return s;
 }
 
@@ -155,10 +191,7 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
         for (int p = tid; p < nc * F; p += nt) {
             int c = p / F, f = p % F;
             if (count[c] == 0) continue;  // an empty cluster keeps its centre
-            double s = 0.0;
-            for (int h = 0; h < H; ++h)
-                if (a[h] == c) s = __dadd_rn(s, X[(size_t)h * F + f]);
-            C[(size_t)c * F + f] = __ddiv_rn(s, (double)count[c]);
+            C[(size_t)c * F + f] = __ddiv_rn(member_sum(X, a, c, f, H, F), (double)count[c]);
         }
         __syncthreads();
     }
@@ -199,10 +232,7 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
     __syncthreads();
     for (int p = tid; p < ke * F; p += nt) {
         int c = p / F, f = p % F;
-        double s = 0.0;
-        for (int h = 0; h < H; ++h)
-            if (a[h] == c) s = __dadd_rn(s, X[(size_t)h * F + f]);
-        C[(size_t)c * F + f] = __ddiv_rn(s, (double)count[c]);
+        C[(size_t)c * F + f] = __ddiv_rn(member_sum(X, a, c, f, H, F), (double)count[c]);
     }
     __syncthreads();
     // heads in (cluster, head) order: that is the order of the sum below
@@ -249,10 +279,7 @@ select_reps_kernel(const float* __restrict__ features, const int32_t* __restrict
     for (int p = tid; p < k * F; p += nt) {
         const int c = p / F, f = p % F;
         if (count[c] == 0) continue;
-        double s = 0.0;
-        for (int h = 0; h < H; ++h)
-            if (a[h] == c) s = __dadd_rn(s, X[(size_t)h * F + f]);
-        C[(size_t)c * F + f] = __ddiv_rn(s, (double)count[c]);
+        C[(size_t)c * F + f] = __ddiv_rn(member_sum(X, a, c, f, H, F), (double)count[c]);
     }
     __syncthreads();
     for (int h = tid; h < H; h += nt)
