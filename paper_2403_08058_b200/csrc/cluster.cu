@@ -120,15 +120,19 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
     double* dmin = dist;
     for (int h = tid; h < H; h += nt) dmin[h] = sqdist(X + (size_t)h * F, C, F);
     __syncthreads();
-    // The traversal is a chain of k - 1 dependent steps (farthest head, then every head's distance to it), so
-    // one warp walks it without block-wide barriers: lane l owns heads l, l + 32, ... and their dmin entries.
-    if (tid < 32) {
-        const int lane = tid;
+    // The traversal is a chain of k - 1 dependent steps (farthest head, then every head's distance to it).  Four
+    // warps walk it, one per scheduler of the SM (the distances are bound by fp64 throughput, which is per
+    // scheduler): warp w owns the heads h with h mod 4 = w and their dmin entries; per step the warps exchange
+    // their candidates through shared memory and meet at one named barrier.
+    if (tid < 128) {
+        const int w = tid >> 5, lane = tid & 31;
+        __shared__ double s_cd[2][4];
+        __shared__ int s_ch[2][4];
         int ncent = 1;
         for (int n = 1; n < k; ++n) {
             double bd = -1.0;  // farthest head so far: largest dmin, lowest index on ties
             int bh = 0x7fffffff;
-            for (int h = lane; h < H; h += 32) {
+            for (int h = w + 4 * lane; h < H; h += 128) {
                 const double d = dmin[h];
                 if (d > bd) {
                     bd = d;
@@ -144,16 +148,31 @@ __global__ void __launch_bounds__(256) kmeans_kernel(const float* __restrict__ f
                     bh = oh;
                 }
             }
-            if (bd == 0.0) break;  // fewer than k distinct points (warp-uniform)
+            if (lane == 0) {
+                s_cd[n & 1][w] = bd;
+                s_ch[n & 1][w] = bh;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const double od = s_cd[n & 1][x];
+                const int oh = s_ch[n & 1][x];
+                if (od > bd || (od == bd && oh < bh)) {
+                    bd = od;
+                    bh = oh;
+                }
+            }
+            if (bd == 0.0) break;  // fewer than k distinct points (the same decision in all four warps)
             const double* xf = X + (size_t)bh * F;
-            for (int f = lane; f < F; f += 32) C[(size_t)n * F + f] = xf[f];
-            for (int h = lane; h < H; h += 32) {
+            if (w == 0)
+                for (int f = lane; f < F; f += 32) C[(size_t)n * F + f] = xf[f];
+            for (int h = w + 4 * lane; h < H; h += 128) {
                 const double d = sqdist(X + (size_t)h * F, xf, F);
                 if (d < dmin[h]) dmin[h] = d;
             }
             ncent = n + 1;
         }
-        if (lane == 0) s_ncentres = ncent;
+        if (tid == 0) s_ncentres = ncent;
     }
     __syncthreads();
     const int nc = s_ncentres;
