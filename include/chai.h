@@ -211,6 +211,24 @@ int chai_decode_attention_host_async(const void* q_host, void* out_host, void* q
                                      int dtype, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The host-buffer decode step spread over three streams, so that in a run of layer calls the upload of the next
+ * call's queries and the download of the previous call's outputs overlap the kernels: q_host -> q_stage on
+ * upload_stream, the kernels on `stream` (after uploaded_event), out_stage -> out_host on download_stream (after
+ * computed_event).  Streams and events (cudaStream_t / cudaEvent_t passed as void*) belong to the caller; the
+ * two events are recorded by this call and must not be reused before it has run.  Nothing is synchronised:
+ * out_host is valid once download_stream has drained.  Calls that may be in flight together need staging
+ * buffers of their own (q_stage is overwritten as soon as upload_stream gets there; out_stage is read until
+ * download_stream is done), while the workspace may be shared, since the kernels of all calls run in order on
+ * `stream`.  Pinned host memory is required for the copies to overlap anything.
+ */
+int chai_decode_attention_host_streams(const void* q_host, void* out_host, void* q_stage, void* out_stage,
+                                       const void* k_rep, const void* v, const int32_t* membership,
+                                       const int32_t* reps, int B, int H, int k, int T, int T_cap, int D, float scale,
+                                       int dtype, void* workspace, size_t workspace_bytes, void* stream,
+                                       void* upload_stream, void* download_stream, void* uploaded_event,
+                                       void* computed_event);
+
+/*
  * Decode step for callers that can neither pass a workspace nor let the library allocate one
  * (no counterpart in the paper: this is a deployment convenience).  Typical cases: a serving
  * engine that has already handed every free byte of HBM to its KV-cache pool, so a later

@@ -22,7 +22,7 @@ CHAI_F32, CHAI_BF16 = 0, 1
 # every symbol include/chai.h declares
 EXPORTS = [
     "chai_prefix_features", "chai_cluster_heads", "chai_compact_k_cache", "chai_decode_attention",
-    "chai_decode_workspace_bytes", "chai_decode_attention_host", "chai_decode_attention_host_async", "chai_prefill_attention",
+    "chai_decode_workspace_bytes", "chai_decode_attention_host", "chai_decode_attention_host_async", "chai_decode_attention_host_streams", "chai_prefill_attention",
     "chai_prefill_attention_simt", "chai_prefill_workspace_bytes", "chai_device_status",
     "chai_status_string", "chai_last_error", "chai_version", "chai_decode_attention_static",
     "chai_decode_attention_ragged", "chai_append_kv", "chai_compact_k_cache_inplace",
@@ -58,6 +58,8 @@ def load() -> ctypes.CDLL:
     lib.chai_decode_attention.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp, sz, vp]
     for name in ("chai_decode_attention_host", "chai_decode_attention_host_async"):
         getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp, sz, vp]
+    lib.chai_decode_attention_host_streams.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp,
+                                                       sz, vp, vp, vp, vp, vp]
     for name in ("chai_prefill_attention", "chai_prefill_attention_simt"):
         getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
     lib.chai_decode_attention_qkv.argtypes = [vp, vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp, sz, vp]
@@ -299,6 +301,26 @@ def chai_decode_attention_host_async(q_host, out_host, q_stage, out_stage, k_rep
     """As above but only enqueued on the current stream: out_host is valid after the caller synchronises it."""
     return _decode_host("chai_decode_attention_host_async", q_host, out_host, q_stage, out_stage, k_rep, v,
                         membership, reps, scale, workspace, T)
+
+
+def chai_decode_attention_host_streams(q_host, out_host, q_stage, out_stage, k_rep, v, membership, reps, scale: float,
+                                       workspace, stream, upload_stream, download_stream, uploaded_event,
+                                       computed_event, T: int | None = None):
+    """Host-buffer decode step over three torch streams and two torch events (see the header); nothing is
+    synchronised here: out_host is valid once download_stream has drained."""
+    _dev(q_stage, out_stage, k_rep, v, membership, reps, workspace)
+    B, H, D = q_host.shape
+    k, T_cap = k_rep.shape[1], k_rep.shape[2]
+    T = T_cap if T is None else T
+    # a torch event has no CUDA handle before its first record: record once where it does no harm
+    for ev, st in ((uploaded_event, upload_stream), (computed_event, stream)):
+        if not ev.cuda_event:
+            ev.record(st)
+    _check(load().chai_decode_attention_host_streams(
+        q_host.data_ptr(), out_host.data_ptr(), _ptr(q_stage), _ptr(out_stage), _ptr(k_rep), _ptr(v), _ptr(membership),
+        _ptr(reps), B, H, k, T, T_cap, D, scale, _dt(q_host), _ptr(workspace), workspace.numel(), stream.cuda_stream,
+        upload_stream.cuda_stream, download_stream.cuda_stream, uploaded_event.cuda_event, computed_event.cuda_event))
+    return out_host
 
 
 def _prefill(fn_name, q, k_rep, v, membership, reps, scale, causal, out, workspace):

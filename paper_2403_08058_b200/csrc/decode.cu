@@ -339,6 +339,35 @@ int chai_decode_attention_host_async(const void* q_host, void* out_host, void* q
     return CHAI_OK;
 }
 
+int chai_decode_attention_host_streams(const void* q_host, void* out_host, void* q_stage, void* out_stage,
+                                       const void* k_rep, const void* v, const int32_t* membership, const int32_t* reps,
+                                       int B, int H, int k, int T, int T_cap, int D, float scale, int dtype,
+                                       void* workspace, size_t workspace_bytes, void* stream, void* upload_stream,
+                                       void* download_stream, void* uploaded_event, void* computed_event) {
+    using namespace chai;
+    const char* fn = "chai_decode_attention_host_streams";
+    CHAI_REQUIRE(q_host && out_host && q_stage && out_stage, CHAI_ERR_INVALID_ARG, "%s: null pointer", fn);
+    CHAI_REQUIRE(uploaded_event && computed_event, CHAI_ERR_INVALID_ARG, "%s: both events are required", fn);
+    CHAI_REQUIRE(B > 0 && H > 0 && D > 0 && (dtype == CHAI_F32 || dtype == CHAI_BF16), CHAI_ERR_INVALID_ARG,
+                 "%s: bad sizes or dtype", fn);
+    cudaStream_t s = static_cast<cudaStream_t>(stream), up = static_cast<cudaStream_t>(upload_stream),
+                 down = static_cast<cudaStream_t>(download_stream);
+    cudaEvent_t e_up = static_cast<cudaEvent_t>(uploaded_event), e_k = static_cast<cudaEvent_t>(computed_event);
+    const size_t bytes = (size_t)B * H * D * elem_size(dtype);
+    cudaError_t e = cudaMemcpyAsync(q_stage, q_host, bytes, cudaMemcpyHostToDevice, up);
+    if (e == cudaSuccess) e = cudaEventRecord(e_up, up);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, e_up, 0);
+    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_host_streams: query upload");
+    int rc = chai_decode_attention(q_stage, k_rep, v, membership, reps, out_stage, B, H, k, T, T_cap, D, scale, dtype,
+                                   workspace, workspace_bytes, stream);
+    if (rc != CHAI_OK) return rc;
+    e = cudaEventRecord(e_k, s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(down, e_k, 0);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_host, out_stage, bytes, cudaMemcpyDeviceToHost, down);
+    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_host_streams: output download");
+    return CHAI_OK;
+}
+
 int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage, void* out_stage, const void* k_rep,
                                const void* v, const int32_t* membership, const int32_t* reps, int B, int H, int k,
                                int T, int T_cap, int D, float scale, int dtype, void* workspace,

@@ -183,6 +183,19 @@ def test_decode_host_entry_point():
                                               case["scale"], ws)
     torch.cuda.current_stream().synchronize()
     assert torch.equal(oh1, oh) and torch.equal(oh2, oh)
+    # the three-stream form: three calls in flight, each with its own staging buffers and events
+    s_comp, s_up, s_down = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    outs = [torch.zeros_like(oh).pin_memory() for _ in range(3)]
+    stages = [(torch.empty_like(d["q"]), torch.empty_like(d["q"])) for _ in range(3)]
+    events = [(torch.cuda.Event(), torch.cuda.Event()) for _ in range(3)]
+    torch.cuda.synchronize()
+    for o, (qs3, os3), (e_up, e_k) in zip(outs, stages, events):
+        chai.chai_decode_attention_host_streams(qh, o, qs3, os3, d["k_rep"], d["v"], d["membership"], d["reps"],
+                                                case["scale"], ws, s_comp, s_up, s_down, e_up, e_k)
+    s_down.synchronize()
+    s_comp.synchronize()
+    s_up.synchronize()
+    assert all(torch.equal(o, oh) for o in outs)
 
 
 # ---- k-means, features, compaction ---------------------------------------------------------------------
