@@ -311,7 +311,8 @@ def test_prefill_ragged_lengths(fn_name, dtype, T):
 
 
 @pytest.mark.parametrize("H,k,kind", [(8, 8, "even"), (8, 1, "even"), (12, 3, "even"), (16, 2, "uneven"),
-                                      (52, 13, "uneven"), (9, 4, "uneven")])
+                                      (52, 13, "uneven"), (9, 4, "uneven"), (72, 36, "uneven"), (100, 7, "uneven"),
+                                      (64, 64, "even"), (33, 2, "uneven")])
 def test_prefill_cluster_shapes(H, k, kind):
     """Singletons (plain MHA), one cluster of everything, groups of 1..many members."""
     case = prefill_inputs(H * k, 1, H, 160, k, "bf16", kind, peaked=4.0)
