@@ -160,7 +160,8 @@ prefill_plan_kernel(const int32_t* __restrict__ membership, const int32_t* __res
             }
         }
     }
-    // zero-fill groups for unresolved heads (rare): one thread, after the usable clusters' slots
+    // zero-fill groups for unresolved heads (rare): one thread, after the usable clusters' slots; like every
+    // other group they hold at most gmax heads, which is all an attention CTA looks at
     const int total = s_total, nbad = s_nbad;
     if (tid == 0) {
         if (nbad > 0) {
@@ -168,22 +169,22 @@ prefill_plan_kernel(const int32_t* __restrict__ membership, const int32_t* __res
             for (int h = 0; h < H; ++h) {
                 const int c = mem[h];
                 if (!(c < 0 || c >= k || rep[c] < 0)) continue;
-                if (cnt % kGroupMax == 0) {
+                if (cnt % gmax == 0) {
 #pragma unroll
                     for (int x = 0; x < kGroupMax; ++x) hd[x] = h;
                 }
 #pragma unroll
                 for (int x = 0; x < kGroupMax; ++x)
-                    if (x == cnt % kGroupMax) hd[x] = h;
+                    if (x == cnt % gmax) hd[x] = h;
                 ++cnt;
-                if (cnt % kGroupMax == 0 || cnt == nbad) {
-                    int4* dst = reinterpret_cast<int4*>(out + total + (cnt - 1) / kGroupMax);
-                    dst[0] = make_int4(-1, -1, (cnt - 1) % kGroupMax + 1, 0);
+                if (cnt % gmax == 0 || cnt == nbad) {
+                    int4* dst = reinterpret_cast<int4*>(out + total + (cnt - 1) / gmax);
+                    dst[0] = make_int4(-1, -1, (cnt - 1) % gmax + 1, 0);
                     dst[1] = make_int4(hd[0], hd[1], hd[2], hd[3]);
                 }
             }
         }
-        n_groups[b] = total + (nbad + kGroupMax - 1) / kGroupMax;
+        n_groups[b] = total + (nbad + gmax - 1) / gmax;
         bad_out[b] = nbad > 0 ? s_first_bad + 1 : 0;
     }
 }

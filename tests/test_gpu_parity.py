@@ -382,6 +382,31 @@ def test_prefill_negative_controls_and_bad_membership():
     assert gate_ok(got[0, keep], ref[0, keep], "bf16")
 
 
+@pytest.mark.parametrize("fn_name", ["chai_prefill_attention", "chai_prefill_attention_simt"])
+def test_prefill_many_unresolved_heads(fn_name):
+    """A whole cluster loses its representative and two more heads carry ids out of range: seven heads in all,
+    i.e. more than one zero-fill group; the others are untouched."""
+    case = prefill_inputs(5, 2, 40, 200, 8, "bf16", "even", peaked=4.0)   # 8 clusters of 5 heads
+    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], True)
+    d = to_dev(case)
+    mem, reps = d["membership"].clone(), d["reps"].clone()
+    lost = [h for h in range(40) if int(case["membership"][1, h]) == 3]
+    reps[1, 3] = -1                                                     # cluster 3 of request 1: no representative
+    others = [h for h in range(40) if h not in lost and h not in case["reps"][1].tolist()][:2]
+    mem[1, others[0]] = 99
+    mem[1, others[1]] = -1
+    bad = sorted(lost + others)
+    ws = chai.new_workspace(chai.chai_prefill_workspace_bytes(2, 40, 8, 200, 128, chai.CHAI_BF16), DEV)
+    out = torch.full_like(d["q"], 7.0)
+    getattr(chai, fn_name)(d["q"], d["k_rep"], d["v"], mem, reps, case["scale"], True, out=out, workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_ERR_BAD_MEMBERSHIP
+    got = out.float().cpu().numpy()
+    assert not got[1, bad].any()
+    keep = np.array([h not in bad for h in range(40)])
+    assert gate_ok(got[1, keep], ref[1, keep], "bf16")
+    assert gate_ok(got[0], ref[0], "bf16")
+
+
 def test_prefill_full_size_sampled_rows():
     """Workload 5 at full size: the first 192 rows and the last 64 rows of every request and head
     (causal attention of the first rows depends only on the first keys; the last rows see everything)."""
