@@ -407,6 +407,39 @@ def test_prefill_many_unresolved_heads(fn_name):
     assert gate_ok(got[0], ref[0], "bf16")
 
 
+def test_prefill_more_requests_than_one_launch_holds():
+    """70 requests: the tensor-core path walks them in two launches of at most 64, each with its own work counter."""
+    case = prefill_inputs(8, 70, 4, 140, 2, "bf16", "uneven", peaked=4.0)
+    got = run_prefill(case)
+    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], True)
+    assert_parity(got, ref, "bf16", "B 70")
+
+
+def test_unused_cluster_slots():
+    """k = 5 slots of which only 3 hold a cluster (what clustering returns when it finds fewer distinct points):
+    reps = -1 at the end, no head points there; decode and prefill skip the dead planes."""
+    B, H, k, T = 2, 8, 5, 200
+    case = prefill_inputs(3, B, H, T, 3, "bf16", "even", peaked=4.0)
+    mem = case["membership"]
+    reps = torch.full((B, k), -1, dtype=torch.int32)
+    reps[:, :3] = case["reps"]
+    k_rep = torch.zeros(B, k, T, 128, dtype=torch.bfloat16)
+    k_rep[:, :3] = case["k_rep"]
+    k_rep[:, 3:] = float("nan")                                       # dead planes: never read into a result
+    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], mem, case["reps"], case["scale"], True)
+    d = {n: x.to(DEV) for n, x in (("q", case["q"]), ("k_rep", k_rep), ("v", case["v"]), ("mem", mem), ("reps", reps))}
+    for fn in (chai.chai_prefill_attention, chai.chai_prefill_attention_simt):
+        ws = chai.new_workspace(chai.chai_prefill_workspace_bytes(B, H, k, T, 128, chai.CHAI_BF16), DEV)
+        out = fn(d["q"], d["k_rep"], d["v"], d["mem"], d["reps"], case["scale"], True, workspace=ws)
+        assert chai.chai_device_status(ws) == chai.CHAI_OK
+        assert_parity(out.float().cpu().numpy(), ref, "bf16", f"{fn.__name__} with unused slots")
+    q_last = d["q"][:, :, -1].contiguous()
+    ws = chai.new_workspace(chai.chai_decode_workspace_bytes(B, H, k, T, 128, chai.CHAI_BF16), DEV)
+    dec = chai.chai_decode_attention(q_last, d["k_rep"], d["v"], d["mem"], d["reps"], case["scale"], workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_OK
+    assert_parity(dec.float().cpu().numpy(), ref[:, :, -1], "bf16", "decode with unused slots")
+
+
 def test_prefill_full_size_sampled_rows():
     """Workload 5 at full size: the first 192 rows and the last 64 rows of every request and head
     (causal attention of the first rows depends only on the first keys; the last rows see everything)."""
