@@ -685,16 +685,19 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
     rc = prefill_run_plan(membership, reps, B, H, k, tc::G, ws, s);
     if (rc != CHAI_OK) return rc;
     const PrefillLayout L = prefill_layout(B, H);
-    static int n_sms = 0;
-    static bool configured = false;
-    if (!configured) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+    // per device: SM count, and the kernel's opt-in to its shared-memory size
+    static int sms_of_device[64] = {};
+    int dev = 0;
+    cudaError_t de = cudaGetDevice(&dev);
+    if (de != cudaSuccess) return cuda_fail(de, "prefill_tc_kernel set-up");
+    int& n_sms = sms_of_device[dev & 63];
+    if (n_sms == 0) {
+        int count = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(tc::prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
         if (e != cudaSuccess) return cuda_fail(e, "prefill_tc_kernel set-up");
-        configured = true;
+        n_sms = count;
     }
     const int n_qtiles = (T + tc::BM - 1) / tc::BM;
     // one persistent CTA per SM; requests are processed in chunks of MAX_B (the per-request group counts of
