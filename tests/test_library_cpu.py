@@ -100,3 +100,38 @@ def test_product_code_never_touches_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 assert "oracle" not in open(os.path.join(dirpath, f)).read().lower().replace(
                     "cpu oracle", ""), f
+
+
+def header_prototypes():
+    """name -> list of C parameter declarations, from include/chai.h (comments removed)."""
+    text = open(os.path.join(ROOT, "include", "chai.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    protos = {}
+    for m in re.finditer(r"\b(chai_[a-z0-9_]+)\s*\(([^;{]*?)\)\s*;", text, flags=re.S):
+        params = [p.strip() for p in m.group(2).replace("\n", " ").split(",")]
+        protos[m.group(1)] = [] if params == ["void"] else params
+    return protos
+
+
+def test_binding_signatures_match_the_header(lib):
+    """Every entry point that takes arguments has ctypes argtypes of the header's arity, with pointers where the
+    header has pointers, 64-bit integers for size_t / uint64_t and a float for float (a mismatch would corrupt the
+    call silently)."""
+    protos = header_prototypes()
+    assert set(protos) == set(chai.EXPORTS)
+    for name, params in protos.items():
+        fn = getattr(lib, name)
+        if not params:
+            continue
+        assert fn.argtypes is not None, f"{name}: no argtypes declared in the binding"
+        assert len(fn.argtypes) == len(params), f"{name}: header has {len(params)} parameters, binding {len(fn.argtypes)}"
+        for i, (decl, ct) in enumerate(zip(params, fn.argtypes)):
+            where = f"{name} parameter {i} ({decl})"
+            if "*" in decl:
+                assert ct in (ctypes.c_void_p, ctypes.c_char_p) or issubclass(ct, ctypes._Pointer), where
+            elif decl.startswith(("size_t", "uint64_t")):
+                assert ctypes.sizeof(ct) == 8 and ct not in (ctypes.c_void_p, ctypes.c_double), where
+            elif decl.startswith("float"):
+                assert ct is ctypes.c_float, where
+            else:
+                assert ct is ctypes.c_int, where
