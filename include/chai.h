@@ -257,8 +257,8 @@ int chai_decode_attention_static(const void* q, const void* k_rep, const void* v
  * query rows; decoder-only models attend causally, Section 2).
  *   q [B,H,T,D] (only representative heads' rows are read), k_rep [B,k,T,D],
  *   v [B,H,T,D], out [B,H,T,D];  causal != 0: row i sees keys j <= i.
- * bf16 with D = 128 runs on the tcgen05 tensor-core kernel; fp32 (and D = 64) on
- * the CUDA-core kernel, which chai_prefill_attention_simt selects for any dtype.
+ * bf16 (D = 128 or 64) runs on the tcgen05 tensor-core kernel; fp32 on the CUDA-core
+ * kernel, which chai_prefill_attention_simt selects for any dtype.
  * Errors: CHAI_ERR_INVALID_ARG / CHAI_ERR_WORKSPACE as for decode; CHAI_ERR_UNSUPPORTED for another head_dim or
  * dtype, for H or B above 65535, and when the work list of one request does not fit the planning kernel's
  * 48 KB of shared memory (4 * (H + 3 k + k * ceil(H / 32)) bytes: e.g. H = k = 512 still fits).  Inconsistent

@@ -16,6 +16,8 @@
 // (TMEM lane quadrant = warp index mod 4; warps 2..5 take columns 0..63 of a tile, warps 6..9
 // columns 64..127); warps 10..13 = epilogue (O / l -> bf16 -> global) of the previous unit while
 // the next one computes; warp 14 = issuer of the P V batches.
+// head_dim 64 is a second instantiation: a tile is one 64-column block (in the first half of the same 32 KB
+// slots), the accumulators have 64 columns, and the P V instructions have N = 64 (one member) or 128 (two).
 // Every mbarrier wait is bounded: on expiry the CTA records CHAI_ERR_TIMEOUT in the workspace
 // status word, skips the rest of its work, frees its tensor memory and returns.
 #include <cuda.h>
@@ -37,11 +39,11 @@ namespace tc {
 
 constexpr int BM = 128;            // query rows per CTA
 constexpr int BN = 128;            // keys per tile
-constexpr int HD = 128;            // head dimension
 constexpr int G = 2;               // member heads per CTA
 constexpr int KST = 2;             // K tile stages (tile kt uses stage kt & 1)
 constexpr int VST = 2 * G;         // V tile slots: tile kt uses slots (kt & 1) * G + g
-constexpr int TILE_BYTES = BN * HD * 2;        // 32 KB: one 128 x 128 bf16 tile = two 64-column boxes
+constexpr int TILE_BYTES = BN * 128 * 2;       // 32 KB: a tile slot; a 128 x 128 bf16 tile fills it with two 64-column boxes,
+                                               // a 128 x 64 tile (head_dim 64) uses its first half
 constexpr int HALF_BYTES = TILE_BYTES / 2;     // 16 KB: one 128-row x 64-column swizzled box
 constexpr int SOFTMAX_WARPS = 8;    // two per TMEM lane quadrant: each thread owns half a row (64 columns)
 constexpr int EPILOGUE_WARPS = 4;   // one thread per query row: O / l -> bf16 -> global while the next item computes
@@ -114,12 +116,18 @@ struct Item {
 // by an atomic counter in descending order of cost.  While the softmax warps finish one item, the
 // producer is already fetching the next item's Q, K and V tiles and the tensor core computes its
 // first scores, so the pipeline fill of an item hides behind the drain of the previous one.
+template <int HD>
 __global__ void __launch_bounds__(THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int* __restrict__ n_groups,
                   const GroupEntry* __restrict__ groups, __nv_bfloat16* __restrict__ out, WsHeader* __restrict__ hdr,
                   const int* __restrict__ bad, int B_total, int b_begin, int B, int H, int k, int T_len, int q_start,
                   float scale_log2, int causal, int n_qtiles, int counter_slot) {
+    static_assert(HD == 128 || HD == 64, "head_dim 128 or 64");
+    constexpr int LOAD_BYTES = BN * HD * 2;  // bytes one tile copy brings
+    // stride between the 64-column blocks an MN-major V operand walks: the two halves of a 128-wide tile, or
+    // (head_dim 64, two members in one instruction) the single blocks of two neighbouring slots
+    constexpr int V_LBO = HD == 128 ? HALF_BYTES : TILE_BYTES;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw;
@@ -244,13 +252,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // Q: wait until the previous item's last S = Q K^T has been computed
                 ok = mbar_wait(bar.q_empty(), (qi & 1) ^ 1, abort_flag);
                 if (!ok) break;
-                mbar_expect_tx(bar.q_full(), TILE_BYTES);
+                mbar_expect_tx(bar.q_full(), LOAD_BYTES);
                 tma_load_4d(sbase + OFF_Q, &map_q, q0, q_plane, bar.q_full());
                 // key tile number kt + j of this CTA's life: K stage and V slots (kt + j) & 1
                 auto load_k = [&](int j) -> bool {
                     const int n = kt + j, ts = n & 1;
                     if (!mbar_wait(bar.qk_done(ts), ((n >> 1) & 1) ^ 1, abort_flag)) return false;  // stage free
-                    mbar_expect_tx(bar.k_full(ts), TILE_BYTES);
+                    mbar_expect_tx(bar.k_full(ts), LOAD_BYTES);
                     tma_load_4d(sbase + OFF_K + ts * TILE_BYTES, &map_k, j * BN, k_plane, bar.k_full(ts));
                     return true;
                 };
@@ -262,7 +270,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     const int n = kt + j, ts = n & 1;
                     ok = mbar_wait(bar.pv_done(ts), ((n >> 1) & 1) ^ 1, abort_flag);  // the tile's V slots are free
                     if (!ok) break;
-                    mbar_expect_tx(bar.v_full(ts), n_members * TILE_BYTES);
+                    mbar_expect_tx(bar.v_full(ts), n_members * LOAD_BYTES);
                     for (int g = 0; g < n_members; ++g)
                         tma_load_4d(sbase + OFF_V + (ts * G + g) * TILE_BYTES, &map_v, j * BN, v_plane[g], bar.v_full(ts));
                     if (j == 0) resolve(nxt);  // two tiles are on their way: time to look at the claim's answer
@@ -281,7 +289,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // streams goes through an mbarrier, and tcgen05.commit tracks the issuing thread's own MMAs, so the
         // streams need no program order between them.  Each warp walks its loop as a whole, which keeps the
         // control flow and the descriptor arithmetic warp-uniform; one elected lane issues.
-        constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc(true), IDESC_PV2 = make_idesc_n(true, 2 * HD);
+        constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc_n(true, HD), IDESC_PV2 = make_idesc_n(true, 2 * HD);
         auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
         auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_polling(b, parity, abort_flag)); };
         const bool qk_role = warp == 1;
@@ -289,7 +297,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // moves, by compile-time offsets, so issuing an MMA costs an add and the instruction.
         const uint64_t dq = make_desc(sbase + OFF_Q, 16, 1024);
         const uint64_t dk = make_desc(sbase + OFF_K, 16, 1024);
-        const uint64_t dv = make_desc(sbase + OFF_V, HALF_BYTES, 1024);
+        const uint64_t dv = make_desc(sbase + OFF_V, V_LBO, 1024);
         const uint32_t hi_k = (uint32_t)(dq >> 32), hi_v = (uint32_t)(dv >> 32);
         const uint32_t q_lo = (uint32_t)dq, k_lo = (uint32_t)dk, v_lo = (uint32_t)dv;
         bool ok = true;
@@ -403,9 +411,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (n_kv == 0) {  // unresolved heads: zero rows
                 if (row_abs >= q_start && row_abs < T_len)
                     for (int g = 0; g < n_members; ++g) {
-                        uint4* o = reinterpret_cast<uint4*>(out + ((size_t)item.o_plane[g] * T_len + row_abs) * HD + cbase);
+                        uint4* o = reinterpret_cast<uint4*>(out + ((size_t)item.o_plane[g] * T_len + row_abs) * HD + half * (HD / 2));
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) o[u] = make_uint4(0, 0, 0, 0);
+                        for (int u = 0; u < HD / 16; ++u) o[u] = make_uint4(0, 0, 0, 0);
                     }
                 ++it;
                 continue;
@@ -521,15 +529,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done((kt - 1) & 1), ((kt - 1) >> 1) & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
-                    for (int g = 0; g < n_members; ++g) {  // this thread rescales its 64 columns of each O
-                        const uint32_t o_addr = lane_addr + O_COL0 + g * HD + cbase;
+                    for (int g = 0; g < n_members; ++g) {  // this thread rescales its half of the columns of each O
+                        const uint32_t o_addr = lane_addr + O_COL0 + g * HD + half * (HD / 2);
                         tc_ld32(o_addr, r);
-                        tc_ld32(o_addr + 32, r + 32);
+                        if constexpr (HD == 128) tc_ld32(o_addr + 32, r + 32);
                         tc_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 64; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
+                        for (int i = 0; i < HD / 2; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
                         tc_st32(o_addr, r);
-                        tc_st32(o_addr + 32, r + 32);
+                        if constexpr (HD == 128) tc_st32(o_addr + 32, r + 32);
                     }
                 }
                 tc_wait_st();          // P (and any rescaled O) is in tensor memory
@@ -582,11 +590,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             for (int g = 0; g < ep.n_members; ++g) {
                 __nv_bfloat16* orow = out + ((size_t)ep.o_plane[g] * T_len + row_abs) * HD;
 #pragma unroll
-                for (int ch = 0; ch < 2; ++ch) {  // 64 columns per round: two loads in flight
+                for (int ch = 0; ch < HD / 64; ++ch) {  // 64 columns per round: two loads in flight
                     tc_ld32(lane_addr + O_COL0 + g * HD + ch * 64, r);
                     tc_ld32(lane_addr + O_COL0 + g * HD + ch * 64 + 32, r + 32);
                     tc_wait_ld();
-                    if (ch == 1) {  // this row of the member's accumulator is in registers
+                    if (ch == HD / 64 - 1) {  // this row of the member's accumulator is in registers
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) {
@@ -643,18 +651,19 @@ static EncodeTiledFn encode_tiled_fn() {
 // box = 64 x 128 x 2 x 1, i.e. a whole 128 x 128 tile per copy, stored as two swizzled 64-column blocks.
 // [planes, T, 128] bf16 seen as (64 columns, T rows, 2 column halves, planes); one copy moves box_rows rows of
 // both halves, which land as two consecutive blocks of 128-byte swizzled rows.
-static bool make_map_rows(CUtensorMap* map, const void* base, int planes, int T, int box_rows) {
+static bool make_map_rows(CUtensorMap* map, const void* base, int planes, int T, int box_rows, int HD) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (fn == nullptr) return false;
-    cuuint64_t dims[4] = {64, (cuuint64_t)T, 2, (cuuint64_t)planes};
+    const cuuint32_t halves = (cuuint32_t)(HD / 64);  // head_dim 64: one 64-column block per row
+    cuuint64_t dims[4] = {64, (cuuint64_t)T, halves, (cuuint64_t)planes};
     cuuint64_t strides[3] = {(cuuint64_t)HD * 2, 128, (cuuint64_t)T * HD * 2};
-    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 2, 1};
+    cuuint32_t box[4] = {64, (cuuint32_t)box_rows, halves, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-static bool make_map(CUtensorMap* map, const void* base, int planes, int T) { return make_map_rows(map, base, planes, T, BN); }
+static bool make_map(CUtensorMap* map, const void* base, int planes, int T, int HD) { return make_map_rows(map, base, planes, T, BN, HD); }
 
 }  // namespace tc
 }  // namespace chai
@@ -669,7 +678,7 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
                                            float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
                                            void* stream) {
     using namespace chai;
-    if (dtype != CHAI_BF16 || D != tc::HD || B > 60 * tc::MAX_B)
+    if (dtype != CHAI_BF16 || (D != 128 && D != 64) || B > 60 * tc::MAX_B)
         return chai_prefill_attention_simt_from(q, k_rep, v, membership, reps, out, B, H, k, T, q_start, D, scale, causal,
                                                 dtype, workspace, workspace_bytes, stream);
     int rc = prefill_check_args("chai_prefill_attention", q, k_rep, v, membership, reps, out, B, H, k, T, D, dtype,
@@ -678,7 +687,7 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
     CHAI_REQUIRE(q_start >= 0 && q_start < T, CHAI_ERR_INVALID_ARG,
                  "chai_prefill_attention: need 0 <= q_start < T (q_start=%d, T=%d)", q_start, T);
     CUtensorMap mq, mk, mv;
-    CHAI_REQUIRE(tc::make_map(&mq, q, B * H, T) && tc::make_map(&mk, k_rep, B * k, T) && tc::make_map(&mv, v, B * H, T),
+    CHAI_REQUIRE(tc::make_map(&mq, q, B * H, T, D) && tc::make_map(&mk, k_rep, B * k, T, D) && tc::make_map(&mv, v, B * H, T, D),
                  CHAI_ERR_CUDA, "chai_prefill_attention: cuTensorMapEncodeTiled failed");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
@@ -695,7 +704,9 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
         int count = 0;
         cudaError_t e = cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc::prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+            e = cudaFuncSetAttribute(tc::prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc::prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
         if (e != cudaSuccess) return cuda_fail(e, "prefill_tc_kernel set-up");
         n_sms = count;
     }
@@ -716,11 +727,17 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        cudaError_t le = cudaLaunchKernelEx(
-            &cfg, tc::prefill_tc_kernel, mq, mk, mv, reinterpret_cast<const int*>(ws + L.off_ngroups),
-            reinterpret_cast<const GroupEntry*>(ws + L.off_groups), static_cast<__nv_bfloat16*>(out),
-            reinterpret_cast<WsHeader*>(ws), reinterpret_cast<const int*>(ws + L.off_bad), B, b0, nb, H, k, T, q_start,
-            scale * 1.4426950408889634f, causal, n_qtiles, chunk);
+        const int* ng = reinterpret_cast<const int*>(ws + L.off_ngroups);
+        const GroupEntry* gr = reinterpret_cast<const GroupEntry*>(ws + L.off_groups);
+        __nv_bfloat16* o = static_cast<__nv_bfloat16*>(out);
+        WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
+        const int* bad = reinterpret_cast<const int*>(ws + L.off_bad);
+        const float scale_log2 = scale * 1.4426950408889634f;
+        cudaError_t le =
+            D == 128 ? cudaLaunchKernelEx(&cfg, tc::prefill_tc_kernel<128>, mq, mk, mv, ng, gr, o, hdr, bad, B, b0, nb, H, k, T,
+                                          q_start, scale_log2, causal, n_qtiles, chunk)
+                     : cudaLaunchKernelEx(&cfg, tc::prefill_tc_kernel<64>, mq, mk, mv, ng, gr, o, hdr, bad, B, b0, nb, H, k, T,
+                                          q_start, scale_log2, causal, n_qtiles, chunk);
         if (le != cudaSuccess) return cuda_fail(le, "prefill_tc_kernel launch");
         CHAI_LAUNCH_CHECK("prefill_tc_kernel launch");
     }

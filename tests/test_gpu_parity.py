@@ -353,11 +353,19 @@ def test_prefill_reference_moves(direction, causal):
     assert_parity(got, ref, "bf16", f"reference moves: {direction} causal {causal}")
 
 
-def test_prefill_head_dim_64():
-    case = prefill_inputs(9, 2, 6, 150, 2, "bf16", D=64, peaked=4.0)
-    got = run_prefill(case)
-    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], True)
-    assert_parity(got, ref, "bf16", "D 64")
+@pytest.mark.parametrize("T", [1, 33, 128, 129, 150, 300, 700])
+@pytest.mark.parametrize("H,k,kind", [(6, 2, "uneven"), (8, 8, "even"), (8, 2, "even")])
+def test_prefill_head_dim_64(T, H, k, kind):
+    """head_dim 64 on the tensor-core kernel (one 64-column block per tile; pairs of members, single members and
+    the moving-reference path all occur), causal and not, against the oracle; the CUDA-core kernel beside it."""
+    case = prefill_inputs(9 + T, 2, H, T, k, "bf16", kind, D=64, peaked=4.0)
+    for causal in (True, False):
+        ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], causal)
+        assert_parity(run_prefill(case, causal), ref, "bf16", f"D 64 T {T} H {H} k {k} causal {causal}")
+    if T == 150:
+        got = run_prefill(case, True, chai.chai_prefill_attention_simt)
+        ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], True)
+        assert_parity(got, ref, "bf16", "D 64, CUDA-core kernel")
 
 
 def test_prefill_negative_controls_and_bad_membership():
