@@ -387,3 +387,41 @@ def test_e4m3_table_and_quantiser():
     q, s = orc.quantize_cache_fp8(y, 2)
     assert s[0] == np.float32(4.0) / np.float32(448.0) and s[1] == 1.0
     assert np.allclose(vals[q[0, :2]] * s[0], y[0, :2], rtol=2 ** -4) and not q[0, 2].any() and not q[1].any()
+
+
+def test_fp8_decode_is_the_decode_definition_on_what_the_bytes_stand_for():
+    """Values chosen from the e4m3 grid (built here from the format's definition, not from the oracle's table):
+    with scale 1 the byte caches stand for exactly the original numbers, so the fp8 decode must equal plain
+    clustered attention on them; scaling a plane's bytes' scale by 2 must equal doubling that plane."""
+    rng = np.random.default_rng(5)
+    grid = np.array([0.0] + [m / 8 * 2.0 ** -6 for m in range(1, 8)] +
+                    [(1 + m / 8) * 2.0 ** (e - 7) for e in range(1, 16) for m in range(8)][:-1])   # up to 448
+    assert grid[-1] == 448.0 and len(grid) == 127
+    B, H, k, T, D = 2, 4, 2, 9, 8
+    mem = np.array([[0, 1, 0, 1], [0, 0, 0, 1]], dtype=np.int32)
+    reps = np.array([[0, 1], [0, 3]], dtype=np.int32)
+    pick = lambda shape: (grid[rng.integers(0, 60, size=shape)] * rng.choice([-1.0, 1.0], size=shape)).astype(np.float32)
+    k_rep, v = pick((B, k, T, D)), pick((B, H, T, D))
+    k_rep[:, :, 0, 0] = 448.0          # every plane's largest magnitude is 448: scale 1
+    v[:, :, 0, 0] = -448.0
+    q = rng.standard_normal((B, H, D)).astype(np.float32)
+    k8, ks = orc.quantize_cache_fp8(k_rep, T)
+    v8, vs = orc.quantize_cache_fp8(v, T)
+    assert np.all(ks == 1.0) and np.all(vs == 1.0)
+    lens = [T, 5]
+    got = orc.decode_attention_fp8(q, k8, v8, ks, vs, mem, reps, lens, 0.3)
+    want = orc.decode_attention_ragged(q, k_rep, v, mem, reps, lens, 0.3)
+    assert np.abs(got - want).max() <= 1e-12
+    # plane scales are plain multipliers of the plane
+    vs2 = vs.copy()
+    vs2[1, 2] = 2.0
+    v2 = v.copy()
+    v2[1, 2] *= 2.0
+    got2 = orc.decode_attention_fp8(q, k8, v8, ks, vs2, mem, reps, lens, 0.3)
+    assert np.abs(got2 - orc.decode_attention_ragged(q, k_rep, v2, mem, reps, lens, 0.3)).max() <= 1e-12
+    ks2 = ks.copy()
+    ks2[0, 1] = 0.5
+    k2 = k_rep.copy()
+    k2[0, 1] *= 0.5
+    got3 = orc.decode_attention_fp8(q, k8, v8, ks2, vs, mem, reps, lens, 0.3)
+    assert np.abs(got3 - orc.decode_attention_ragged(q, k2, v, mem, reps, lens, 0.3)).max() <= 1e-12
