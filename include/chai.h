@@ -16,7 +16,8 @@
  *     between calls other than the text of the last error.
  *   - Asynchrony: a call validates its scalar arguments on the host, enqueues its
  *     kernels on `stream` (a cudaStream_t passed as void*) and returns; it never
- *     synchronises, except chai_device_status and the *_host entry points.
+ *     synchronises, except chai_device_status and chai_decode_attention_host (the
+ *     other host-buffer entry points, *_host_async and *_host_streams, leave the wait to the caller).
  *   - Errors: the return value is a chai_status_t.  Anything checkable on the host
  *     (null or misaligned pointer, non-positive size, k > H, unsupported head
  *     dimension, workspace too small) is refused before any launch.  Errors in
