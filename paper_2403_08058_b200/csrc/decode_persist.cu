@@ -43,11 +43,11 @@ namespace pd {
 // slots and more warps work side by side.
 template <typename T>
 struct Cfg {
-    static constexpr int W = 8, STAGES = 6, TILE = kTileBytes;      // 192 KB of cache rows in flight per SM
+    static constexpr int W = 12, STAGES = 6, TILE = kTileBytes;      // 192 KB of cache rows in flight per SM; 12 consumer warps
 };
 template <>
 struct Cfg<Fp8E4M3> {
-    static constexpr int W = 12, STAGES = 12, TILE = kTileBytesFp8;  // 192 KB in 12 slots, 12 consumer warps
+    static constexpr int W = 16, STAGES = 12, TILE = kTileBytesFp8;  // 192 KB in 12 slots, 16 consumer warps
 };
 constexpr int MAX_IV = 4;                  // tiles per value item
 constexpr int ITEM_SLOTS = 8;              // value items whose tile partials may be open in one CTA
