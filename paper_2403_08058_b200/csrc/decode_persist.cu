@@ -52,6 +52,7 @@ struct Cfg<Fp8E4M3> {
 constexpr int MAX_IV = 4;                  // tiles per value item
 constexpr int ITEM_SLOTS = 8;              // value items whose tile partials may be open in one CTA
 constexpr int TABLE_CAP = 2048;            // heads whose cluster id is cached in shared memory
+constexpr int LATE_ITEMS = 2;              // the last LATE_ITEMS items per CTA are claimed only when the producer is free
 constexpr long long TIMEOUT_CYCLES = 2000000000ll;
 
 struct TileMeta {
@@ -390,12 +391,18 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             int next = ok ? atomicAdd(work_counter, 1) : n_items;
             while (ok && next < n_items) {
                 const int item = next;
-                next = atomicAdd(work_counter, 1);
+                // The next claim is fetched while this item streams -- except near the end of the item list,
+                // where a claimed but unstarted item on a slow SM is work a faster one could have taken.
+                const bool ahead = item < n_items - LATE_ITEMS * ncta;
+                if (ahead) next = atomicAdd(work_counter, 1);
                 const int head = item / P.nVi, chunk = item % P.nVi;
                 const int tile0 = chunk * P.IV;
                 const int b_item = RAGGED ? head / H : 0;
                 const int ntiles = min(P.IV, tiles_of(b_item) - tile0);
-                if (RAGGED && ntiles <= 0) continue;  // the request is shorter: this item does not exist
+                if (RAGGED && ntiles <= 0) {  // the request is shorter: this item does not exist
+                    if (!ahead) next = atomicAdd(work_counter, 1);
+                    continue;
+                }
                 const int islot = n_open % ITEM_SLOTS;
                 ++n_open;
                 ok = word_wait(&sm.item_free[islot], 1, abort_flag);  // the slot's previous item is fully reduced
@@ -407,6 +414,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                     ok = issue(vc + ((size_t)head * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
                                (uint32_t)tile_rows(b_item, tile) * G::ROW_BYTES, m);
                 }
+                if (!ahead) next = atomicAdd(work_counter, 1);
             }
             // The claim that comes back with the largest id is the last one of the launch: every CTA has started
             // (and read the launch count) by then, so the count can move on for the next launch.
