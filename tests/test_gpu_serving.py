@@ -140,10 +140,11 @@ def test_inplace_compaction_refuses_unordered_reps():
 
 
 @pytest.mark.parametrize("fn_name", ["chai_prefill_attention_from", "chai_prefill_attention_simt_from"])
-@pytest.mark.parametrize("T,q_start", [(300, 5), (300, 128), (300, 131), (64, 5), (129, 128), (640, 257)])
-def test_prefill_from_q_start(fn_name, T, q_start):
+@pytest.mark.parametrize("T,q_start,D", [(300, 5, 128), (300, 128, 128), (300, 131, 128), (64, 5, 128), (129, 128, 128),
+                                         (640, 257, 128), (300, 5, 64), (300, 131, 64)])
+def test_prefill_from_q_start(fn_name, T, q_start, D):
     """Rows from q_start on equal the full clustered prefill; earlier rows of the output are not written."""
-    B, H, k, D = 2, 6, 2, 128
+    B, H, k = 2, 6, 2
     r = synth.batch_partitions(B, H, k, "uneven", T, 79, q_start)
     g = torch.Generator().manual_seed(T + q_start)
     q = (torch.randn(B, H, T, D, generator=g) * 2.0).to(torch.bfloat16)
