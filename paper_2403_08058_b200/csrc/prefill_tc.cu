@@ -16,8 +16,9 @@
 // (TMEM lane quadrant = warp index mod 4; warps 2..5 take columns 0..63 of a tile, warps 6..9
 // columns 64..127); warps 10..13 = epilogue (O / l -> bf16 -> global) of the previous unit while
 // the next one computes; warp 14 = issuer of the P V batches.
-// head_dim 64 is a second instantiation: a tile is one 64-column block (in the first half of the same 32 KB
-// slots), the accumulators have 64 columns, and the P V instructions have N = 64 (one member) or 128 (two).
+// head_dim 64 is a second instantiation: a tile is one 64-column block (two members' V tiles share a 32 KB
+// slot), the accumulators have 64 columns, a work item carries up to four members, and one P V instruction of
+// N = 64 x members serves them all.
 // Every mbarrier wait is bounded: on expiry the CTA records CHAI_ERR_TIMEOUT in the workspace
 // status word, skips the rest of its work, frees its tensor memory and returns.
 #include <cuda.h>
@@ -39,7 +40,8 @@ namespace tc {
 
 constexpr int BM = 128;            // query rows per CTA
 constexpr int BN = 128;            // keys per tile
-constexpr int G = 2;               // member heads per CTA
+constexpr int G = 2;               // V tile slots per key tile: two 128-wide tiles, or four 64-wide ones (two per slot)
+constexpr int GMAX = 4;            // member heads per work item at most (head_dim 64; two with head_dim 128)
 constexpr int KST = 2;             // K tile stages (tile kt uses stage kt & 1)
 constexpr int VST = 2 * G;         // V tile slots: tile kt uses slots (kt & 1) * G + g
 constexpr int TILE_BYTES = BN * 128 * 2;       // 32 KB: a tile slot; a 128 x 128 bf16 tile fills it with two 64-column boxes,
@@ -57,12 +59,12 @@ constexpr int OFF_Q = 0;
 constexpr int OFF_K = OFF_Q + TILE_BYTES;
 constexpr int OFF_V = OFF_K + KST * TILE_BYTES;
 constexpr int OFF_BAR = OFF_V + VST * TILE_BYTES;
-constexpr int NUM_BARS = 36;
+constexpr int NUM_BARS = 38;
 constexpr int OFF_XCH = OFF_BAR + 8 * NUM_BARS + 16;               // after the barriers and the tmem slot / abort word
 constexpr int XCH_BYTES = 2 * BM * 4;                              // row maxima exchanged between the two halves
 constexpr int OFF_LSUM = OFF_XCH + XCH_BYTES;                      // row sums handed to the epilogue warps
 constexpr int OFF_ITEM = OFF_LSUM + 2 * BM * 4;                    // two work-item descriptors + one for the epilogue
-constexpr int ITEM_BYTES = 3 * 32;
+constexpr int ITEM_BYTES = 3 * 48;
 constexpr int OFF_PREFIX = OFF_ITEM + ITEM_BYTES;                  // running sum of groups per request
 constexpr int MAX_B = 64;                                          // requests per launch on this path
 // No alignment slack: the dynamic shared memory of a kernel without static shared memory starts right
@@ -81,7 +83,7 @@ struct Bars {
     uint32_t base;
     __device__ __forceinline__ uint32_t q_full() const { return base; }
     __device__ __forceinline__ uint32_t q_empty() const { return base + 8; }
-    __device__ __forceinline__ uint32_t o_free(int g) const { return g == 0 ? base + 16 : base + 8 * 35; }  // per member
+    __device__ __forceinline__ uint32_t o_free(int g) const { return g == 0 ? base + 16 : base + 8 * (34 + g); }  // per member
     __device__ __forceinline__ uint32_t p_full() const { return base + 24; }
     __device__ __forceinline__ uint32_t item_full(int i) const { return base + 8 * (4 + i); }
     __device__ __forceinline__ uint32_t item_empty(int i) const { return base + 8 * (6 + i); }
@@ -99,18 +101,20 @@ struct Bars {
         return base + 8 * (19 + ((quad * 2 + half) * 2 + (tile & 1)));
     }
 };
-static_assert(NUM_BARS == 36, "barrier count");
+static_assert(NUM_BARS == 38, "barrier count");
 
 // One unit of work, published by the producer to the other roles through shared memory.
-struct Item {
+template <int GM>
+struct ItemT {
     int n_kv;        // key tiles to walk; 0 = zero-fill item (unresolved heads); -1 = no more work
-    int n_members;   // heads in this group (1..G)
+    int n_members;   // heads in this group (1..GM)
     int q0;          // first query row of the tile
     int q_plane;     // b * H + representative head
     int k_plane;     // b * k + cluster
-    int o_plane[G];  // b * H + member head
-    int pad;
+    int o_plane[GM]; // b * H + member head
+    int pad[GM == 2 ? 1 : 3];
 };
+static_assert(sizeof(ItemT<2>) == 32 && sizeof(ItemT<4>) == 48, "item descriptors");
 
 // Persistent kernel: one CTA per SM walks work items (request, member group, query tile) handed out
 // by an atomic counter in descending order of cost.  While the softmax warps finish one item, the
@@ -127,7 +131,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     constexpr int LOAD_BYTES = BN * HD * 2;  // bytes one tile copy brings
     // stride between the 64-column blocks an MN-major V operand walks: the two halves of a 128-wide tile, or
     // (head_dim 64, two members in one instruction) the single blocks of two neighbouring slots
-    constexpr int V_LBO = HD == 128 ? HALF_BYTES : TILE_BYTES;
+    constexpr int V_LBO = HALF_BYTES;        // (with head_dim 64 the members' single blocks lie 16 KB apart, two per slot)
+    constexpr int GM = HD == 128 ? 2 : 4;    // member heads per work item
+    using Item = ItemT<GM>;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = smem_raw;
@@ -148,8 +154,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         mbar_init(bar.q_empty(), 1);
         // Barriers that a whole role signals count warps, not threads: the lanes of a warp meet first and one
         // lane arrives (hundreds of arrivals on one barrier word serialise and cost more than the work between them).
-        mbar_init(bar.o_free(0), EPILOGUE_WARPS);
-        mbar_init(bar.o_free(1), EPILOGUE_WARPS);
+        for (int g = 0; g < GMAX; ++g) mbar_init(bar.o_free(g), EPILOGUE_WARPS);
         mbar_init(bar.epi_full(), SOFTMAX_WARPS);
         mbar_init(bar.epi_empty(), EPILOGUE_WARPS);
         mbar_init(bar.s_free(), SOFTMAX_WARPS);
@@ -228,10 +233,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 }
                 const int qt = cur.qt, b = cur.b;
                 const GroupEntry e = cur.e;
-                const int n_members = min(e.n, G);
+                const int n_members = min(e.n, GM);
                 item.q0 = qt * BM;
                 item.n_members = n_members;
-                for (int g = 0; g < G; ++g) item.o_plane[g] = b * H + e.heads[g < n_members ? g : 0];
+                for (int g = 0; g < GM; ++g) item.o_plane[g] = b * H + e.heads[g < n_members ? g : 0];
                 if (e.cluster < 0) {                       // unresolved heads: zero rows, nothing to load
                     item.n_kv = 0;
                     item.q_plane = item.k_plane = 0;
@@ -247,8 +252,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 item.k_plane = b * k + e.cluster;
                 mbar_arrive(bar.item_full(is));
                 const int q_plane = item.q_plane, k_plane = item.k_plane, q0 = item.q0;
-                int v_plane[G];
-                for (int g = 0; g < G; ++g) v_plane[g] = item.o_plane[g];
+                int v_plane[GM];
+                for (int g = 0; g < GM; ++g) v_plane[g] = item.o_plane[g];
                 // Q: wait until the previous item's last S = Q K^T has been computed
                 ok = mbar_wait(bar.q_empty(), (qi & 1) ^ 1, abort_flag);
                 if (!ok) break;
@@ -272,7 +277,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (!ok) break;
                     mbar_expect_tx(bar.v_full(ts), n_members * LOAD_BYTES);
                     for (int g = 0; g < n_members; ++g)
-                        tma_load_4d(sbase + OFF_V + (ts * G + g) * TILE_BYTES, &map_v, j * BN, v_plane[g], bar.v_full(ts));
+                        tma_load_4d(sbase + OFF_V + ts * G * TILE_BYTES + g * LOAD_BYTES, &map_v, j * BN, v_plane[g], bar.v_full(ts));
                     if (j == 0) resolve(nxt);  // two tiles are on their way: time to look at the claim's answer
                 }
                 kt += n_kv;
@@ -289,7 +294,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // streams goes through an mbarrier, and tcgen05.commit tracks the issuing thread's own MMAs, so the
         // streams need no program order between them.  Each warp walks its loop as a whole, which keeps the
         // control flow and the descriptor arithmetic warp-uniform; one elected lane issues.
-        constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc_n(true, HD), IDESC_PV2 = make_idesc_n(true, 2 * HD);
+        constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc_n(true, HD);
         auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
         auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_polling(b, parity, abort_flag)); };
         const bool qk_role = warp == 1;
@@ -342,24 +347,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (!ok) break;
                     const uint32_t p_addr = tmem_base + P_COL0 + ts * 64;  // P buffer of this tile
                     const bool reuse = j == 0 && qi > 0;  // the accumulators still hold the previous item's output
-                    if (n_members == G && G == 2 && !reuse) {
-                        // Both members at once: their V tiles lie side by side in shared memory (four 64-column
-                        // blocks at one stride) and so do their accumulators in tensor memory, so one N = 256
-                        // instruction per 16 keys does the work of two N = 128 ones and reads P once.
+                    if (n_members > 1 && !reuse) {
+                        // All members at once: their V tiles lie side by side in shared memory (64-column blocks
+                        // at one stride) and so do their accumulators in tensor memory, so one instruction of
+                        // N = head_dim x members per 16 keys does the work of one per member and reads P once.
                         tc_fence_after();
                         if (elect_one()) {
                             const uint32_t d = tmem_base + O_COL0;
                             const uint32_t vb = v_lo + (ts * G) * (TILE_BYTES >> 4);
+                            const uint32_t idesc_all = make_idesc_n(true, (unsigned)(HD * n_members));
 #pragma unroll
                             for (int s = 0; s < BN / 16; ++s)
-                                tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV2, (j > 0 || s > 0) ? 1u : 0u);
+                                tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), idesc_all, (j > 0 || s > 0) ? 1u : 0u);
                             tc_commit(bar.pv_done(ts));
                         }
                         __syncwarp();
                         continue;
                     }
 #pragma unroll
-                    for (int g = 0; g < G; ++g) {
+                    for (int g = 0; g < GM; ++g) {
                         if (g >= n_members) break;
                         // each member's accumulator is released by the epilogue warps on its own
                         if (reuse && !wait_all(bar.o_free(g), (qi - 1) & 1)) {
@@ -369,7 +375,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         tc_fence_after();
                         if (elect_one()) {
                             const uint32_t d = tmem_base + O_COL0 + g * HD;
-                            const uint32_t vb = v_lo + (ts * G + g) * (TILE_BYTES >> 4);
+                            const uint32_t vb = v_lo + ((ts * G * TILE_BYTES + g * LOAD_BYTES) >> 4);
 #pragma unroll
                             for (int s = 0; s < BN / 16; ++s)  // 16 keys per step: 8 TMEM columns of P, 2048 bytes of V
                                 tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV, (j > 0 || s > 0) ? 1u : 0u);
@@ -433,9 +439,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 vis = max(0, min(vis - cbase, 64));
                 // the whole tile is visible to every row unless it is the diagonal tile or runs past T
                 const bool full_tile = col0 + BN <= T_len && (!causal || col0 + BN - 1 <= q0);
-                tc_ld32(s_addr + cbase, r);
-                tc_ld32(s_addr + cbase + 32, r + 32);
-                tc_wait_ld();
+                tc_ld64_wait(s_addr + cbase, r);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar.s_free());  // the scores are in registers: the next S = Q K^T may overwrite the buffer
@@ -531,9 +535,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     tc_fence_after();
                     for (int g = 0; g < n_members; ++g) {  // this thread rescales its half of the columns of each O
                         const uint32_t o_addr = lane_addr + O_COL0 + g * HD + half * (HD / 2);
-                        tc_ld32(o_addr, r);
-                        if constexpr (HD == 128) tc_ld32(o_addr + 32, r + 32);
-                        tc_wait_ld();
+                        if constexpr (HD == 128) tc_ld64_wait(o_addr, r);
+                        else tc_ld32_wait(o_addr, r);
 #pragma unroll
                         for (int i = 0; i < HD / 2; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * corr);
                         tc_st32(o_addr, r);
@@ -591,15 +594,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 __nv_bfloat16* orow = out + ((size_t)ep.o_plane[g] * T_len + row_abs) * HD;
 #pragma unroll
                 for (int ch = 0; ch < HD / 64; ++ch) {  // 64 columns per round: two loads in flight
-                    tc_ld32(lane_addr + O_COL0 + g * HD + ch * 64, r);
-                    tc_ld32(lane_addr + O_COL0 + g * HD + ch * 64 + 32, r + 32);
-                    tc_wait_ld();
+                    tc_ld64_wait(lane_addr + O_COL0 + g * HD + ch * 64, r);
                     if (ch == HD / 64 - 1) {  // this row of the member's accumulator is in registers
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) {
                             mbar_arrive(bar.o_free(g));
-                            if (ep.n_members == 1) mbar_arrive(bar.o_free(1));  // keep the unused barrier's phase in step
+                            if (g == ep.n_members - 1)  // keep the phases of the unused members' barriers in step
+                                for (int x = ep.n_members; x < GM; ++x) mbar_arrive(bar.o_free(x));
                         }
                     }
                     if (row_abs >= q_start && row_abs < T_len) {  // rows before q_start belong to the caller
@@ -691,7 +693,7 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
                  CHAI_ERR_CUDA, "chai_prefill_attention: cuTensorMapEncodeTiled failed");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
-    rc = prefill_run_plan(membership, reps, B, H, k, tc::G, ws, s);
+    rc = prefill_run_plan(membership, reps, B, H, k, D == 128 ? 2 : 4, ws, s);
     if (rc != CHAI_OK) return rc;
     const PrefillLayout L = prefill_layout(B, H);
     // per device: SM count, and the kernel's opt-in to its shared-memory size

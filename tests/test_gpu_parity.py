@@ -485,6 +485,23 @@ def test_prefill_long_prompt_sampled_rows():
         assert_parity(got[:, :, lo:hi], ref[:, :, lo:hi], "bf16", f"long prompt rows {lo}..{hi}")
 
 
+def test_prefill_head_dim_64_full_size_sampled_rows():
+    """Workload 5's shape with 64-wide heads (groups of four members on the tensor-core kernel): run-to-run
+    bitwise identical, first and last rows against the oracle."""
+    B, H, k, T, D = 4, 32, 8, 2048, 64
+    case = prefill_inputs(21, B, H, T, k, "bf16", "even", D=D, peaked=4.0)
+    d = to_dev(case)
+    out = chai.chai_prefill_attention(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"])
+    out2 = chai.chai_prefill_attention(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"])
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    q, kr, v, mem, reps = case["q"], case["k_rep"], case["v"], case["membership"], case["reps"]
+    head = orc.cha_attention(q[:, :, :192], kr[:, :, :192], v[:, :, :192], mem, reps, case["scale"], True)
+    assert_parity(out[:, :, :192].float().cpu().numpy(), head, "bf16", "D 64 first rows")
+    tail = orc.cha_attention(q[:, :, T - 64:], kr, v, mem, reps, case["scale"], True)
+    assert_parity(out[:, :, T - 64:].float().cpu().numpy(), tail, "bf16", "D 64 last rows")
+
+
 def test_prefill_flow_features_kmeans_compaction_attention():
     """Workload 5's whole flow at reduced length: both sides derive the membership themselves."""
     case = synth.prefill_case(seed=1, B=2, T=192, peaked=4.0)
