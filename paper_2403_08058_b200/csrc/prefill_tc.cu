@@ -276,8 +276,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     ok = mbar_wait(bar.pv_done(ts), ((n >> 1) & 1) ^ 1, abort_flag);  // the tile's V slots are free
                     if (!ok) break;
                     mbar_expect_tx(bar.v_full(ts), n_members * LOAD_BYTES);
-                    for (int g = 0; g < n_members; ++g)
-                        tma_load_4d(sbase + OFF_V + ts * G * TILE_BYTES + g * LOAD_BYTES, &map_v, j * BN, v_plane[g], bar.v_full(ts));
+#pragma unroll
+                    for (int g = 0; g < GM; ++g)  // (member arrays are indexed statically: they stay in registers)
+                        if (g < n_members) tma_load_4d(sbase + OFF_V + ts * G * TILE_BYTES + g * LOAD_BYTES, &map_v, j * BN, v_plane[g], bar.v_full(ts));
                     if (j == 0) resolve(nxt);  // two tiles are on their way: time to look at the claim's answer
                 }
                 kt += n_kv;
@@ -294,7 +295,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // streams goes through an mbarrier, and tcgen05.commit tracks the issuing thread's own MMAs, so the
         // streams need no program order between them.  Each warp walks its loop as a whole, which keeps the
         // control flow and the descriptor arithmetic warp-uniform; one elected lane issues.
-        constexpr uint32_t IDESC_QK = make_idesc(false), IDESC_PV = make_idesc_n(true, HD);
+        constexpr uint32_t IDESC_QK = make_idesc(false);
         auto desc = [](uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; };
         auto wait_all = [&](uint32_t b, uint32_t parity) { return __all_sync(0xffffffffu, mbar_wait_polling(b, parity, abort_flag)); };
         const bool qk_role = warp == 1;
@@ -347,42 +348,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (!ok) break;
                     const uint32_t p_addr = tmem_base + P_COL0 + ts * 64;  // P buffer of this tile
                     const bool reuse = j == 0 && qi > 0;  // the accumulators still hold the previous item's output
-                    if (n_members > 1 && !reuse) {
-                        // All members at once: their V tiles lie side by side in shared memory (64-column blocks
-                        // at one stride) and so do their accumulators in tensor memory, so one instruction of
-                        // N = head_dim x members per 16 keys does the work of one per member and reads P once.
-                        tc_fence_after();
-                        if (elect_one()) {
-                            const uint32_t d = tmem_base + O_COL0;
-                            const uint32_t vb = v_lo + (ts * G) * (TILE_BYTES >> 4);
-                            const uint32_t idesc_all = make_idesc_n(true, (unsigned)(HD * n_members));
+                    // An item's first tile overwrites the accumulators, which still hold the previous item's output
+                    // until the epilogue warps have drained them (each member's is released on its own).
+                    if (reuse)
+                        for (int g = 0; g < n_members && ok; ++g) ok = wait_all(bar.o_free(g), (qi - 1) & 1);
+                    if (!ok) break;
+                    // All members at once: their V tiles lie side by side in shared memory (64-column blocks at
+                    // one stride) and so do their accumulators in tensor memory, so one instruction of
+                    // N = head_dim x members per 16 keys serves them all and reads P once.
+                    tc_fence_after();
+                    if (elect_one()) {
+                        const uint32_t d = tmem_base + O_COL0;
+                        const uint32_t vb = v_lo + (ts * G) * (TILE_BYTES >> 4);
+                        const uint32_t idesc_all = make_idesc_n(true, (unsigned)(HD * n_members));
 #pragma unroll
-                            for (int s = 0; s < BN / 16; ++s)
-                                tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), idesc_all, (j > 0 || s > 0) ? 1u : 0u);
-                            tc_commit(bar.pv_done(ts));
-                        }
-                        __syncwarp();
-                        continue;
+                        for (int s = 0; s < BN / 16; ++s)  // 16 keys per step: 8 TMEM columns of P, 2048 bytes of each V block
+                            tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), idesc_all, (j > 0 || s > 0) ? 1u : 0u);
+                        tc_commit(bar.pv_done(ts));
                     }
-#pragma unroll
-                    for (int g = 0; g < GM; ++g) {
-                        if (g >= n_members) break;
-                        // each member's accumulator is released by the epilogue warps on its own
-                        if (reuse && !wait_all(bar.o_free(g), (qi - 1) & 1)) {
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after();
-                        if (elect_one()) {
-                            const uint32_t d = tmem_base + O_COL0 + g * HD;
-                            const uint32_t vb = v_lo + ((ts * G * TILE_BYTES + g * LOAD_BYTES) >> 4);
-#pragma unroll
-                            for (int s = 0; s < BN / 16; ++s)  // 16 keys per step: 8 TMEM columns of P, 2048 bytes of V
-                                tc_mma_ts(d, p_addr + s * 8, desc(hi_v, vb + s * (2048 >> 4)), IDESC_PV, (j > 0 || s > 0) ? 1u : 0u);
-                            if (g + 1 == n_members) tc_commit(bar.pv_done(ts));
-                        }
-                        __syncwarp();
-                    }
+                    __syncwarp();
                 }
             }
             ++it;
@@ -416,7 +400,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const int row_abs = q0 + row;
             if (n_kv == 0) {  // unresolved heads: zero rows
                 if (row_abs >= q_start && row_abs < T_len)
-                    for (int g = 0; g < n_members; ++g) {
+#pragma unroll
+                    for (int g = 0; g < GM; ++g) {
+                        if (g >= n_members) break;
                         uint4* o = reinterpret_cast<uint4*>(out + ((size_t)item.o_plane[g] * T_len + row_abs) * HD + half * (HD / 2));
 #pragma unroll
                         for (int u = 0; u < HD / 16; ++u) o[u] = make_uint4(0, 0, 0, 0);
@@ -590,7 +576,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const int row_abs = ep.q0 + row;
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const uint64_t inv2 = pack2(inv, inv);
-            for (int g = 0; g < ep.n_members; ++g) {
+#pragma unroll
+            for (int g = 0; g < GM; ++g) {
+                if (g >= ep.n_members) break;
                 __nv_bfloat16* orow = out + ((size_t)ep.o_plane[g] * T_len + row_abs) * HD;
 #pragma unroll
                 for (int ch = 0; ch < HD / 64; ++ch) {  // 64 columns per round: two loads in flight
