@@ -502,6 +502,27 @@ def test_prefill_head_dim_64_full_size_sampled_rows():
     assert_parity(out[:, :, T - 64:].float().cpu().numpy(), tail, "bf16", "D 64 last rows")
 
 
+@pytest.mark.parametrize("B,H,k,T,D,kind", [
+    (4, 32, 3, 3000, 64, "even"),      # clusters of 10-11 heads: items of three and four members, T not a tile multiple
+    (3, 32, 5, 2048, 64, "uneven"),
+    (4, 32, 3, 3000, 128, "even"),
+    (2, 16, 2, 1500, 128, "uneven"),
+])
+def test_prefill_is_bitwise_repeatable_with_full_groups(B, H, k, T, D, kind):
+    """Large clusters fill every work item with the most members the kernel takes; a work item's accumulators
+    are reused from item to item.  Four runs must agree bit for bit, and the last rows must match the oracle."""
+    case = prefill_inputs(40 + k, B, H, T, k, "bf16", kind, D=D, peaked=4.0)
+    d = to_dev(case)
+    outs = [chai.chai_prefill_attention(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"])
+            for _ in range(4)]
+    torch.cuda.synchronize()
+    for o in outs[1:]:
+        assert torch.equal(outs[0], o)
+    q, kr, v, mem, reps = case["q"], case["k_rep"], case["v"], case["membership"], case["reps"]
+    tail = orc.cha_attention(q[:1, :, T - 32:], kr[:1], v[:1], mem[:1], reps[:1], case["scale"], True)
+    assert_parity(outs[0][:1, :, T - 32:].float().cpu().numpy(), tail, "bf16", "last rows")
+
+
 def test_prefill_flow_features_kmeans_compaction_attention():
     """Workload 5's whole flow at reduced length: both sides derive the membership themselves."""
     case = synth.prefill_case(seed=1, B=2, T=192, peaked=4.0)
