@@ -24,6 +24,7 @@
 #include <cuda.h>
 #include <stdlib.h>
 #include <string.h>
+#include <type_traits>
 
 #include "prefill_plan.cuh"
 #include "tc_ptx.cuh"
@@ -437,21 +438,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     for (int i = 0; i < 64; ++i)
                         if (i >= vis) r[i] = 0xff800000u;
                 }
-                // own half-row maximum (eight independent chains)
+                // Own half-row maximum, eight independent chains.  On an item's first tile it is taken here, ahead of
+                // the exponentials, which need the reference it gives; on every later tile the exponentials run
+                // first against the current reference (see below) and the maxima are taken along with them, in
+                // the issue slots the special-function unit leaves free.
                 float mxa[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) mxa[c] = -INFINITY;
-#pragma unroll
-                for (int i = 0; i < 64; i += 2) mxa[(i >> 1) & 7] = max3(mxa[(i >> 1) & 7], __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
                 // The two threads of a row must agree on one reference.  Each rounds its half-row maximum up to
                 // bf16 and publishes it (slots alternate with the tile's parity); both take the larger of the two
                 // rounded values, a reference slightly above the true maximum being as good.
-                const __nv_bfloat16 mx_up =
-                    __float2bfloat16_ru(max3(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
+                __nv_bfloat16 mx_up;
                 __nv_bfloat16* xs = xch + (kt & 1) * 2 * BM;
-                xs[half * BM + row] = mx_up;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar.pair(quad, half, kt));
+                auto publish = [&]() {
+                    mx_up = __float2bfloat16_ru(max3(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
+                    xs[half * BM + row] = mx_up;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar.pair(quad, half, kt));
+                };
                 float m_new = m_used, corr = 1.f;
                 // Meet the partner: reference of this tile, by the lazy-rescale rule (it moves only when the
                 // maximum outgrew it by more than 2^8).
@@ -468,7 +472,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // probabilities against reference m, rounded to bf16, two per 32-bit column: the layout of an A
                 // operand in tensor memory (score columns 64 h + c map to column 32 h + c / 2 of the tile's P
                 // buffer); they leave in chunks of 16 as they are ready.  Returns the row's partial sum.
-                auto emit = [&](float m) -> float {
+                auto emit = [&](float m, auto with_max) -> float {
                     const float m_ref = m == -INFINITY ? 0.f : m;
                     const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m_ref, -m_ref);
                     uint64_t acc01 = 0ull, acc23 = 0ull;  // two packed pairs of partial row sums
@@ -482,6 +486,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             unpack2(fma2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), sc2, nm2), x0, x1);
                             unpack2(fma2(pack2(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3])), sc2, nm2), x2, x3);
                             const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+                            if constexpr (decltype(with_max)::value) {
+                                mxa[(i >> 1) & 7] = max3(mxa[(i >> 1) & 7], __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                                mxa[((i >> 1) + 1) & 7] = max3(mxa[((i >> 1) + 1) & 7], __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                            }
                             acc01 = add2(acc01, pack2(p0, p1));
                             acc23 = add2(acc23, pack2(p2, p3));
                             __nv_bfloat162 pa = __floats2bfloat162_rn(p0, p1), pb = __floats2bfloat162_rn(p2, p3);
@@ -503,12 +511,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // After an item's first tile the reference hardly ever moves, so the tile is computed against
                 // the current reference at once, without waiting for the partner's maximum; the meeting follows
                 // the arithmetic, and only if some row's reference did move is the tile computed and stored again.
-                const bool speculate = j > 0;
-                float ls = 0.f;
-                if (speculate) ls = emit(m_used);
-                ok = meet();
-                if (!ok) break;
-                if (!speculate || __any_sync(0xffffffffu, m_new != m_used)) ls = emit(m_new);
+                float ls;
+                if (j > 0) {
+                    ls = emit(m_used, std::true_type{});
+                    publish();
+                    ok = meet();
+                    if (!ok) break;
+                    if (__any_sync(0xffffffffu, m_new != m_used)) ls = emit(m_new, std::false_type{});
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 64; i += 2) mxa[(i >> 1) & 7] = max3(mxa[(i >> 1) & 7], __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                    publish();
+                    ok = meet();
+                    if (!ok) break;
+                    ls = emit(m_new, std::false_type{});
+                }
                 l_run = l_run * corr + ls;
                 m_used = m_new;
                 // Rescaling touches the O accumulators, so the previous tile's P V must be complete first; a warp
