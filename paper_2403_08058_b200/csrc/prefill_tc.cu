@@ -52,6 +52,7 @@ constexpr int SOFTMAX_WARPS = 8;    // two per TMEM lane quadrant: each thread o
 constexpr int EPILOGUE_WARPS = 4;   // one thread per query row: O / l -> bf16 -> global while the next item computes
 constexpr int PV_WARP = 2 + SOFTMAX_WARPS + EPILOGUE_WARPS;  // the warp that issues the P V batches
 constexpr int THREADS = 96 + (SOFTMAX_WARPS + EPILOGUE_WARPS) * 32;
+constexpr float REF_WINDOW = 32.f;   // log2 of how far a row's maximum may be from the softmax reference
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t S_COL0 = 0, P_COL0 = 128, O_COL0 = 256;  // S at 0..127, P buffers at 128 + 64 i, O_g at 256 + 128 g
 
@@ -411,7 +412,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 ++it;
                 continue;
             }
-            float m_used = -INFINITY, l_run = 0.f;
+            // The reference the exponentials are taken against starts at 0 for every row and moves only when a
+            // tile's row maximum leaves a window of 2^+-32 around it (first tile) or outgrows it by 2^32 (later
+            // tiles): a common factor 2^-m cancels in P V / l, bf16 and fp32 keep their relative precision at
+            // any magnitude, and 2^32 times the row's largest term is far from fp32's range for any number of
+            // keys.  For scores of ordinary size the reference therefore never moves, no tile waits for its
+            // maxima before its exponentials, and no accumulator is ever rescaled; the reference is a function
+            // of the row's own scores alone, so results do not depend on how work was scheduled.
+            float m_used = 0.f, l_run = 0.f;
             for (int j = 0; j < n_kv && ok; ++j, ++kt) {
                 const int sb = kt & 1;
                 ok = __all_sync(0xffffffffu, mbar_wait(bar.qk_done(sb), (kt >> 1) & 1, abort_flag));
@@ -438,10 +446,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     for (int i = 0; i < 64; ++i)
                         if (i >= vis) r[i] = 0xff800000u;
                 }
-                // Own half-row maximum, eight independent chains.  On an item's first tile it is taken here, ahead of
-                // the exponentials, which need the reference it gives; on every later tile the exponentials run
-                // first against the current reference (see below) and the maxima are taken along with them, in
-                // the issue slots the special-function unit leaves free.
+                // Own half-row maximum, eight independent chains, taken along with the exponentials (which run
+                // against the current reference at once, see below) in the issue slots the special-function unit
+                // leaves free.
                 float mxa[8];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) mxa[c] = -INFINITY;
@@ -457,15 +464,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (lane == 0) mbar_arrive(bar.pair(quad, half, kt));
                 };
                 float m_new = m_used, corr = 1.f;
-                // Meet the partner: reference of this tile, by the lazy-rescale rule (it moves only when the
-                // maximum outgrew it by more than 2^8).
+                // Meet the partner: reference of this tile, by the lazy-rescale rule above.
                 auto meet = [&]() -> bool {
                     if (!__all_sync(0xffffffffu, mbar_wait(bar.pair(quad, half ^ 1, kt), (kt >> 1) & 1, abort_flag))) return false;
                     const float mx = fmaxf(__bfloat162float(mx_up), __bfloat162float(xs[(half ^ 1) * BM + row]));
                     const float m_tile = mx * scale_log2;
-                    if (m_tile > m_used + 8.f) {
+                    if (m_tile > m_used + REF_WINDOW || (j == 0 && m_tile < m_used - REF_WINDOW)) {
                         m_new = m_tile;
-                        corr = fast_exp2(m_used - m_new);  // 0 on the first tile (m_used = -inf)
+                        corr = j == 0 ? 1.f : fast_exp2(m_used - m_new);  // (nothing has been accumulated before the first tile)
                     }
                     return true;
                 };
@@ -508,24 +514,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (!ok) break;
                     tc_fence_after();
                 }
-                // After an item's first tile the reference hardly ever moves, so the tile is computed against
-                // the current reference at once, without waiting for the partner's maximum; the meeting follows
-                // the arithmetic, and only if some row's reference did move is the tile computed and stored again.
-                float ls;
-                if (j > 0) {
-                    ls = emit(m_used, std::true_type{});
-                    publish();
-                    ok = meet();
-                    if (!ok) break;
-                    if (__any_sync(0xffffffffu, m_new != m_used)) ls = emit(m_new, std::false_type{});
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 64; i += 2) mxa[(i >> 1) & 7] = max3(mxa[(i >> 1) & 7], __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-                    publish();
-                    ok = meet();
-                    if (!ok) break;
-                    ls = emit(m_new, std::false_type{});
-                }
+                // The reference hardly ever moves, so the tile is computed against the current reference at once,
+                // without waiting for the partner's maximum; the meeting follows the arithmetic, and only if some
+                // row's reference did move is the tile computed and stored again.
+                float ls = emit(m_used, std::true_type{});
+                publish();
+                ok = meet();
+                if (!ok) break;
+                if (__any_sync(0xffffffffu, m_new != m_used)) ls = emit(m_new, std::false_type{});
                 l_run = l_run * corr + ls;
                 m_used = m_new;
                 // Rescaling touches the O accumulators, so the previous tile's P V must be complete first; a warp

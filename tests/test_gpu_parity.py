@@ -523,6 +523,34 @@ def test_prefill_is_bitwise_repeatable_with_full_groups(B, H, k, T, D, kind):
     assert_parity(outs[0][:1, :, T - 32:].float().cpu().numpy(), tail, "bf16", "last rows")
 
 
+@pytest.mark.parametrize("D", [128, 64])
+@pytest.mark.parametrize("shape", ["all_far_below", "all_far_above", "growing", "shrinking"])
+def test_prefill_scores_far_from_the_softmax_reference(D, shape):
+    """Scores whose size forces the kernel's running softmax reference to move: all of a row's scores far below
+    or far above zero, and scores that grow (or fall) by hundreds of powers of two along the keys.  One
+    coordinate of Q and K carries the offset, so the oracle sees the same stored values."""
+    B, H, k, T = 2, 8, 3, 700
+    case = prefill_inputs(60, B, H, T, k, "bf16", "uneven", D=D, peaked=2.0)
+    q, kr = case["q"].clone(), case["k_rep"].clone()
+    unit = float(np.sqrt(D)) / 1.4427           # a product of this size moves a score by one power of two
+    ramp = torch.linspace(0.0, 1.0, T)
+    if shape == "all_far_below":                # every score about 2^-100 relative to the reference at zero
+        q[..., 0], kr[..., 0] = 10.0, -10.0 * unit
+    elif shape == "all_far_above":
+        q[..., 0], kr[..., 0] = 10.0, 10.0 * unit
+    elif shape == "growing":                    # later keys outweigh earlier ones by up to 2^300
+        q[..., 0] = 10.0
+        kr[..., 0] = (30.0 * unit * ramp).to(torch.bfloat16)
+    else:                                       # the first keys dominate; later tiles lie far below the reference
+        q[..., 0] = 10.0
+        kr[..., 0] = (-30.0 * unit * ramp).to(torch.bfloat16)
+    case["q"], case["k_rep"] = q, kr
+    got = run_prefill(case)
+    assert np.isfinite(got).all()
+    ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], case["scale"], True)
+    assert_parity(got, ref, "bf16", f"scores {shape}, D {D}")
+
+
 def test_prefill_flow_features_kmeans_compaction_attention():
     """Workload 5's whole flow at reduced length: both sides derive the membership themselves."""
     case = synth.prefill_case(seed=1, B=2, T=192, peaked=4.0)
