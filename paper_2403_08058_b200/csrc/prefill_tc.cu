@@ -573,7 +573,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int row = quad * 32 + lane;
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
         const float* lsum = reinterpret_cast<const float*>(smem + OFF_LSUM);
-        uint32_t r[64];
         for (int ei = 0;; ++ei) {
             bool ok = __all_sync(0xffffffffu, mbar_wait(bar.epi_full(), ei & 1, abort_flag));
             if (!ok) break;
@@ -589,37 +588,46 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const int row_abs = ep.q0 + row;
             const float inv = l > 0.f ? 1.f / l : 0.f;
             const uint64_t inv2 = pack2(inv, inv);
+            // The accumulators leave in pieces of 32 columns through two register buffers: the load of the next
+            // piece is in flight while the current one is scaled, rounded and stored, and a member's
+            // accumulator is released as soon as its last piece is in registers.
+            constexpr int NSUB = HD / 32;
+            const int n_sub = ep.n_members * NSUB;
+            uint32_t ra[32], rb[32];
+            tc_ld32(lane_addr + O_COL0, ra);
+            tc_wait_ld32(ra);
 #pragma unroll
-            for (int g = 0; g < GM; ++g) {
-                if (g >= ep.n_members) break;
-                __nv_bfloat16* orow = out + ((size_t)ep.o_plane[g] * T_len + row_abs) * HD;
-#pragma unroll
-                for (int ch = 0; ch < HD / 64; ++ch) {  // 64 columns per round: two loads in flight
-                    tc_ld64_wait(lane_addr + O_COL0 + g * HD + ch * 64, r);
-                    if (ch == HD / 64 - 1) {  // this row of the member's accumulator is in registers
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) {
-                            mbar_arrive(bar.o_free(g));
-                            if (g == ep.n_members - 1)  // keep the phases of the unused members' barriers in step
-                                for (int x = ep.n_members; x < GM; ++x) mbar_arrive(bar.o_free(x));
-                        }
-                    }
-                    if (row_abs >= q_start && row_abs < T_len) {  // rows before q_start belong to the caller
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            uint32_t w[8];
-#pragma unroll
-                            for (int x = 0; x < 8; ++x) {
-                                float y0, y1;
-                                unpack2(mul2(pack2(__uint_as_float(r[16 * u + 2 * x]), __uint_as_float(r[16 * u + 2 * x + 1])), inv2), y0, y1);
-                                __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
-                                w[x] = *reinterpret_cast<uint32_t*>(&pk);
-                            }
-                            st_global_32B(orow + ch * 64 + u * 16, w);
-                        }
+            for (int c = 0; c < GM * NSUB; ++c) {
+                if (c >= n_sub) break;
+                uint32_t* cur = (c & 1) ? rb : ra;
+                uint32_t* nxt = (c & 1) ? ra : rb;
+                const int g = c / NSUB, sc = c % NSUB;
+                if (c + 1 < n_sub) tc_ld32(lane_addr + O_COL0 + (c + 1) * 32, nxt);  // (members' accumulators are contiguous)
+                if (sc == NSUB - 1) {  // this row of the member's accumulator is in registers
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(bar.o_free(g));
+                        if (g == ep.n_members - 1)  // keep the phases of the unused members' barriers in step
+                            for (int x = ep.n_members; x < GM; ++x) mbar_arrive(bar.o_free(x));
                     }
                 }
+                if (row_abs >= q_start && row_abs < T_len) {  // rows before q_start belong to the caller
+                    __nv_bfloat16* orow = out + ((size_t)ep.o_plane[g] * T_len + row_abs) * HD + sc * 32;
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int x = 0; x < 8; ++x) {
+                            float y0, y1;
+                            unpack2(mul2(pack2(__uint_as_float(cur[16 * u + 2 * x]), __uint_as_float(cur[16 * u + 2 * x + 1])), inv2), y0, y1);
+                            __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+                            w[x] = *reinterpret_cast<uint32_t*>(&pk);
+                        }
+                        st_global_32B(orow + u * 16, w);
+                    }
+                }
+                if (c + 1 < n_sub) tc_wait_ld32(nxt);
             }
         }
     }
