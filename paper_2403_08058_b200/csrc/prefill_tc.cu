@@ -6,8 +6,8 @@
 // S = Q K^T and O_g += P V_g are tcgen05.mma instructions with fp32 accumulators in tensor memory
 // (one S buffer of 128 columns, two P buffers of 64 columns, one O accumulator of 128 columns per
 // member: 512 columns).  The softmax threads read S from tensor memory, keep the running reference
-// and sum of the softmax (rescaling O only when the maximum grew by more than 2^8, which leaves the
-// result exact because p and l use the same reference) and write P as bf16 back into tensor memory,
+// and sum of the softmax (the reference starts at 0 and moves, with a rescaling of O, only when a row maximum
+// leaves a window of 2^32 around it, which leaves the result exact because p and l use the same reference) and write P as bf16 back into tensor memory,
 // from where it is the A operand of the P V product; the probabilities of a cluster are therefore
 // computed once and applied to every member's values (Fig. 3(b)).
 //
