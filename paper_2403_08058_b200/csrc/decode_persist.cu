@@ -732,8 +732,8 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                     for (int e = 0; e < DPL; ++e) o[e] += __ldcg(src + (size_t)i * D + e);
                     ll += __ldcg(lsrc + i);
                 }
-#pragma unroll
                 const float vscale = P.v_scale ? __ldg(P.v_scale + head) : 1.f;  // fp8 values carry a scale per plane
+#pragma unroll
                 for (int e = 0; e < DPL; ++e)  // (an empty context has no probabilities: the output is zero)
                     outp[(size_t)head * D + lane * DPL + e] = from_float<TQ>(ll > 0.f ? o[e] / ll * vscale : 0.f);
             }
