@@ -145,6 +145,17 @@ struct Vec16<Fp8E4M3> {
             f[4 * i + 3] = b.y;
         }
     }
+    // the same 16 values as eight fp16 pairs (every e4m3 value is an fp16 value): h[j] = elements 2j, 2j + 1
+    __device__ __forceinline__ static void unpack_h2(const uint4& r, __half2* h) {
+        const unsigned w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __half2_raw lo = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(w[i] & 0xffffu), __NV_E4M3);
+            const __half2_raw hi = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(w[i] >> 16), __NV_E4M3);
+            h[2 * i] = *reinterpret_cast<const __half2*>(&lo);
+            h[2 * i + 1] = *reinterpret_cast<const __half2*>(&hi);
+        }
+    }
 };
 
 // Streaming 16-byte load that does not pollute L1 (cache data are read exactly once).

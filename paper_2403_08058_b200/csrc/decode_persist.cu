@@ -26,6 +26,7 @@
 // flags go up.  The softmax is the exact two-pass form; all sums are taken in a fixed order, so results
 // are bitwise repeatable whatever the schedule.  Every wait is bounded; on expiry the CTA records
 // CHAI_ERR_TIMEOUT, stops consuming and returns.
+#include <type_traits>
 #include <stdlib.h>
 
 #include <atomic>
@@ -467,7 +468,29 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 for (int x = 0; x < G::EPV / Vec16<TQ>::N; ++x)
                     Vec16<TQ>::unpack(*reinterpret_cast<const uint4*>(qsrc + x * Vec16<TQ>::N), qf + x * Vec16<TQ>::N);
             }
-            const float kscale = P.k_scale ? P.scale * __ldg(P.k_scale + plane) : P.scale;  // fp8 keys carry a scale per plane
+            float kscale = P.k_scale ? P.scale * __ldg(P.k_scale + plane) : P.scale;  // fp8 keys carry a scale per plane
+            // fp8 keys: as on the value side, the conversions to fp32 bound the path, so a lane's 16 products are
+            // formed and summed as fp16 pairs.  The query slice is brought below 16 in size by a power of two
+            // (exact; undone in the score's scale), so that eight products with e4m3 values (at most 448) cannot
+            // overflow fp16.
+            __half2 qh[8];
+            if constexpr (std::is_same<T, Fp8E4M3>::value) {
+                static_assert(G::EPV == 16, "sixteen fp8 values per lane and row");
+                float qmax = 0.f;
+#pragma unroll
+                for (int e = 0; e < G::EPV; ++e) qmax = fmaxf(qmax, fabsf(qf[e]));
+#pragma unroll
+                for (int o = G::LPR / 2; o >= 1; o >>= 1) qmax = fmaxf(qmax, __shfl_xor_sync(0xffffffffu, qmax, o));
+                float fac = 1.f;
+                if (qmax > 16.f && qmax < INFINITY) {
+                    int ex;
+                    frexpf(qmax, &ex);          // qmax = m * 2^ex with m in [0.5, 1)
+                    fac = ldexpf(1.f, 4 - ex);  // qmax * fac in [8, 16)
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) qh[j] = __floats2half2_rn(qf[2 * j] * fac, qf[2 * j + 1] * fac);
+                kscale /= fac;
+            }
             unsigned long long cnt_seen = 0;
             if (lane == 0) cnt_seen = plane_peek(P.pcnt + plane);
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
@@ -488,15 +511,25 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                     for (int ii = 0; ii < G::LPR; ++ii) {
                         const int row = (bt * G::LPR + ii) * G::RPW + sub;
                         const uint4 raw = *reinterpret_cast<const uint4*>(data + row * G::ROW_BYTES + part * 16);
-                        float kf[G::EPV];
-                        Vec16<T>::unpack(raw, kf);
-                        float s0 = 0.f, s1 = 0.f;
+                        if constexpr (std::is_same<T, Fp8E4M3>::value) {
+                            __half2 kh[8];
+                            Vec16<T>::unpack_h2(raw, kh);
+                            __half2 s2 = __hmul2(qh[0], kh[0]);
 #pragma unroll
-                        for (int e = 0; e < G::EPV; e += 2) {
-                            s0 = fmaf(qf[e], kf[e], s0);
-                            s1 = fmaf(qf[e + 1], kf[e + 1], s1);
+                            for (int j = 1; j < 8; ++j) s2 = __hfma2(qh[j], kh[j], s2);
+                            const float2 f = __half22float2(s2);
+                            v[ii] = f.x + f.y;
+                        } else {
+                            float kf[G::EPV];
+                            Vec16<T>::unpack(raw, kf);
+                            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                            for (int e = 0; e < G::EPV; e += 2) {
+                                s0 = fmaf(qf[e], kf[e], s0);
+                                s1 = fmaf(qf[e + 1], kf[e + 1], s1);
+                            }
+                            v[ii] = s0 + s1;
                         }
-                        v[ii] = s0 + s1;
                     }
 #pragma unroll
                     for (int o = G::LPR / 2; o >= 1; o >>= 1) {
@@ -619,7 +652,45 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             if (ok && have_p) {
                 {
                     const unsigned char* data = sm.ring[slot];
-                    if (rows == G::TR) {
+                    if constexpr (std::is_same<T, Fp8E4M3>::value) {
+                        // fp8 values: the per-element conversions to fp32 are what bounds this path, so the
+                        // products are formed and summed as fp16 pairs (every e4m3 value is an fp16 value; a
+                        // probability is at most 1 and an e4m3 value at most 448, so FLUSH of them cannot
+                        // overflow) and join the fp32 sums every FLUSH rows.
+                        constexpr int FLUSH = 8;
+                        static_assert(G::EPV == 16, "sixteen fp8 values per lane and row");
+                        __half2 hacc[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) hacc[j] = __float2half2_rn(0.f);
+                        auto flush = [&]() {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float2 f = __half22float2(hacc[j]);
+                                acc[2 * j] += f.x;
+                                acc[2 * j + 1] += f.y;
+                                hacc[j] = __float2half2_rn(0.f);
+                            }
+                        };
+#pragma unroll
+                        for (int u = 0; u < G::PV; ++u) {
+#pragma unroll
+                            for (int i = 0; i < G::IT; ++i) {
+                                const int r32 = i * G::RPW + sub;
+                                const float pr = __shfl_sync(0xffffffffu, pv[u], r32);
+                                const int row = u * 32 + r32;
+                                if (row < rows) {  // never touch stale bytes of a ragged last tile (its probabilities are 0 anyway)
+                                    const uint4 raw = *reinterpret_cast<const uint4*>(data + row * G::ROW_BYTES + part * 16);
+                                    __half2 vh[8];
+                                    Vec16<T>::unpack_h2(raw, vh);
+                                    const __half2 ph = __float2half2_rn(pr);
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) hacc[j] = __hfma2(ph, vh[j], hacc[j]);
+                                }
+                                if ((u * G::IT + i) % FLUSH == FLUSH - 1) flush();
+                            }
+                        }
+                        if ((G::PV * G::IT) % FLUSH != 0) flush();
+                    } else if (rows == G::TR) {
 #pragma unroll
                         for (int u = 0; u < G::PV; ++u) {
 #pragma unroll
