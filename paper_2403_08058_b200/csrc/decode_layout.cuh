@@ -13,11 +13,16 @@ constexpr int kTileBytes = 32768;     // persistent kernel: one ring slot = TR c
 constexpr int kTileBytesFp8 = 16384;  // ... of half the size for one-byte elements (same number of elements per tile)
 inline int decode_tile_bytes(int dtype) { return dtype == CHAI_FP8_E4M3 ? kTileBytesFp8 : kTileBytes; }
 
+// Long contexts: a head's item partials are added in groups of this many, then the group sums (a fixed tree,
+// so the result does not depend on who adds).
+constexpr int kCombineGroup = 16;
+
 struct DecodeLayout {
     int CK, CV, nK, nV;  // split kernels: rows per key / value chunk and chunks per plane
     int TR;              // persistent kernel: rows per 16 KB tile
     int capK, capV;      // entries per plane reserved for chunk maxima / partials (either implementation)
-    size_t off_counters, off_flags, off_scores, off_cmax, off_pmax, off_lpart, off_opart, total;
+    int capG;            // groups of kCombineGroup value items per head (tickets of the two-level combine)
+    size_t off_counters, off_gcnt, off_flags, off_scores, off_cmax, off_pmax, off_lpart, off_opart, total;
 };
 
 // off_flags: 64-bit words of the persistent kernel: [0] carries the launch token once the layer's first key tile
@@ -41,6 +46,9 @@ inline bool decode_layout(int B, int H, int k, int T, int D, int dtype, DecodeLa
     size_t off = sizeof(WsHeader);
     L->off_counters = off;
     off = round_up(off + sizeof(int) * (size_t)B * H, 256);
+    L->capG = (L->capV + kCombineGroup - 1) / kCombineGroup;
+    L->off_gcnt = off;
+    off = round_up(off + sizeof(int) * (size_t)B * H * L->capG, 256);
     L->off_flags = off;
     off = round_up(off + sizeof(unsigned long long) * (2 * (size_t)B * k + 2), 256);
     L->off_scores = off;

@@ -53,6 +53,8 @@ struct Cfg<Fp8E4M3> {
 constexpr int MAX_IV = 4;                  // tiles per value item
 constexpr int ITEM_SLOTS = 8;              // value items whose tile partials may be open in one CTA
 constexpr int TABLE_CAP = 2048;            // heads whose cluster id is cached in shared memory
+// groups a head's n items are first added in (1 = all at once)
+__host__ __device__ inline int combine_groups(int n) { return n > 4 * kCombineGroup ? (n + kCombineGroup - 1) / kCombineGroup : 1; }
 constexpr int LATE_ITEMS = 2;              // the last LATE_ITEMS items per CTA are claimed only when the producer is free
 constexpr long long TIMEOUT_CYCLES = 2000000000ll;
 
@@ -94,6 +96,8 @@ struct Params {
     void* out;
     WsHeader* hdr;
     int* counters;               // tickets, one per head
+    int* gcnt;                   // tickets of the groups of kCombineGroup items, capG per head
+    int capG;
     unsigned long long* flags;   // [0]: the layer's first key tile is done
     unsigned long long* pflag;   // per key plane: all its tiles are done and pmax holds its largest score
     unsigned long long* pcnt;    // per key plane: finished tiles of this launch (launch tag in the upper bits)
@@ -251,6 +255,83 @@ struct Ring {
 // skipping of tiles beyond a request's end compile away (the streaming loops are sensitive to every
 // instruction on the producer thread and in the per-tile consumer chain).
 // T = element type of the caches, TQ = element type of the queries and the output (they differ for fp8 caches).
+// Long contexts.  A head with hundreds of value items would have its item partials added by one warp in one go: a
+// long chain of dependent L2 round trips (measured: 58 us of a 227 us call at T = 131072, H = 32).  Instead the
+// items are added in groups of kCombineGroup by whichever warp completes a group (tickets, nobody waits; the
+// group's sum replaces its first item's partial), and the warp that completes the head's last group adds the
+// group sums: a fixed tree, so the result does not depend on who adds what.  Called by a whole warp that has
+// just published item `chunk` of `head`; `done` is set in the warp that completed the head, with the head's
+// sums (lane l holds columns l * DPL ..).  Kept out of line: the short-context path stays as it was.
+template <int DPL>
+struct GroupedSum {
+    float o[DPL];
+    float l;
+    bool done;
+};
+template <int D>
+__device__ __noinline__ GroupedSum<D / 32> combine_grouped(float* opart, float* lpart, int* gcnt, int* counters, int nVi,
+                                                           int capG, int head, int chunk, int n_chunks, int lane) {
+    constexpr int DPL = D / 32;
+    GroupedSum<DPL> r;
+    r.done = false;
+    r.l = 0.f;
+#pragma unroll
+    for (int e = 0; e < DPL; ++e) r.o[e] = 0.f;
+    const float* src = opart + (size_t)head * nVi * D + lane * DPL;
+    const float* lsrc = lpart + (size_t)head * nVi;
+    // adds `count` partials, `stride` slots apart, starting at slot `first`, in order, eight loads in flight
+    auto add_partials = [&](int first, int count, int stride) {
+#pragma unroll
+        for (int e = 0; e < DPL; ++e) r.o[e] = 0.f;
+        r.l = 0.f;
+        int i = 0;
+        for (; i + 8 <= count; i += 8) {
+            float t8[8][DPL], l8[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const size_t slot = (size_t)first + (size_t)(i + u) * stride;
+#pragma unroll
+                for (int e = 0; e < DPL; ++e) t8[u][e] = __ldcg(src + slot * D + e);
+                l8[u] = __ldcg(lsrc + slot);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+#pragma unroll
+                for (int e = 0; e < DPL; ++e) r.o[e] += t8[u][e];
+                r.l += l8[u];
+            }
+        }
+        for (; i < count; ++i) {
+            const size_t slot = (size_t)first + (size_t)i * stride;
+#pragma unroll
+            for (int e = 0; e < DPL; ++e) r.o[e] += __ldcg(src + slot * D + e);
+            r.l += __ldcg(lsrc + slot);
+        }
+    };
+    const int n_groups = combine_groups(n_chunks);
+    const int grp = chunk / kCombineGroup;
+    const int in_grp = min(kCombineGroup, n_chunks - grp * kCombineGroup);
+    int ticket = 0;
+    if (lane == 0) ticket = atomicAdd(&gcnt[(size_t)head * capG + grp], 1);
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    if (ticket != in_grp - 1) return r;
+    __threadfence();
+    add_partials(grp * kCombineGroup, in_grp, 1);
+    float* gp = opart + ((size_t)head * nVi + (size_t)grp * kCombineGroup) * D;
+#pragma unroll
+    for (int e = 0; e < DPL; ++e) gp[lane * DPL + e] = r.o[e];
+    if (lane == 0) lpart[(size_t)head * nVi + (size_t)grp * kCombineGroup] = r.l;
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) ticket = atomicAdd(&counters[head], 1);
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    if (ticket != n_groups - 1) return r;
+    __threadfence();
+    add_partials(0, n_groups, kCombineGroup);
+    r.done = true;
+    return r;
+}
+
 template <typename T, typename TQ, int D, bool RAGGED>
 __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kernel(const Params P) {
     using G = Geom<T, D>;
@@ -566,7 +647,12 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 if (tile == 0 && live) {
                     const int c = plane % k;
                     for (int h = lane; h < H; h += 32)
-                        if (cluster_of(b, h) == c) P.counters[(size_t)b * H + h] = 0;
+                        if (cluster_of(b, h) == c) {
+                            P.counters[(size_t)b * H + h] = 0;
+                            const int n_groups = combine_groups(items_of(b));
+                            if (n_groups > 1)
+                                for (int gq = 0; gq < n_groups; ++gq) P.gcnt[((size_t)b * H + h) * P.capG + gq] = 0;
+                        }
                 }
                 __syncwarp();
                 unsigned done = 0;
@@ -771,10 +857,20 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             if (lane == 0) P.lpart[(size_t)head * P.nVi + chunk] = l;
             __threadfence();
             __syncwarp();
+            const int n_chunks = items_of(b);  // items this head really has
+            if (combine_groups(n_chunks) > 1) {  // long context: the items are added group by group (see combine_grouped)
+                const GroupedSum<D / 32> gs = combine_grouped<D>(P.opart, P.lpart, P.gcnt, P.counters, P.nVi, P.capG, head, chunk, n_chunks, lane);
+                if (gs.done) {
+                    const float vscale = P.v_scale ? __ldg(P.v_scale + head) : 1.f;
+#pragma unroll
+                    for (int e = 0; e < D / 32; ++e)
+                        outp[(size_t)head * D + lane * (D / 32) + e] = from_float<TQ>(gs.l > 0.f ? gs.o[e] / gs.l * vscale : 0.f);
+                }
+                continue;
+            }
             int ticket = 0;
             if (lane == 0) ticket = atomicAdd(&P.counters[head], 1);
             ticket = __shfl_sync(0xffffffffu, ticket, 0);
-            const int n_chunks = items_of(b);  // items this head really has
             if (ticket == n_chunks - 1) {  // this warp completed the head: add the item partials in chunk order
                 __threadfence();
 #pragma unroll
@@ -889,6 +985,8 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     P.k_batch_bytes = k_batch_stride * elem_size(dtype);
     P.hdr = reinterpret_cast<WsHeader*>(ws);
     P.counters = reinterpret_cast<int*>(ws + L.off_counters);
+    P.gcnt = reinterpret_cast<int*>(ws + L.off_gcnt);
+    P.capG = L.capG;
     P.flags = reinterpret_cast<unsigned long long*>(ws + L.off_flags);
     P.pflag = P.flags + 2;
     P.pcnt = P.flags + 2 + (size_t)B * k;

@@ -127,6 +127,25 @@ def test_decode_extreme_shapes(B, H, k, T):
         assert_parity(got[b:b + 1], ref, "bf16", f"B {B} H {H} k {k} T {T} request {b}")
 
 
+def test_decode_ragged_long_contexts_mix_one_pass_and_grouped_sums():
+    """Requests of very different lengths in one call: a head's item partials are added in one pass for the
+    short ones and group by group for the long ones (with a last group that is not full); one request is empty."""
+    B, H, k, T = 4, 4, 2, 70001
+    case = synth.decode_layer(2, layer=2, seed=9, device=DEV, B=B, H=H, T=T, k=k, with_k_full=False, peaked=4.0)
+    lens = np.array([T, 40000, 20000, 0], np.int32)
+    seq = torch.as_tensor(lens, device=DEV)
+    ws = chai.new_workspace(chai.chai_decode_workspace_bytes(B, H, k, T, 128, chai.CHAI_BF16), DEV)
+    outs = [chai.chai_decode_attention_ragged(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], seq,
+                                              case["scale"], T_max=T, workspace=ws) for _ in range(2)]
+    torch.cuda.synchronize()
+    assert chai.chai_device_status(ws) == chai.CHAI_OK
+    assert torch.equal(outs[0], outs[1])
+    c = {n: case[n].cpu() for n in ("q", "k_rep", "v", "membership", "reps")}
+    ref = orc.decode_attention_ragged(c["q"], c["k_rep"], c["v"], c["membership"], c["reps"], lens, case["scale"])
+    assert_parity(outs[0].float().cpu().numpy(), ref, "bf16", "ragged long contexts")
+    assert not outs[0][3].float().abs().max().item()  # the empty request's rows are zero
+
+
 def test_decode_bad_membership_is_reported_not_faulted():
     case = synth.decode_layer(2, seed=1, B=2, H=8, T=200, k=4)
     ref = oracle_decode(case)
