@@ -460,13 +460,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 auto publish = [&]() {
                     mx_up = __float2bfloat16_ru(max3(max3(mxa[0], mxa[1], mxa[2]), max3(mxa[3], mxa[4], mxa[5]), fmaxf(mxa[6], mxa[7])));
                     xs[half * BM + row] = mx_up;
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar.pair(quad, half, kt));
                 };
                 float m_new = m_used, corr = 1.f;
                 // Meet the partner: reference of this tile, by the lazy-rescale rule above.
                 auto meet = [&]() -> bool {
-                    if (!__all_sync(0xffffffffu, mbar_wait(bar.pair(quad, half ^ 1, kt), (kt >> 1) & 1, abort_flag))) return false;
+                    // The two warps of a quadrant meet at a named barrier (hardware barrier 1 + quad, 64 threads):
+                    // a fraction of the latency of an mbarrier round trip, once per tile on the path that bounds
+                    // the kernel.  It has no time limit of its own, so a warp that gives up (a bounded wait
+                    // elsewhere ran out: the abort flag is set) arrives here once on its way out, and everyone
+                    // looks at the flag right after the barrier: nobody can be left waiting for a warp that is gone.
+                    asm volatile("bar.sync %0, 64;" ::"r"(quad + 1) : "memory");
+                    if (*abort_flag) return false;
                     const float mx = fmaxf(__bfloat162float(mx_up), __bfloat162float(xs[(half ^ 1) * BM + row]));
                     const float m_tile = mx * scale_log2;
                     if (m_tile > m_used + REF_WINDOW || (j == 0 && m_tile < m_used - REF_WINDOW)) {
@@ -567,6 +571,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(bar.epi_full());
         }
+        if (!ok) asm volatile("bar.arrive %0, 64;" ::"r"(quad + 1) : "memory");  // release a partner that may be waiting to meet
     } else {
         // ---------------- epilogue: O_g / l -> bf16 -> global, one thread per query row ----------------
         const int quad = warp & 3;
