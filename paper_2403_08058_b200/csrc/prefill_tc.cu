@@ -61,7 +61,7 @@ constexpr int OFF_Q = 0;
 constexpr int OFF_K = OFF_Q + TILE_BYTES;
 constexpr int OFF_V = OFF_K + KST * TILE_BYTES;
 constexpr int OFF_BAR = OFF_V + VST * TILE_BYTES;
-constexpr int NUM_BARS = 38;
+constexpr int NUM_BARS = 22;
 constexpr int OFF_XCH = OFF_BAR + 8 * NUM_BARS + 16;               // after the barriers and the tmem slot / abort word
 constexpr int XCH_BYTES = 2 * BM * 4;                              // row maxima exchanged between the two halves
 constexpr int OFF_LSUM = OFF_XCH + XCH_BYTES;                      // row sums handed to the epilogue warps
@@ -85,7 +85,7 @@ struct Bars {
     uint32_t base;
     __device__ __forceinline__ uint32_t q_full() const { return base; }
     __device__ __forceinline__ uint32_t q_empty() const { return base + 8; }
-    __device__ __forceinline__ uint32_t o_free(int g) const { return g == 0 ? base + 16 : base + 8 * (34 + g); }  // per member
+    __device__ __forceinline__ uint32_t o_free(int g) const { return g == 0 ? base + 16 : base + 8 * (18 + g); }  // per member
     __device__ __forceinline__ uint32_t p_full() const { return base + 24; }
     __device__ __forceinline__ uint32_t item_full(int i) const { return base + 8 * (4 + i); }
     __device__ __forceinline__ uint32_t item_empty(int i) const { return base + 8 * (6 + i); }
@@ -96,14 +96,8 @@ struct Bars {
     __device__ __forceinline__ uint32_t epi_full() const { return base + 8 * 16; }
     __device__ __forceinline__ uint32_t epi_empty() const { return base + 8 * 17; }
     __device__ __forceinline__ uint32_t s_free() const { return base + 8 * 18; }
-    // Softmax half `half` of TMEM lane quadrant `quad` has published its row maxima of a tile.  Tiles
-    // alternate between two barriers: the publisher may be a whole tile ahead of the reader (who looks at
-    // the end of its own tile), and one phase bit can tell apart only adjacent phases.
-    __device__ __forceinline__ uint32_t pair(int quad, int half, int tile) const {
-        return base + 8 * (19 + ((quad * 2 + half) * 2 + (tile & 1)));
-    }
 };
-static_assert(NUM_BARS == 38, "barrier count");
+static_assert(NUM_BARS == 22, "barrier count");
 
 // One unit of work, published by the producer to the other roles through shared memory.
 template <int GM>
@@ -161,7 +155,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         mbar_init(bar.epi_empty(), EPILOGUE_WARPS);
         mbar_init(bar.s_free(), SOFTMAX_WARPS);
         mbar_init(bar.p_full(), SOFTMAX_WARPS);
-        for (int i = 0; i < 16; ++i) mbar_init(bar.pair(i >> 2, (i >> 1) & 1, i & 1), 1);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar.item_full(i), 1);
             mbar_init(bar.item_empty(i), 2 + SOFTMAX_WARPS);
