@@ -61,7 +61,7 @@ constexpr int OFF_Q = 0;
 constexpr int OFF_K = OFF_Q + TILE_BYTES;
 constexpr int OFF_V = OFF_K + KST * TILE_BYTES;
 constexpr int OFF_BAR = OFF_V + VST * TILE_BYTES;
-constexpr int NUM_BARS = 22;
+constexpr int NUM_BARS = 23;
 constexpr int OFF_XCH = OFF_BAR + 8 * NUM_BARS + 16;               // after the barriers and the tmem slot / abort word
 constexpr int XCH_BYTES = 2 * BM * 4;                              // row maxima exchanged between the two halves
 constexpr int OFF_LSUM = OFF_XCH + XCH_BYTES;                      // row sums handed to the epilogue warps
@@ -86,7 +86,12 @@ struct Bars {
     __device__ __forceinline__ uint32_t q_full() const { return base; }
     __device__ __forceinline__ uint32_t q_empty() const { return base + 8; }
     __device__ __forceinline__ uint32_t o_free(int g) const { return g == 0 ? base + 16 : base + 8 * (18 + g); }  // per member
-    __device__ __forceinline__ uint32_t p_full() const { return base + 24; }
+    // One arrival per softmax warp and tile; tiles alternate between two barriers.  With a single one, a warp of
+    // one quadrant could arrive for tile kt + 1 while a warp of another quadrant (whose reference moved: it computes
+    // its tile twice and rescales) has not arrived for tile kt -- the scores of tile kt + 1 only need everybody to
+    // have LOADED tile kt -- and complete the wrong phase.  Two tiles ahead is impossible: P(kt + 2) overwrites
+    // P(kt), which waits for the P V of tile kt, which waits for this barrier.
+    __device__ __forceinline__ uint32_t p_full(int i) const { return i == 0 ? base + 24 : base + 8 * 22; }
     __device__ __forceinline__ uint32_t item_full(int i) const { return base + 8 * (4 + i); }
     __device__ __forceinline__ uint32_t item_empty(int i) const { return base + 8 * (6 + i); }
     __device__ __forceinline__ uint32_t k_full(int i) const { return base + 8 * (8 + i); }
@@ -97,7 +102,7 @@ struct Bars {
     __device__ __forceinline__ uint32_t epi_empty() const { return base + 8 * 17; }
     __device__ __forceinline__ uint32_t s_free() const { return base + 8 * 18; }
 };
-static_assert(NUM_BARS == 22, "barrier count");
+static_assert(NUM_BARS == 23, "barrier count");
 
 // One unit of work, published by the producer to the other roles through shared memory.
 template <int GM>
@@ -154,7 +159,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         mbar_init(bar.epi_full(), SOFTMAX_WARPS);
         mbar_init(bar.epi_empty(), EPILOGUE_WARPS);
         mbar_init(bar.s_free(), SOFTMAX_WARPS);
-        mbar_init(bar.p_full(), SOFTMAX_WARPS);
+        mbar_init(bar.p_full(0), SOFTMAX_WARPS);
+        mbar_init(bar.p_full(1), SOFTMAX_WARPS);
         for (int i = 0; i < 2; ++i) {
             mbar_init(bar.item_full(i), 1);
             mbar_init(bar.item_empty(i), 2 + SOFTMAX_WARPS);
@@ -339,7 +345,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             } else {
                 for (int j = 0; j < n_kv && ok; ++j, ++kt) {
                     const int ts = kt & 1;
-                    ok = wait_all(bar.p_full(), kt & 1) && wait_all(bar.v_full(ts), (kt >> 1) & 1);
+                    ok = wait_all(bar.p_full(ts), (kt >> 1) & 1) && wait_all(bar.v_full(ts), (kt >> 1) & 1);
                     if (!ok) break;
                     const uint32_t p_addr = tmem_base + P_COL0 + ts * 64;  // P buffer of this tile
                     const bool reuse = j == 0 && qi > 0;  // the accumulators still hold the previous item's output
@@ -542,7 +548,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tc_wait_st();          // P (and any rescaled O) is in tensor memory
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar.p_full());
+                if (lane == 0) mbar_arrive(bar.p_full(sb));
             }
             // hand the item to the epilogue warps: row sums of both halves and where the output goes
             ok = __all_sync(0xffffffffu, ok && mbar_wait(bar.epi_empty(), (ei & 1) ^ 1, abort_flag));

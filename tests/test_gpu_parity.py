@@ -543,12 +543,12 @@ def test_prefill_is_bitwise_repeatable_with_full_groups(B, H, k, T, D, kind):
 
 
 @pytest.mark.parametrize("D", [128, 64])
-@pytest.mark.parametrize("shape", ["all_far_below", "all_far_above", "growing", "shrinking"])
+@pytest.mark.parametrize("shape", ["all_far_below", "all_far_above", "growing", "shrinking", "growing_in_one_quadrant"])
 def test_prefill_scores_far_from_the_softmax_reference(D, shape):
     """Scores whose size forces the kernel's running softmax reference to move: all of a row's scores far below
     or far above zero, and scores that grow (or fall) by hundreds of powers of two along the keys.  One
     coordinate of Q and K carries the offset, so the oracle sees the same stored values."""
-    B, H, k, T = 2, 8, 3, 700
+    B, H, k, T = 2, 8, 3, 1900
     case = prefill_inputs(60, B, H, T, k, "bf16", "uneven", D=D, peaked=2.0)
     q, kr = case["q"].clone(), case["k_rep"].clone()
     unit = float(np.sqrt(D)) / 1.4427           # a product of this size moves a score by one power of two
@@ -559,6 +559,11 @@ def test_prefill_scores_far_from_the_softmax_reference(D, shape):
         q[..., 0], kr[..., 0] = 10.0, 10.0 * unit
     elif shape == "growing":                    # later keys outweigh earlier ones by up to 2^300
         q[..., 0] = 10.0
+        kr[..., 0] = (30.0 * unit * ramp).to(torch.bfloat16)
+    elif shape == "growing_in_one_quadrant":    # only rows 32..63 of every 128: their warps recompute and rescale tile
+        q[..., 0] = 0.0                         # after tile and fall behind the warps of the other rows
+        rows = torch.arange(T)
+        q[:, :, (rows % 128 >= 32) & (rows % 128 < 64), 0] = 10.0
         kr[..., 0] = (30.0 * unit * ramp).to(torch.bfloat16)
     else:                                       # the first keys dominate; later tiles lie far below the reference
         q[..., 0] = 10.0
