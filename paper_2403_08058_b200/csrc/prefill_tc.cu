@@ -524,14 +524,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 publish();
                 ok = meet();
                 if (!ok) break;
-                if (__any_sync(0xffffffffu, m_new != m_used)) ls = emit(m_new, std::false_type{});
+                const bool moved = __any_sync(0xffffffffu, m_new != m_used);  // some row of this warp changed its reference
+                if (moved) ls = emit(m_new, std::false_type{});
                 l_run = l_run * corr + ls;
                 m_used = m_new;
                 // Rescaling touches the O accumulators, so the previous tile's P V must be complete first; a warp
                 // whose rows all keep their reference (the usual case after the first tiles) has nothing to wait
                 // for.  Skipping the wait cannot confuse the barrier's phase parity: the P V of tile kt - 3 (same
                 // barrier, previous phase) was awaited before P(kt - 1) was written.
-                if (j > 0 && __any_sync(0xffffffffu, corr != 1.f)) {
+                if (j > 0 && moved) {  // (after the first tile a moved reference always comes with a factor other than 1)
                     ok = __all_sync(0xffffffffu, mbar_wait(bar.pv_done((kt - 1) & 1), ((kt - 1) >> 1) & 1, abort_flag));
                     if (!ok) break;
                     tc_fence_after();
