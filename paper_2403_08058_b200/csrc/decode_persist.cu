@@ -199,6 +199,15 @@ __device__ __forceinline__ unsigned plane_arrive(unsigned long long* cnt, unsign
     asm volatile("atom.acq_rel.gpu.global.add.u64 %0, [%1], 1;" : "=l"(prev) : "l"(cnt) : "memory");
     return (unsigned)(prev & 0xffffffull) + 1u;
 }
+// A ticket: an acquire-release increment by one lane.  Release: what the warp's lanes wrote before the __syncwarp()
+// that precedes the call is visible to whoever draws a later ticket; acquire: what earlier ticket holders published
+// is visible to this warp once the ticket has been passed round by a shuffle.  One instruction instead of a
+// device-wide fence (a round trip of its own) before and after a plain atomic.
+__device__ __forceinline__ int ticket_acq_rel(int* counter) {
+    int prev;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(counter) : "memory");
+    return prev;
+}
 // ... and by a whole warp for `n` consecutive flags.
 __device__ __forceinline__ bool flags_wait(const unsigned long long* flags, int n, unsigned long long token, int lane,
                                            volatile int* abort_flag) {
@@ -312,21 +321,18 @@ __device__ __noinline__ GroupedSum<D / 32> combine_grouped(float* opart, float* 
     const int grp = chunk / kCombineGroup;
     const int in_grp = min(kCombineGroup, n_chunks - grp * kCombineGroup);
     int ticket = 0;
-    if (lane == 0) ticket = atomicAdd(&gcnt[(size_t)head * capG + grp], 1);
+    if (lane == 0) ticket = ticket_acq_rel(&gcnt[(size_t)head * capG + grp]);
     ticket = __shfl_sync(0xffffffffu, ticket, 0);
     if (ticket != in_grp - 1) return r;
-    __threadfence();
     add_partials(grp * kCombineGroup, in_grp, 1);
     float* gp = opart + ((size_t)head * nVi + (size_t)grp * kCombineGroup) * D;
 #pragma unroll
     for (int e = 0; e < DPL; ++e) gp[lane * DPL + e] = r.o[e];
     if (lane == 0) lpart[(size_t)head * nVi + (size_t)grp * kCombineGroup] = r.l;
-    __threadfence();
     __syncwarp();
-    if (lane == 0) ticket = atomicAdd(&counters[head], 1);
+    if (lane == 0) ticket = ticket_acq_rel(&counters[head]);
     ticket = __shfl_sync(0xffffffffu, ticket, 0);
     if (ticket != n_groups - 1) return r;
-    __threadfence();
     add_partials(0, n_groups, kCombineGroup);
     r.done = true;
     return r;
@@ -855,8 +861,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
 #pragma unroll
             for (int e = 0; e < DPL; ++e) op[lane * DPL + e] = o[e];
             if (lane == 0) P.lpart[(size_t)head * P.nVi + chunk] = l;
-            __threadfence();
-            __syncwarp();
+            __syncwarp();  // (the ticket below is the release of these stores)
             const int n_chunks = items_of(b);  // items this head really has
             if (combine_groups(n_chunks) > 1) {  // long context: the items are added group by group (see combine_grouped)
                 const GroupedSum<D / 32> gs = combine_grouped<D>(P.opart, P.lpart, P.gcnt, P.counters, P.nVi, P.capG, head, chunk, n_chunks, lane);
@@ -869,10 +874,9 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 continue;
             }
             int ticket = 0;
-            if (lane == 0) ticket = atomicAdd(&P.counters[head], 1);
+            if (lane == 0) ticket = ticket_acq_rel(&P.counters[head]);
             ticket = __shfl_sync(0xffffffffu, ticket, 0);
             if (ticket == n_chunks - 1) {  // this warp completed the head: add the item partials in chunk order
-                __threadfence();
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) o[e] = 0.f;
                 float ll = 0.f;
