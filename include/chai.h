@@ -12,8 +12,14 @@
  *   - All tensor arguments are DEVICE pointers to contiguous row-major arrays
  *     unless the name ends in _host.  Pointers must be 16-byte aligned.
  *   - Ownership: the caller allocates and frees every buffer, including the
- *     workspace.  The library allocates no device memory and keeps no state
- *     between calls other than the text of the last error.
+ *     workspace.  The library allocates no device memory.  State it keeps between
+ *     calls, all of it host-side and safe to reach from several host threads at
+ *     once: the text of the last error (per thread); per device, what the first
+ *     call on that device found out or set up (SM count, cooperative-launch
+ *     support, each kernel's opt-in to its shared-memory size); a process-wide
+ *     counter from which decode launches draw their tokens; the wait limit set by
+ *     chai_set_decode_wait_limit_cycles.  On the device it owns one thing, the
+ *     8 MiB scratch array of chai_decode_attention_static.
  *   - Asynchrony: a call validates its scalar arguments on the host, enqueues its
  *     kernels on `stream` (a cudaStream_t passed as void*) and returns; it never
  *     synchronises, except chai_device_status and chai_decode_attention_host (the
@@ -241,8 +247,10 @@ int chai_decode_attention_host_streams(const void* q_host, void* out_host, void*
  * routine).
  *   - A problem whose scratch (chai_decode_workspace_bytes) exceeds the array is refused with
  *     CHAI_ERR_WORKSPACE and a message that states both sizes.
- *   - The first call on each device looks up the array's device address (the device that is
- *     current at the time of the call); make that first call before any stream capture begins.
+ *   - Every call looks up the array's address on the device that is current at the time of the
+ *     call (nothing is remembered, so a cudaDeviceReset in between does no harm).  The first call
+ *     on a device is the one that loads the library's module there: make it before any stream
+ *     capture begins.
  *   - All calls on a device share the one array, which still holds whatever the previous call left;
  *     the kernels clear the parts that must start at zero.  Two calls that can overlap on the GPU
  *     (different streams without ordering) race on it: order them, or use chai_decode_attention
@@ -258,8 +266,10 @@ int chai_decode_attention_static(const void* q, const void* k_rep, const void* v
  * query rows; decoder-only models attend causally, Section 2).
  *   q [B,H,T,D] (only representative heads' rows are read), k_rep [B,k,T,D],
  *   v [B,H,T,D], out [B,H,T,D];  causal != 0: row i sees keys j <= i.
- * bf16 (D = 128 or 64) runs on the tcgen05 tensor-core kernel; fp32 on the CUDA-core
- * kernel, which chai_prefill_attention_simt selects for any dtype.
+ * bf16 (D = 128 or 64) with a positive, finite scale runs on the tcgen05 tensor-core
+ * kernel; fp32 (and any other scale) on the CUDA-core kernel, a correct but far slower
+ * path (milliseconds where the tensor-core kernel needs a tenth of one), which
+ * chai_prefill_attention_simt selects for any dtype.
  * Errors: CHAI_ERR_INVALID_ARG / CHAI_ERR_WORKSPACE as for decode; CHAI_ERR_UNSUPPORTED for another head_dim or
  * dtype, for H or B above 65535, and when the work list of one request does not fit the planning kernel's
  * 48 KB of shared memory (4 * (H + 3 k + k * ceil(H / 32)) bytes: e.g. H = k = 512 still fits).  Inconsistent
@@ -346,9 +356,20 @@ int chai_decode_attention_fp8(const void* q, const void* k_rep, const void* v, c
                               int H, int k, int T, int T_cap, int D, size_t k_batch_stride, float scale, void* workspace,
                               size_t workspace_bytes, void* stream);
 
-/* Blocking read of the status word a decode/prefill call left in `workspace`
+/* Blocking read of the status a decode/prefill call left in `workspace`
  * (synchronises `stream`).  *status_out receives a chai_status_t. */
 int chai_device_status(const void* workspace, int* status_out, void* stream);
+
+/*
+ * Test hook (no counterpart in the paper).  Every wait inside the persistent decode kernel -- on a
+ * ring slot, a copy, another CTA's flag -- gives up after a number of SM cycles, after which the
+ * launch stops taking work, waits for the copies it has in flight, records CHAI_ERR_TIMEOUT for
+ * chai_device_status and returns; the next launch on the same workspace starts clean.  The limit
+ * is 2e9 cycles (about a second) unless this call changes it for the launches that follow, in
+ * every thread of the process; cycles <= 0 restores the default.  Tests use a limit of a few
+ * cycles to run the give-up path without any fault or hang; production code has no reason to call it.
+ */
+void chai_set_decode_wait_limit_cycles(long long cycles);
 
 const char* chai_status_string(int status);
 const char* chai_last_error(void); /* text of the last CHAI_ERR_CUDA / refusal on this thread */

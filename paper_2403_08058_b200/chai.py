@@ -30,6 +30,7 @@ EXPORTS = [
     "chai_decode_qkv_workspace_bytes", "chai_decode_attention_qkv", "chai_prefill_qkv_workspace_bytes",
     "chai_prefill_attention_qkv", "chai_broadcast_membership", "chai_select_representatives", "chai_cluster_sweep",
     "chai_quantize_cache_fp8", "chai_decode_fp8_workspace_bytes", "chai_decode_attention_fp8",
+    "chai_set_decode_wait_limit_cycles",
 ]
 DECODE_STATIC_SCRATCH_BYTES = 8 << 20   # CHAI_DECODE_STATIC_SCRATCH_BYTES
 
@@ -82,6 +83,8 @@ def load() -> ctypes.CDLL:
         getattr(lib, name).argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, ci, vp, sz, vp]
     lib.chai_decode_attention_static.argtypes = [vp, vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, cf, ci, vp]
     lib.chai_device_status.argtypes = [vp, ctypes.POINTER(ci), vp]
+    lib.chai_set_decode_wait_limit_cycles.argtypes = [ctypes.c_longlong]
+    lib.chai_set_decode_wait_limit_cycles.restype = None
     lib.chai_status_string.argtypes = [ci]
     lib.chai_status_string.restype = ctypes.c_char_p
     lib.chai_last_error.restype = ctypes.c_char_p
@@ -453,6 +456,11 @@ def chai_decode_attention_fp8(q, k_rep8, v8, k_scale, v_scale, membership, reps,
                                             _ptr(membership), _ptr(reps), _ptr(seq_lens), _ptr(out), B, H, k, T, T_cap, D,
                                             stride, scale, _ptr(workspace), workspace.numel(), _stream()))
     return out
+
+
+def chai_set_decode_wait_limit_cycles(cycles: int) -> None:
+    """Test hook: cycle limit of the decode kernel's device-side waits for the launches that follow (<= 0: default)."""
+    load().chai_set_decode_wait_limit_cycles(int(cycles))
 
 
 def chai_device_status(workspace) -> int:

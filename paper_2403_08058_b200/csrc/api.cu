@@ -15,6 +15,10 @@ void set_last_error(const char* fmt, ...) {
     va_end(ap);
 }
 
+// Cycle limit of the decode kernel's device-side waits (see chai_set_decode_wait_limit_cycles).
+static std::atomic<long long> g_decode_wait_limit{kDefaultWaitLimitCycles};
+long long decode_wait_limit_cycles() { return g_decode_wait_limit.load(std::memory_order_relaxed); }
+
 int cuda_fail(cudaError_t e, const char* what) {
     set_last_error("%s: %s", what, cudaGetErrorString(e));
     return CHAI_ERR_CUDA;
@@ -42,15 +46,24 @@ const char* chai_last_error(void) { return chai::g_last_error; }
 
 int chai_version(void) { return 100; }
 
+void chai_set_decode_wait_limit_cycles(long long cycles) {
+    chai::g_decode_wait_limit.store(cycles > 0 ? cycles : chai::kDefaultWaitLimitCycles, std::memory_order_relaxed);
+}
+
 int chai_device_status(const void* workspace, int* status_out, void* stream) {
     CHAI_REQUIRE(workspace && status_out, CHAI_ERR_INVALID_ARG, "chai_device_status: null argument");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int st = 0;
-    cudaError_t e = cudaMemcpyAsync(&st, workspace, sizeof(int), cudaMemcpyDeviceToHost, s);
+    chai::WsHeader h;
+    cudaError_t e = cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, s);
     if (e != cudaSuccess) return chai::cuda_fail(e, "chai_device_status copy");
     e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return chai::cuda_fail(e, "chai_device_status sync");
-    *status_out = st;
+    // A decode launch in which a wait ran out says so with its own token (see WsHeader): that cannot be lost to
+    // the status word's reset by the CTA that owns the launch's first tile, whichever of the two comes first.
+    unsigned long long gave_up, latest;
+    memcpy(&gave_up, &h.pad[chai::kHdrGaveUpToken], 8);
+    memcpy(&latest, &h.pad[chai::kHdrLaunchToken], 8);
+    *status_out = (gave_up != 0 && gave_up == latest) ? (int)CHAI_ERR_TIMEOUT : h.status;
     return CHAI_OK;
 }
 

@@ -7,6 +7,8 @@
 #include <stdint.h>
 #include <stdio.h>
 
+#include <atomic>
+#include <mutex>
 #include <utility>
 
 #include "chai.h"
@@ -22,6 +24,16 @@ struct WsHeader {
     int pad[61];
 };
 static_assert(sizeof(WsHeader) == 256, "workspace header is 256 bytes");
+// Words of pad[] with a fixed meaning.  Decode: pad[0] work counter, pad[8] launch count of the workspace, and two
+// 64-bit launch tokens (8-byte aligned): the token of the latest launch that started or gave up, and the token of
+// the latest launch in which a bounded wait ran out.  Equal and non-zero = the latest launch timed out.  Prefill:
+// pad[0..59] are per-launch work counters, cleared by the planner (both tokens then read 0).
+constexpr int kHdrGaveUpToken = 11, kHdrLaunchToken = 13;
+static_assert((12 + 4 * kHdrGaveUpToken) % 8 == 0 && (12 + 4 * kHdrLaunchToken) % 8 == 0, "token words are 8-byte aligned");
+
+// Every device-side wait is bounded by a cycle count; this is the default (about a second).
+constexpr long long kDefaultWaitLimitCycles = 2000000000ll;
+long long decode_wait_limit_cycles();  // current limit of the decode kernel's waits (api.cu)
 
 void set_last_error(const char* fmt, ...);
 int cuda_fail(cudaError_t e, const char* what);  // records the text, returns CHAI_ERR_CUDA
@@ -29,6 +41,29 @@ int cuda_fail(cudaError_t e, const char* what);  // records the text, returns CH
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline size_t elem_size(int dtype) { return dtype == CHAI_BF16 ? 2 : (dtype == CHAI_FP8_E4M3 ? 1 : 4); }
+
+// Per-device set-up that the first call on a device performs (attribute queries, a kernel's opt-in to its
+// shared-memory size), safe when several host threads make their first call at once: the flag is read with
+// acquire order, the set-up runs under a mutex, and the flag is set only when it succeeded (a failed set-up is
+// tried again by the next call).  What the set-up stored is visible to every thread that sees the flag.
+constexpr int kMaxDevices = 64;
+struct PerDeviceOnce {
+    std::atomic<bool> done[kMaxDevices];
+    std::mutex lock;
+    PerDeviceOnce() {
+        for (auto& d : done) d.store(false, std::memory_order_relaxed);
+    }
+    template <typename F>
+    int run(int dev, F&& setup) {  // setup() returns a chai status
+        std::atomic<bool>& flag = done[dev & (kMaxDevices - 1)];
+        if (flag.load(std::memory_order_acquire)) return CHAI_OK;
+        std::lock_guard<std::mutex> guard(lock);
+        if (flag.load(std::memory_order_relaxed)) return CHAI_OK;
+        const int rc = setup();
+        if (rc == CHAI_OK) flag.store(true, std::memory_order_release);
+        return rc;
+    }
+};
 
 #define CHAI_REQUIRE(cond, code, ...)            \
     do {                                         \
@@ -165,6 +200,15 @@ __device__ __forceinline__ uint4 ld_stream16(const void* p) {
                  : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
                  : "l"(p));
     return r;
+}
+
+// Start of a call that reports through the status word: no error yet, and no launch token that says "gave up"
+// (a fresh workspace may hold anything there, two equal words included).
+__device__ __forceinline__ void reset_status(WsHeader* hdr) {
+    hdr->status = CHAI_OK;
+    hdr->bad_b = -1;
+    hdr->bad_h = -1;
+    *reinterpret_cast<unsigned long long*>(&hdr->pad[kHdrGaveUpToken]) = 0ull;
 }
 
 // Records the first data inconsistency a kernel meets; never traps.

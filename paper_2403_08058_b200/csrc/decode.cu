@@ -68,11 +68,7 @@ decode_scores_kernel(const T* __restrict__ q, const T* __restrict__ k_rep, const
     // housekeeping for the value kernel that follows on the stream: tickets and status word
     if (chunk == 0 && c == 0) {
         for (int h = tid; h < H; h += kDecThreads) counters[(size_t)b * H + h] = 0;
-        if (b == 0 && tid == 0) {
-            hdr->status = CHAI_OK;
-            hdr->bad_b = -1;
-            hdr->bad_h = -1;
-        }
+        if (b == 0 && tid == 0) reset_status(hdr);
     }
     const int r = reps[(size_t)b * k + c];
     if (r < 0 || r >= H) return;  // unused cluster slot: nothing reads its scores
@@ -392,11 +388,6 @@ int chai_decode_attention_host(const void* q_host, void* out_host, void* q_stage
 constexpr size_t kStaticScratchBytes = CHAI_DECODE_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-namespace {
-constexpr int kMaxDevices = 64;
-void* g_static_scratch_ptr[kMaxDevices] = {};  // device address of g_static_scratch, per device
-}  // namespace
-
 int chai_decode_attention_static(const void* q, const void* k_rep, const void* v, const int32_t* membership,
                                  const int32_t* reps, void* out, int B, int H, int k, int T, int T_cap, int D,
                                  float scale, int dtype, void* stream) {
@@ -408,24 +399,19 @@ int chai_decode_attention_static(const void* q, const void* k_rep, const void* v
     CHAI_REQUIRE(D == 64 || D == 128, CHAI_ERR_UNSUPPORTED,
                  "chai_decode_attention_static: head_dim %d (64 or 128 supported)", D);
     DecodeLayout L;
-    decode_layout(B, H, k, T, D, dtype, &L);
+    CHAI_REQUIRE(decode_layout(B, H, k, T, D, dtype, &L), CHAI_ERR_UNSUPPORTED,
+                 "chai_decode_attention_static: no scratch layout for head_dim %d, dtype %d", D, dtype);
     CHAI_REQUIRE(L.total <= kStaticScratchBytes, CHAI_ERR_WORKSPACE,
                  "chai_decode_attention_static: this problem needs %zu bytes of scratch but the built-in array holds "
                  "%zu; use chai_decode_attention with a caller-owned workspace",
                  L.total, kStaticScratchBytes);
-    int dev = -1;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_static: cudaGetDevice");
-    CHAI_REQUIRE(dev >= 0 && dev < kMaxDevices, CHAI_ERR_UNSUPPORTED,
-                 "chai_decode_attention_static: device index %d out of range", dev);
-    // The array's name is only a host-side handle here; kernels need the address it has on the
-    // current device, looked up once per device (benign if two threads race: same value).
-    void* ptr = g_static_scratch_ptr[dev];
-    if (ptr == nullptr) {
-        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
-        if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_static: cudaGetSymbolAddress");
-        g_static_scratch_ptr[dev] = ptr;
-    }
+    // The array's name is only a host-side handle here; kernels need the address it has on the current
+    // device.  It is looked up on every call (a table lookup in the runtime once this device has the
+    // library's module loaded) rather than remembered: an address kept across a cudaDeviceReset would dangle.
+    // The first call on a device is the one that loads the module: make it before any stream capture.
+    void* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (e != cudaSuccess) return cuda_fail(e, "chai_decode_attention_static: cudaGetSymbolAddress");
     // The decode kernels reset the tickets and the status word themselves at the start of every
     // call, so whatever the previous call left in the array does not matter.
     return chai_decode_attention(q, k_rep, v, membership, reps, out, B, H, k, T, T_cap, D, scale, dtype, ptr,

@@ -56,7 +56,18 @@ constexpr int TABLE_CAP = 2048;            // heads whose cluster id is cached i
 // groups a head's n items are first added in (1 = all at once)
 __host__ __device__ inline int combine_groups(int n) { return n > 4 * kCombineGroup ? (n + kCombineGroup - 1) / kCombineGroup : 1; }
 constexpr int LATE_ITEMS = 2;              // the last LATE_ITEMS items per CTA are claimed only when the producer is free
-constexpr long long TIMEOUT_CYCLES = 2000000000ll;
+constexpr long long TIMEOUT_CYCLES = kDefaultWaitLimitCycles;  // bound of the final wait for copies in flight
+
+// Shared by all waiting threads of a CTA: set when some wait ran out (everybody then stops), and the limit in
+// cycles that the launch was given.  Waits receive a pointer to abort_flag and find the limit behind it.
+struct alignas(8) WaitCtl {
+    int abort_flag;
+    int reserved;
+    long long limit;
+};
+__device__ __forceinline__ long long wait_limit(const volatile int* abort_flag) {
+    return reinterpret_cast<const volatile WaitCtl*>(abort_flag)->limit;
+}
 
 struct TileMeta {
     int item;      // value item id (phase V), -1: end of work for the warp that owns this ring position
@@ -78,7 +89,7 @@ struct Smem {
     int item_free[ITEM_SLOTS];  // 1 when the slot may be given to a new item
     int table[TABLE_CAP];
     unsigned ready[TABLE_CAP / 32];  // bit p: every key tile of plane p is known to carry this launch's token
-    int abort_flag;
+    WaitCtl wait;
     int next_pos;               // next ring position a consumer warp may take
     unsigned epoch;             // launch count of this workspace, read once at start
 };
@@ -110,6 +121,7 @@ struct Params {
     int B, H, k, T, T_cap;
     int IV, nVi;                 // tiles per value item, items per head
     float scale;
+    long long wait_limit;        // cycles after which a device-side wait gives up
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -139,7 +151,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > TIMEOUT_CYCLES) {
+        if (clock64() - t0 > wait_limit(abort_flag)) {
             *abort_flag = 1;
             return false;
         }
@@ -153,7 +165,7 @@ __device__ __forceinline__ bool word_wait(const int* word, int want, volatile in
     while (true) {
         if (*w == want) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > TIMEOUT_CYCLES) {
+        if (clock64() - t0 > wait_limit(abort_flag)) {
             *abort_flag = 1;
             return false;
         }
@@ -175,7 +187,7 @@ __device__ __forceinline__ bool flag_wait_one(const unsigned long long* flag, un
             first = false;
         }
         if (*abort_flag) return false;
-        if (clock64() - t0 > TIMEOUT_CYCLES) {
+        if (clock64() - t0 > wait_limit(abort_flag)) {
             *abort_flag = 1;
             return false;
         }
@@ -203,6 +215,14 @@ __device__ __forceinline__ unsigned plane_arrive(unsigned long long* cnt, unsign
 // that precedes the call is visible to whoever draws a later ticket; acquire: what earlier ticket holders published
 // is visible to this warp once the ticket has been passed round by a shuffle.  One instruction instead of a
 // device-wide fence (a round trip of its own) before and after a plain atomic.
+__device__ __forceinline__ unsigned ld_acquire_cta_shared(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"((unsigned)__cvta_generic_to_shared(p)) : "memory");
+    return v;
+}
+__device__ __forceinline__ void or_release_cta_shared(unsigned* p, unsigned bits) {
+    asm volatile("red.release.cta.shared.or.b32 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(p)), "r"(bits) : "memory");
+}
 __device__ __forceinline__ int ticket_acq_rel(int* counter) {
     int prev;
     asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(counter) : "memory");
@@ -225,7 +245,7 @@ __device__ __forceinline__ bool flags_wait(const unsigned long long* flags, int 
             t0 = clock64();
             first = false;
         }
-        const bool give_up = *abort_flag != 0 || clock64() - t0 > TIMEOUT_CYCLES;
+        const bool give_up = *abort_flag != 0 || clock64() - t0 > wait_limit(abort_flag);
         if (__any_sync(0xffffffffu, give_up)) {
             *abort_flag = 1;
             return false;
@@ -323,6 +343,7 @@ __device__ __noinline__ GroupedSum<D / 32> combine_grouped(float* opart, float* 
     int ticket = 0;
     if (lane == 0) ticket = ticket_acq_rel(&gcnt[(size_t)head * capG + grp]);
     ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    __syncwarp();  // what lane 0 acquired with the ticket is ordered before the other lanes' reads of the partials
     if (ticket != in_grp - 1) return r;
     add_partials(grp * kCombineGroup, in_grp, 1);
     float* gp = opart + ((size_t)head * nVi + (size_t)grp * kCombineGroup) * D;
@@ -332,6 +353,7 @@ __device__ __noinline__ GroupedSum<D / 32> combine_grouped(float* opart, float* 
     __syncwarp();
     if (lane == 0) ticket = ticket_acq_rel(&counters[head]);
     ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    __syncwarp();
     if (ticket != n_groups - 1) return r;
     add_partials(0, n_groups, kCombineGroup);
     r.done = true;
@@ -347,7 +369,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
     SmemT& sm = *reinterpret_cast<SmemT*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, ncta = gridDim.x;
-    volatile int* abort_flag = &sm.abort_flag;
+    volatile int* abort_flag = &sm.wait.abort_flag;
     const Ring ring{smem_u32(&sm.full[0]), smem_u32(&sm.empty[0]), smem_u32(&sm.ring[0][0]), (uint32_t)Cfg<T>::TILE};
     const int B = P.B, H = P.H, k = P.k, T_len = P.T;
     const bool use_table = B * H <= TABLE_CAP;
@@ -369,7 +391,8 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             sm.item_free[s] = 1;
         }
         for (int i = 0; i < TABLE_CAP / 32; ++i) sm.ready[i] = 0;
-        sm.abort_flag = 0;
+        sm.wait.abort_flag = 0;
+        sm.wait.limit = P.wait_limit;
         sm.next_pos = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -510,6 +533,17 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             // ---- one end marker per consumer warp ----
             const TileMeta end{-1, 0, 0, 0};
             for (int w = 0; w < W && ok; ++w) ok = issue(nullptr, 0, end);
+            // If the launch gave up, the copies already issued into the ring may still be in flight and nobody will
+            // wait for them: this thread does, for the latest fill of every slot (with the default limit, whatever
+            // limit the launch was given), so that the CTA does not leave while its shared memory is written.
+            if (!ok || *abort_flag) {
+                for (int i = n > STAGES ? n - STAGES : 0; i < n; ++i) {
+                    const uint32_t bar = ring.full(i % STAGES), par = (uint32_t)(i / STAGES) & 1u;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(bar, par) && clock64() - t0 < TIMEOUT_CYCLES) {
+                    }
+                }
+            }
         }
     } else {
         // ------------------------------ consumers: every warp works alone ------------------------------
@@ -646,6 +680,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                     P.hdr->status = CHAI_OK;
                     P.hdr->bad_b = -1;
                     P.hdr->bad_h = -1;
+                    *reinterpret_cast<volatile unsigned long long*>(&P.hdr->pad[kHdrLaunchToken]) = token;
                     *work_counter = 0;
                 }
                 // the warp that owns tile 0 of a plane also clears the tickets of the plane's heads: every value
@@ -712,10 +747,12 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 const size_t plane = (size_t)b * k + c;
                 // all scores of the plane must exist; once seen, remembered per CTA (planes complete in order, so
                 // after the first tiles of phase V this is a shared-memory bit test)
-                const bool cached = plane < TABLE_CAP && ((*reinterpret_cast<volatile unsigned*>(&sm.ready[plane >> 5]) >> (plane & 31)) & 1u);
+                // (the bit is set with release and read with acquire order within the CTA, so a warp that relies on
+                // another warp's wait is ordered after the scores that wait made visible)
+                const bool cached = plane < TABLE_CAP && ((ld_acquire_cta_shared(&sm.ready[plane >> 5]) >> (plane & 31)) & 1u);
                 if (!cached) {
                     ok = flags_wait(P.pflag + plane, 1, token, lane, abort_flag);
-                    if (ok && lane == 0 && plane < TABLE_CAP) atomicOr(&sm.ready[plane >> 5], 1u << (plane & 31));
+                    if (ok && lane == 0 && plane < TABLE_CAP) or_release_cta_shared(&sm.ready[plane >> 5], 1u << (plane & 31));
                 }
                 if (ok && rows > 0) {  // (the only tile of an empty request has no rows: it just passes the ticket on,
                                        //  which the flag wait above has ordered after the ticket's reset)
@@ -876,6 +913,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             int ticket = 0;
             if (lane == 0) ticket = ticket_acq_rel(&P.counters[head]);
             ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            __syncwarp();  // (as above: lane 0's acquire comes before every lane's reads of the partials)
             if (ticket == n_chunks - 1) {  // this warp completed the head: add the item partials in chunk order
 #pragma unroll
                 for (int e = 0; e < DPL; ++e) o[e] = 0.f;
@@ -911,24 +949,38 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
         }
     }
     __syncthreads();
-    if (tid == 0 && sm.abort_flag) atomicExch(&P.hdr->status, CHAI_ERR_TIMEOUT);
+    if (tid == 0 && sm.wait.abort_flag) {
+        // (the status word alone could be reset afterwards by the CTA that owns the launch's first tile)
+        *reinterpret_cast<volatile unsigned long long*>(&P.hdr->pad[kHdrGaveUpToken]) = token;
+        *reinterpret_cast<volatile unsigned long long*>(&P.hdr->pad[kHdrLaunchToken]) = token;
+        atomicExch(&P.hdr->status, CHAI_ERR_TIMEOUT);
+        // A launch that gave up leaves flag words and counters of its token behind.  The launch count moves on
+        // here too (the producer that sees the last claim may never have got there), so that a replay of a
+        // captured graph, whose host token is the same every time, starts from a token nobody has used.
+        atomicAdd(launch_epoch, 1);
+    }
 }
 
 struct DeviceInfo {
     int sms = 0;
     int coop = 0;
-    bool ready = false;
 };
 
-static DeviceInfo& device_info(int dev) {
-    static DeviceInfo info[64];
-    DeviceInfo& d = info[dev & 63];
-    if (!d.ready) {
-        cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaDeviceGetAttribute(&d.coop, cudaDevAttrCooperativeLaunch, dev);
-        d.ready = true;
-    }
-    return d;
+// SM count and cooperative-launch support of a device, queried by the first call on it.
+static int device_info(int dev, DeviceInfo* out) {
+    static PerDeviceOnce once;
+    static DeviceInfo info[kMaxDevices];
+    if (dev < 0 || dev >= kMaxDevices) return CHAI_ERR_UNSUPPORTED;
+    const int rc = once.run(dev, [&]() -> int {
+        DeviceInfo d;
+        if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess)
+            return CHAI_ERR_CUDA;
+        info[dev] = d;
+        return CHAI_OK;
+    });
+    if (rc == CHAI_OK) *out = info[dev];
+    return rc;
 }
 
 template <typename T, typename TQ, int D, bool RAGGED>
@@ -936,17 +988,16 @@ static int launch(const Params& P0, int ncta, int dev, cudaStream_t s) {
     Params P = P0;
     constexpr int THREADS = Cfg<T>::W * 32 + 32;
     const size_t smem = sizeof(Smem<Cfg<T>::STAGES, Cfg<T>::TILE>) + 128;
-    static bool configured_dev[64] = {};  // (one flag array per instantiation)
-    bool& configured = configured_dev[dev & 63];
-    if (!configured) {
+    static PerDeviceOnce once;  // (one per instantiation)
+    const int rc = once.run(dev, [&]() -> int {
         cudaError_t e = cudaFuncSetAttribute(decode_persistent_kernel<T, TQ, D, RAGGED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel shared-memory opt-in");
         int per_sm = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_persistent_kernel<T, TQ, D, RAGGED>, THREADS, smem);
         if (e != cudaSuccess) return cuda_fail(e, "decode_persistent_kernel occupancy query");
-        if (per_sm < 1) return kDecodeNotLaunched;
-        configured = true;
-    }
+        return per_sm < 1 ? kDecodeNotLaunched : CHAI_OK;
+    });
+    if (rc != CHAI_OK) return rc;
     // Cooperative: value tiles wait for flags set by other CTAs, so all CTAs must be resident at once (a plain
     // launch would let two such kernels on different streams starve each other).  Programmatic stream
     // serialisation: the kernel may be scheduled while its predecessor in the stream drains and blocks in
@@ -977,8 +1028,8 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
                              const DecodeLayout& L, cudaStream_t s, const float* k_scale, const float* v_scale) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return kDecodeNotLaunched;
-    const pd::DeviceInfo& info = pd::device_info(dev);
-    if (!info.coop || info.sms <= 0) return kDecodeNotLaunched;
+    pd::DeviceInfo info;
+    if (pd::device_info(dev, &info) != CHAI_OK || !info.coop || info.sms <= 0) return kDecodeNotLaunched;
     const int ncta = info.sms;
     const int tiles = (T + L.TR - 1) / L.TR;
     pd::Params P;
@@ -1011,6 +1062,7 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     P.IV = tiles < pd::MAX_IV ? tiles : pd::MAX_IV;
     P.nVi = (tiles + P.IV - 1) / P.IV;
     P.scale = scale;
+    P.wait_limit = decode_wait_limit_cycles();
     if (tiles > L.capK || P.nVi > L.capV || (long long)B * H * P.nVi > 0x7fffffffll ||
         (long long)B * k * tiles > 0x7fffffffll)  // item and key-tile ids travel as ints
         return kDecodeNotLaunched;

@@ -694,7 +694,9 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
                                            float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
                                            void* stream) {
     using namespace chai;
-    if (dtype != CHAI_BF16 || (D != 128 && D != 64) || B > 60 * tc::MAX_B)
+    // The tensor-core kernel takes a row's largest raw score and scales it afterwards, which is the largest scaled
+    // score only for a positive, finite scale; anything else goes to the CUDA-core kernel, which scales first.
+    if (dtype != CHAI_BF16 || (D != 128 && D != 64) || B > 60 * tc::MAX_B || !(scale > 0.f) || !(scale <= 3.0e38f))
         return chai_prefill_attention_simt_from(q, k_rep, v, membership, reps, out, B, H, k, T, q_start, D, scale, causal,
                                                 dtype, workspace, workspace_bytes, stream);
     int rc = prefill_check_args("chai_prefill_attention", q, k_rep, v, membership, reps, out, B, H, k, T, D, dtype,
@@ -710,13 +712,14 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
     rc = prefill_run_plan(membership, reps, B, H, k, D == 128 ? 2 : 4, ws, s);
     if (rc != CHAI_OK) return rc;
     const PrefillLayout L = prefill_layout(B, H);
-    // per device: SM count, and the kernel's opt-in to its shared-memory size
-    static int sms_of_device[64] = {};
+    // per device, once: SM count, and the kernels' opt-in to their shared-memory size
+    static PerDeviceOnce once;
+    static int sms_of_device[kMaxDevices] = {};
     int dev = 0;
     cudaError_t de = cudaGetDevice(&dev);
     if (de != cudaSuccess) return cuda_fail(de, "prefill_tc_kernel set-up");
-    int& n_sms = sms_of_device[dev & 63];
-    if (n_sms == 0) {
+    CHAI_REQUIRE(dev >= 0 && dev < kMaxDevices, CHAI_ERR_UNSUPPORTED, "chai_prefill_attention: device index %d out of range", dev);
+    rc = once.run(dev, [&]() -> int {
         int count = 0;
         cudaError_t e = cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess)
@@ -724,8 +727,11 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
         if (e == cudaSuccess)
             e = cudaFuncSetAttribute(tc::prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
         if (e != cudaSuccess) return cuda_fail(e, "prefill_tc_kernel set-up");
-        n_sms = count;
-    }
+        sms_of_device[dev] = count;
+        return CHAI_OK;
+    });
+    if (rc != CHAI_OK) return rc;
+    const int n_sms = sms_of_device[dev];
     const int n_qtiles = (T + tc::BM - 1) / tc::BM;
     // one persistent CTA per SM; requests are processed in chunks of MAX_B (the per-request group counts of
     // a chunk are kept in shared memory), each chunk with its own work counter in the workspace header

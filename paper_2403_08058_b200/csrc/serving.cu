@@ -104,9 +104,7 @@ compact_inplace_kernel(uint4* __restrict__ k_cache, const int32_t* __restrict__ 
 
 __global__ void reset_status_kernel(WsHeader* hdr) {
     dependent_grid_sync();
-    hdr->status = CHAI_OK;
-    hdr->bad_b = -1;
-    hdr->bad_h = -1;
+    reset_status(hdr);
 }
 
 }  // namespace chai

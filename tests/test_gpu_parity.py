@@ -21,8 +21,10 @@ def oracle_decode(case, T=None):
                              case["reps"], case["scale"], causal=False)
 
 
-def run_decode(case, T=None, **kw):
+def run_decode(case, T=None, guard=None, **kw):
     d = to_dev(case)
+    if guard is not None:            # output inside guard bands (the workspace always is: see conftest)
+        kw["out"] = guard.empty_like(d["q"])
     out = chai.chai_decode_attention(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"],
                                      T=T or case["T"], **kw)
     torch.cuda.synchronize()
@@ -40,10 +42,10 @@ def test_decode_config1_fp32():
 
 @pytest.mark.parametrize("T", [1, 2, 5, 127, 128, 129, 255, 256, 257, 700])
 @pytest.mark.parametrize("cfg", [1, 2, 3])
-def test_decode_ragged_lengths(cfg, T):
+def test_decode_ragged_lengths(cfg, T, guard):
     """Lengths around the 64/128/256-row chunk edges, capacity larger than the length."""
     case = synth.decode_layer(cfg, layer=T % 7, seed=T, B=2, H=12 if cfg != 1 else 8, T=T, T_cap=T + 3, k=3)
-    got = run_decode(case)
+    got = run_decode(case, guard=guard)
     assert_parity(got, oracle_decode(case), case["dtype"], f"cfg {cfg} T {T}")
 
 
@@ -109,13 +111,13 @@ def test_decode_full_size_layers():
 @pytest.mark.parametrize("B,H,k,T", [(2, 8, 3, 100003),     # long context: hundreds of tiles per plane, ragged tail
                                       (1500, 4, 2, 40),        # many short requests: far more heads than the head table holds
                                       (1, 1, 1, 1)])           # the smallest problem there is
-def test_decode_extreme_shapes(B, H, k, T):
+def test_decode_extreme_shapes(B, H, k, T, guard):
     case = synth.decode_layer(2, layer=1, seed=5, device=DEV, B=B, H=H, T=T, k=k, with_k_full=False, peaked=4.0)
     ws = chai.new_workspace(chai.chai_decode_workspace_bytes(B, H, k, T, 128, chai.CHAI_BF16), DEV)
     out = chai.chai_decode_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"],
-                                     case["scale"], workspace=ws)
+                                     case["scale"], out=guard.empty_like(case["q"]), workspace=ws)
     out2 = chai.chai_decode_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"],
-                                      case["scale"], workspace=ws)
+                                      case["scale"], out=guard.empty_like(case["q"]), workspace=ws)
     torch.cuda.synchronize()
     assert chai.chai_device_status(ws) == chai.CHAI_OK
     assert torch.equal(out, out2)
@@ -127,7 +129,7 @@ def test_decode_extreme_shapes(B, H, k, T):
         assert_parity(got[b:b + 1], ref, "bf16", f"B {B} H {H} k {k} T {T} request {b}")
 
 
-def test_decode_ragged_long_contexts_mix_one_pass_and_grouped_sums():
+def test_decode_ragged_long_contexts_mix_one_pass_and_grouped_sums(guard):
     """Requests of very different lengths in one call: a head's item partials are added in one pass for the
     short ones and group by group for the long ones (with a last group that is not full); one request is empty."""
     B, H, k, T = 4, 4, 2, 70001
@@ -136,7 +138,8 @@ def test_decode_ragged_long_contexts_mix_one_pass_and_grouped_sums():
     seq = torch.as_tensor(lens, device=DEV)
     ws = chai.new_workspace(chai.chai_decode_workspace_bytes(B, H, k, T, 128, chai.CHAI_BF16), DEV)
     outs = [chai.chai_decode_attention_ragged(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], seq,
-                                              case["scale"], T_max=T, workspace=ws) for _ in range(2)]
+                                              case["scale"], T_max=T, out=guard.empty_like(case["q"]), workspace=ws)
+            for _ in range(2)]
     torch.cuda.synchronize()
     assert chai.chai_device_status(ws) == chai.CHAI_OK
     assert torch.equal(outs[0], outs[1])
@@ -309,10 +312,11 @@ def prefill_inputs(seed, B, H, T, k, dtype="bf16", kind="uneven", peaked=1.0, D=
                 scale=1.0 / np.sqrt(D), dtype=dtype)
 
 
-def run_prefill(case, causal=True, fn=None):
+def run_prefill(case, causal=True, fn=None, guard=None):
     fn = fn or chai.chai_prefill_attention
     d = to_dev(case)
-    out = fn(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"], causal)
+    out = fn(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"], causal,
+             out=None if guard is None else guard.empty_like(d["q"]))
     torch.cuda.synchronize()
     return out.float().cpu().numpy()
 
@@ -320,10 +324,10 @@ def run_prefill(case, causal=True, fn=None):
 @pytest.mark.parametrize("fn_name", ["chai_prefill_attention", "chai_prefill_attention_simt"])
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("T", [1, 5, 31, 33, 64, 100, 128, 129, 200, 257, 300])
-def test_prefill_ragged_lengths(fn_name, dtype, T):
+def test_prefill_ragged_lengths(fn_name, dtype, T, guard):
     case = prefill_inputs(T, 2, 7, T, 3, dtype, peaked=4.0)
     for causal in (True, False):
-        got = run_prefill(case, causal, getattr(chai, fn_name))
+        got = run_prefill(case, causal, getattr(chai, fn_name), guard=guard)
         ref = orc.cha_attention(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"],
                                 case["scale"], causal)
         assert_parity(got, ref, dtype, f"{fn_name} {dtype} T {T} causal {causal}")

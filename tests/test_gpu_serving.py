@@ -29,12 +29,13 @@ def ragged_case(cfg, seed, B, H, k, T_cap, D=128):
 
 @pytest.mark.parametrize("cfg,D", [(1, 128), (2, 128), (2, 64)])
 @pytest.mark.parametrize("lens", [[700, 1, 129, 0, 333], [128, 256, 384, 512, 640], [5, 5, 5, 5, 5], [0, 0, 0, 0, 1]])
-def test_ragged_decode(cfg, D, lens):
+def test_ragged_decode(cfg, D, lens, guard):
     case = ragged_case(cfg, sum(lens), 5, 12, 3, 700, D)
     seq = torch.tensor(lens, dtype=torch.int32, device=DEV)
-    out = chai.chai_decode_attention_ragged(case["q"].to(DEV), case["k_rep"].to(DEV), case["v"].to(DEV),
+    q = case["q"].to(DEV)
+    out = chai.chai_decode_attention_ragged(q, case["k_rep"].to(DEV), case["v"].to(DEV),
                                             case["membership"].to(DEV), case["reps"].to(DEV), seq, case["scale"],
-                                            T_max=max(max(lens), 1))
+                                            T_max=max(max(lens), 1), out=guard.empty_like(q))
     torch.cuda.synchronize()
     got = out.float().cpu().numpy()
     ref = orc.decode_attention_ragged(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], lens,
@@ -46,7 +47,7 @@ def test_ragged_decode(cfg, D, lens):
             assert not got[b].any()
 
 
-def test_ragged_decode_never_reads_beyond_a_request():
+def test_ragged_decode_never_reads_beyond_a_request(guard):
     """Rows at or after seq_lens[b] hold NaN: the output must not notice."""
     lens = [300, 17, 129]
     case = ragged_case(2, 4, 3, 8, 4, 300)
@@ -55,8 +56,9 @@ def test_ragged_decode_never_reads_beyond_a_request():
         k_rep[b, :, n:] = float("nan")
         v[b, :, n:] = float("nan")
     seq = torch.tensor(lens, dtype=torch.int32, device=DEV)
-    out = chai.chai_decode_attention_ragged(case["q"].to(DEV), k_rep.to(DEV), v.to(DEV), case["membership"].to(DEV),
-                                            case["reps"].to(DEV), seq, case["scale"], T_max=300)
+    q = case["q"].to(DEV)
+    out = chai.chai_decode_attention_ragged(q, k_rep.to(DEV), v.to(DEV), case["membership"].to(DEV),
+                                            case["reps"].to(DEV), seq, case["scale"], T_max=300, out=guard.empty_like(q))
     got = out.float().cpu().numpy()
     ref = orc.decode_attention_ragged(case["q"], case["k_rep"], case["v"], case["membership"], case["reps"], lens,
                                       case["scale"])
@@ -65,7 +67,7 @@ def test_ragged_decode_never_reads_beyond_a_request():
 
 
 @pytest.mark.parametrize("cfg", [1, 2])
-def test_inplace_compaction_then_decode_and_append(cfg):
+def test_inplace_compaction_then_decode_and_append(cfg, guard):
     """The whole serving hand-over on one buffer: compaction in place, decode from the strided cache, append a
     token (representatives' keys only, every head's values), decode again over one more position."""
     B, H, k, T_cap = 3, 12, 4, 260
@@ -73,7 +75,8 @@ def test_inplace_compaction_then_decode_and_append(cfg):
     case = ragged_case(cfg, 21, B, H, k, T_cap)
     reps = case["reps"]
     assert all(int(reps[b, c]) >= c for b in range(B) for c in range(k))
-    cache = case["k_full"].to(DEV).clone()
+    cache = guard.empty_like(case["k_full"].to(DEV))   # the caches are written in place: they get guard bands too
+    cache.copy_(case["k_full"])
     before = bits(cache)
     ws = chai.new_workspace(256, DEV)
     chai.chai_compact_k_cache_inplace(cache, reps.to(DEV), T=T_cap, workspace=ws)
@@ -83,9 +86,10 @@ def test_inplace_compaction_then_decode_and_append(cfg):
     assert np.array_equal(after[:, :k], want)                       # bit copy of the representatives
     seq = torch.tensor(lens, dtype=torch.int32, device=DEV)
     d = {n: case[n].to(DEV) for n in ("q", "v", "membership", "reps")}
-    v = d["v"].clone()
+    v = guard.empty_like(d["v"])
+    v.copy_(d["v"])
     out = chai.chai_decode_attention_ragged(d["q"], cache, v, d["membership"], d["reps"], seq, case["scale"],
-                                            T_max=T_cap)
+                                            T_max=T_cap, out=guard.empty_like(d["q"]))
     ref = orc.decode_attention_ragged(case["q"], case["k_rep"], case["v"], case["membership"], reps, lens, case["scale"])
     assert_parity(out.float().cpu().numpy(), ref, case["dtype"], "decode from a cache compacted in place")
     # append one token per request
@@ -99,7 +103,7 @@ def test_inplace_compaction_then_decode_and_append(cfg):
     assert np.array_equal(bits(cache)[:, :k], k_ref) and np.array_equal(bits(v), v_ref)
     assert np.array_equal(bits(cache)[:, k:], after[:, k:])          # dead planes are not touched by the append
     out2 = chai.chai_decode_attention_ragged(d["q"], cache, v, d["membership"], d["reps"], seq, case["scale"],
-                                             T_max=T_cap)
+                                             T_max=T_cap, out=guard.empty_like(d["q"]))
     kf, vf = case["k_rep"].clone(), case["v"].clone()
     for b, n in enumerate(lens):
         vf[b, :, n] = v_new[b]
@@ -142,7 +146,7 @@ def test_inplace_compaction_refuses_unordered_reps():
 @pytest.mark.parametrize("fn_name", ["chai_prefill_attention_from", "chai_prefill_attention_simt_from"])
 @pytest.mark.parametrize("T,q_start,D", [(300, 5, 128), (300, 128, 128), (300, 131, 128), (64, 5, 128), (129, 128, 128),
                                          (640, 257, 128), (300, 5, 64), (300, 131, 64)])
-def test_prefill_from_q_start(fn_name, T, q_start, D):
+def test_prefill_from_q_start(fn_name, T, q_start, D, guard):
     """Rows from q_start on equal the full clustered prefill; earlier rows of the output are not written."""
     B, H, k = 2, 6, 2
     r = synth.batch_partitions(B, H, k, "uneven", T, 79, q_start)
@@ -152,7 +156,8 @@ def test_prefill_from_q_start(fn_name, T, q_start, D):
     v = (torch.randn(B, H, T, D, generator=g) * 0.5).to(torch.bfloat16)
     mem, reps = torch.as_tensor(r[0]), torch.as_tensor(r[1])
     scale = 1.0 / np.sqrt(D)
-    out = torch.full((B, H, T, D), 7.0, dtype=torch.bfloat16, device=DEV)
+    out = guard.empty((B, H, T, D), torch.bfloat16)
+    out.fill_(7.0)
     getattr(chai, fn_name)(q.to(DEV), kr.to(DEV), v.to(DEV), mem.to(DEV), reps.to(DEV), scale, q_start, True, out=out)
     got = out.float().cpu().numpy()
     ref = orc.cha_attention(q, kr, v, mem, reps, scale, True)

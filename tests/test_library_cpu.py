@@ -129,7 +129,7 @@ def test_binding_signatures_match_the_header(lib):
             where = f"{name} parameter {i} ({decl})"
             if "*" in decl:
                 assert ct in (ctypes.c_void_p, ctypes.c_char_p) or issubclass(ct, ctypes._Pointer), where
-            elif decl.startswith(("size_t", "uint64_t")):
+            elif decl.startswith(("size_t", "uint64_t", "long long")):
                 assert ctypes.sizeof(ct) == 8 and ct not in (ctypes.c_void_p, ctypes.c_double), where
             elif decl.startswith("float"):
                 assert ct is ctypes.c_float, where
