@@ -472,8 +472,9 @@ def test_unused_cluster_slots():
 
 
 def test_prefill_full_size_sampled_rows():
-    """Workload 5 at full size: the first 192 rows and the last 64 rows of every request and head
-    (causal attention of the first rows depends only on the first keys; the last rows see everything)."""
+    """Workload 5 at full size: the first 192 rows, 64 rows in the middle of the prompt that straddle a query-tile
+    boundary, and the last 64 rows of every request and head (causal attention of a row depends only on the keys
+    up to it, so the oracle runs on the prefix that ends with the sampled rows; the last rows see everything)."""
     case = synth.prefill_case(seed=0, device=DEV)
     k_rep = chai.chai_compact_k_cache(case["k_full"], case["reps"])
     out = chai.chai_prefill_attention(case["q_full"], k_rep, case["v"], case["membership"], case["reps"], case["scale"])
@@ -487,6 +488,33 @@ def test_prefill_full_size_sampled_rows():
     assert_parity(out[:, :, :192].float().cpu().numpy(), head, "bf16", "first rows")
     tail = orc.cha_attention(q[:, :, T - 64:], kr, v, mem, reps, case["scale"], True)
     assert_parity(out[:, :, T - 64:].float().cpu().numpy(), tail, "bf16", "last rows")
+    lo, hi = 992, 1056                                            # rows 992..1023 end one query tile, 1024..1055 begin the next
+    mid = orc.cha_attention(q[:, :, :hi], kr[:, :, :hi], v[:, :, :hi], mem, reps, case["scale"], True)
+    assert_parity(out[:, :, lo:hi].float().cpu().numpy(), mid[:, :, lo:hi], "bf16", "middle rows")
+
+
+def test_prefill_negative_controls_at_workload_5_statistics():
+    """The gates must tell a wrong clustering from the right one on the bench workload's own value distribution
+    (near-uniform softmax, small outputs), not only on peaked inputs: the same call with the representatives' key
+    planes rolled by one cluster, and with every non-representative head moved to the next cluster, must FAIL
+    the gates that the correct call passes (first 192 rows of every request and head)."""
+    case = synth.prefill_case(seed=0, device=DEV)
+    k_rep = chai.chai_compact_k_cache(case["k_full"], case["reps"])
+    n = 192
+    q, v = case["q_full"][:, :, :n].contiguous(), case["v"][:, :, :n].contiguous()
+    kr = k_rep[:, :, :n].contiguous()
+    mem, reps = case["membership"], case["reps"]
+    ref = orc.cha_attention(q.cpu(), kr.cpu(), v.cpu(), mem.cpu(), reps.cpu(), case["scale"], True)
+    run = lambda kk, mm: chai.chai_prefill_attention(q, kk, v, mm, reps, case["scale"]).float().cpu().numpy()
+    assert gate_ok(run(kr, mem), ref, "bf16")
+    assert not gate_ok(run(torch.roll(kr, 1, dims=1).contiguous(), mem), ref, "bf16")
+    is_rep = torch.zeros_like(mem, dtype=torch.bool)
+    is_rep.scatter_(1, reps.long(), True)
+    moved = torch.where(is_rep, mem, (mem + 1) % case["k"]).to(mem.dtype)   # still consistent: every representative stays put
+    ws = chai.new_workspace(chai.chai_prefill_workspace_bytes(case["B"], case["H"], case["k"], n, case["D"], chai.CHAI_BF16), DEV)
+    out = chai.chai_prefill_attention(q, kr, v, moved, reps, case["scale"], workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_OK
+    assert not gate_ok(out.float().cpu().numpy(), ref, "bf16")
 
 
 def test_prefill_long_prompt_sampled_rows():
@@ -523,6 +551,9 @@ def test_prefill_head_dim_64_full_size_sampled_rows():
     assert_parity(out[:, :, :192].float().cpu().numpy(), head, "bf16", "D 64 first rows")
     tail = orc.cha_attention(q[:, :, T - 64:], kr, v, mem, reps, case["scale"], True)
     assert_parity(out[:, :, T - 64:].float().cpu().numpy(), tail, "bf16", "D 64 last rows")
+    lo, hi = 992, 1056                                            # across the boundary between two query tiles
+    mid = orc.cha_attention(q[:, :, :hi], kr[:, :, :hi], v[:, :, :hi], mem, reps, case["scale"], True)
+    assert_parity(out[:, :, lo:hi].float().cpu().numpy(), mid[:, :, lo:hi], "bf16", "D 64 middle rows")
 
 
 @pytest.mark.parametrize("B,H,k,T,D,kind", [

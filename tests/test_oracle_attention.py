@@ -389,6 +389,31 @@ def test_e4m3_table_and_quantiser():
     assert np.allclose(vals[q[0, :2]] * s[0], y[0, :2], rtol=2 ** -4) and not q[0, 2].any() and not q[1].any()
 
 
+@pytest.mark.parametrize("amax", [448.0, 56.0, 1656.0])   # plane scales 1, 2^-3 and 3.696... (not a power of two)
+def test_quantiser_equals_the_library_cast_on_every_bf16_value(amax):
+    """Every finite bf16 bit pattern of magnitude <= amax in one plane (so the plane's scale is amax / 448):
+    the quantiser's byte must be the one PyTorch's float32 -> float8_e4m3fn cast gives for float32(x) / scale,
+    an independent implementation of round-to-nearest-even onto the same grid (no input exceeds 448 after
+    scaling, so saturation is not involved; NaN and infinity are not cache contents and are left out).  The
+    256-entry value table is checked against the library's decoding of the same bytes."""
+    import torch
+    table = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    vals = orc.e4m3_values()
+    assert np.array_equal(np.isnan(table), np.isnan(vals)) and np.array_equal(table[~np.isnan(table)], vals[~np.isnan(vals)])
+    bits = torch.arange(65536, dtype=torch.int32).to(torch.int16)
+    x = bits.view(torch.bfloat16).float()
+    x = x[torch.isfinite(x) & (x.abs() <= amax)]
+    assert x.numel() > 30000 and float(x.abs().max()) == amax        # both signs, zeros and subnormals included
+    D = 128
+    pad = (-x.numel()) % D
+    plane = torch.cat([x, torch.zeros(pad)]).reshape(1, -1, D).numpy()
+    q, s = orc.quantize_cache_fp8(plane, plane.shape[1])
+    scale = np.float32(amax) / np.float32(448.0)
+    assert s.tolist() == [scale]
+    want = (torch.from_numpy(plane) / torch.tensor(scale)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    assert np.array_equal(q, want), f"{int((q != want).sum())} of {q.size} bytes differ"
+
+
 def test_fp8_decode_is_the_decode_definition_on_what_the_bytes_stand_for():
     """Values chosen from the e4m3 grid (built here from the format's definition, not from the oracle's table):
     with scale 1 the byte caches stand for exactly the original numbers, so the fp8 decode must equal plain

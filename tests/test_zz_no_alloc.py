@@ -13,6 +13,8 @@ from paper_2403_08058_b200 import chai, synth
 
 @pytest.mark.gpu
 def test_static_scratch_decode_matches_workspace_decode_twice():
+    from oracle import chai_oracle as orc
+    from parity import assert_parity
     dev = "cuda"
     # two calls in a row with different shapes: the second one sees stale scratch contents
     for cfg, kw in ((2, dict(seed=11, B=3, H=16, T=700, T_cap=704, k=4)), (3, dict(seed=12, B=2, H=20, T=333, k=7)),
@@ -22,14 +24,26 @@ def test_static_scratch_decode_matches_workspace_decode_twice():
         want = chai.chai_decode_attention(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"],
                                           T=case["T"])
         out = torch.full_like(d["q"], 7.0)
+        again = torch.full_like(d["q"], 7.0)
         chai.chai_decode_attention_static(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"],
                                           T=case["T"], out=out)
-        again = torch.full_like(d["q"], 7.0)
+        # the second call is the one whose footprint is measured: by then the library's module is loaded on this
+        # device, so whatever the call itself allocates would show in the driver's count of free bytes and in the
+        # framework's count of allocations
+        torch.cuda.synchronize()
+        free_before, n_alloc_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_stats()["allocation.all.allocated"]
         chai.chai_decode_attention_static(d["q"], d["k_rep"], d["v"], d["membership"], d["reps"], case["scale"],
                                           T=case["T"], out=again)
         torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+        assert torch.cuda.memory_stats()["allocation.all.allocated"] == n_alloc_before
         # same kernels, same order of operations: the tolerance of the parity tests is met with zero error
         assert torch.equal(out, want) and torch.equal(again, want), (cfg, kw)
+        # ... and against the definition itself, not only against the sibling entry point
+        T = case["T"]
+        ref = orc.cha_attention(case["q"], case["k_rep"][:, :, :T], case["v"][:, :, :T], case["membership"], case["reps"],
+                                case["scale"], causal=False)
+        assert_parity(again.float().cpu().numpy(), ref, case["dtype"], f"static entry, cfg {cfg}")
 
 
 def test_static_scratch_rejects_what_does_not_fit():
