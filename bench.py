@@ -37,6 +37,62 @@ METRIC = "clustered decode attention: algorithmic HBM GB/s over one decode step 
 UNIT = "GB/s"
 
 
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "decode_persistent_kernel_dram_traffic.json")
+
+
+def load_traffic_ratio():
+    """DRAM bytes per launch over algorithmic bytes per launch of the decode kernel, as measured by the ncu capture
+    recorded in profiles/ (written by `bench.py --record-traffic`, which parses that capture); None when absent."""
+    try:
+        rec = json.load(open(TRAFFIC_RECORD))
+        return float(rec["dram_bytes_per_launch"]) / float(rec["algorithmic_bytes_per_launch"]), rec
+    except (OSError, ValueError, KeyError, ZeroDivisionError):
+        return None, None
+
+
+def record_traffic(csv_path: str, layers: int, workload: int):
+    """Turns an ncu CSV (--page raw, or --csv log of --metrics dram__bytes_read.sum,dram__bytes_write.sum) of
+    `bench.py --workload W --layers N --skip-extras` into the tracked record: mean DRAM bytes per captured launch of
+    the decode kernel beside the mean algorithmic bytes of the same layers."""
+    import csv
+    rows = list(csv.reader(open(csv_path, errors="replace")))
+    hdr_i = next(i for i, r in enumerate(rows) if "Kernel Name" in r)
+    hdr = rows[hdr_i]
+    per_launch = {}
+    if "Metric Name" in hdr:          # one row per (launch, metric)
+        ki, mi, vi, ui, idi = (hdr.index(n) for n in ("Kernel Name", "Metric Name", "Metric Value", "Metric Unit", "ID"))
+        for r in rows[hdr_i + 1:]:
+            if len(r) <= vi or "decode_persistent_kernel" not in r[ki] or not r[mi].startswith("dram__bytes_"):
+                continue
+            unit = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}[r[ui]]
+            per_launch[r[idi]] = per_launch.get(r[idi], 0.0) + float(r[vi].replace(",", "")) * unit
+    else:                             # raw page: one row per launch, one column per metric, units in the next row
+        units = rows[hdr_i + 1]
+        ki = hdr.index("Kernel Name")
+        cols = [i for i, n in enumerate(hdr) if n in ("dram__bytes_read.sum", "dram__bytes_write.sum")]
+        for j, r in enumerate(rows[hdr_i + 2:]):
+            if len(r) <= max(cols) or "decode_persistent_kernel" not in r[ki]:
+                continue
+            per_launch[j] = sum(float(r[i].replace(",", "")) * {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}[units[i]]
+                                for i in cols)
+    if not per_launch:
+        raise SystemExit("no decode_persistent_kernel launches with dram__bytes_* metrics in " + csv_path)
+    w = synth.WORKLOADS[workload]
+    es = 2 if w.dtype == "bf16" else 4
+    ks = [min(synth.layer_k(workload, layer, 0), w.H) for layer in range(min(layers, w.layers))]
+    alg = float(np.mean([decode_bytes(w.B, w.H, k, w.T, w.D, es) for k in ks]))
+    rec = {"kernel": "decode_persistent_kernel", "workload": f"{w.name}, first {len(ks)} layers (k = {ks})",
+           "launches_captured": len(per_launch), "dram_bytes_per_launch": float(np.mean(list(per_launch.values()))),
+           "algorithmic_bytes_per_launch": alg,
+           "how": f"`python bench.py --workload {workload} --layers {layers} --skip-extras --no-graph --steps 3 --warmup 3` "
+                  "(exit 0), then the same command under `ncu --metrics dram__bytes_read.sum,dram__bytes_write.sum "
+                  "--clock-control none -k regex:decode_persistent -s 8 -c 12 --csv --log-file traffic.csv`, then "
+                  f"`python bench.py --record-traffic traffic.csv --workload {workload} --layers {layers}`"}
+    rec["ratio"] = rec["dram_bytes_per_launch"] / alg
+    json.dump(rec, open(TRAFFIC_RECORD, "w"), indent=1)
+    print(json.dumps(rec))
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -228,6 +284,31 @@ def cpu_baseline_decode(cfg_id: int, seed: int, budget_s: float = 12.0):
                        f"{spent:.1f} s of oracle time, inputs already widened to fp64)", seconds=spent)
 
 
+def cpu_baseline_prefill(seed: int = 0, budget_s: float = 12.0):
+    """Times the CPU oracle, as it stands, on workload 5 itself: whole requests (all rows, all heads), one after
+    the other and round again until about `budget_s` seconds of oracle time are spent.  Flops counted as for the
+    GPU: 2*D per causal (row, key) pair, once per cluster for the scores and once per head for the values."""
+    from oracle import chai_oracle as orc
+    case = synth.prefill_case(seed=seed, device="cpu")
+    B, H, T, D, k = case["B"], case["H"], case["T"], case["D"], case["k"]
+    mem, reps = case["membership"], case["reps"]
+    idx = reps.long()[:, :, None, None].expand(B, k, T, D)
+    k_rep = torch.gather(case["k_full"], 1, idx)
+    wide = [[orc._f64(x[b:b + 1]) for x in (case["q_full"], k_rep, case["v"])] for b in range(B)]
+    spent, flops, n_req = 0.0, 0.0, 0
+    wall0 = time.perf_counter()
+    while spent < budget_s and time.perf_counter() - wall0 < 90.0:
+        b = n_req % B
+        t0 = time.perf_counter()
+        orc.cha_attention(wide[b][0], wide[b][1], wide[b][2], mem[b:b + 1], reps[b:b + 1], case["scale"], True)
+        spent += time.perf_counter() - t0
+        flops += prefill_flops(1, H, k, T, D)
+        n_req += 1
+    return dict(value=flops / spent / 1e12, unit="TFLOP/s", cores=orc.num_threads(), kind="oracle",
+                sample=f"{n_req} whole requests of workload 5 (its {B} requests in rotation; {spent:.1f} s of oracle time, "
+                       "fp64, inputs already widened)", seconds=spent)
+
+
 def run_reference(args, rank):
     """The reference arm of this tier is the CPU oracle timed on the host cores."""
     if rank != 0:
@@ -348,19 +429,16 @@ def bench_prefill(device, peaks, iters=20, warmup=3):
 
 
 def bench_compaction(device, peaks, iters=20, warmup=3):
-    """Out-of-place compaction of one workload-4 layer (k = 24), layer after layer over six layers' caches
-    (1.2 GB, far more than L2), as a model's 64 layers are compacted one after the other; and the same call
-    after a 256 MB write that leaves L2 full of dirty lines, which the call then has to evict."""
+    """Out-of-place compaction of one workload-4 layer for k = 12, 24 and 36 (the range that workload draws from),
+    layer after layer over six layers' caches (1.2 GB, far more than L2), as a model's 64 layers are compacted one
+    after the other; and, for k = 24, the same call after a 256 MB write that leaves L2 full of dirty lines, which
+    the call then has to evict."""
     w = synth.WORKLOADS[4]
-    k, sets = 24, 6
+    sets = 6
     g = torch.Generator(device=device).manual_seed(4)
     k_full = [torch.randn((w.B, w.H, w.T, w.D), device=device, generator=g).to(torch.bfloat16) for _ in range(sets)]
-    _, reps = synth.batch_partitions(w.B, w.H, k, "uneven", 0, 4, 0)
-    reps = torch.as_tensor(reps, device=device)
-    k_rep = [torch.empty((w.B, k, w.T, w.D), device=device, dtype=torch.bfloat16) for _ in range(sets)]
-    nbytes = 2 * k * w.B * w.T * w.D * 2
 
-    def timed(flush):
+    def timed(k, reps, k_rep, flush):
         ts = []
         for i in range(warmup + iters):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -381,15 +459,27 @@ def bench_compaction(device, peaks, iters=20, warmup=3):
                 ts.append(e0.elapsed_time(e1) / n)
         return statistics.median(ts)
 
-    ms = timed(None)
-    ms_dirty = timed(torch.empty(256 << 20, device=device, dtype=torch.uint8))
-    gbs = nbytes / (ms * 1e-3) / 1e9
-    return {"workload": "config4 one layer, k=24", "us": ms * 1e3, "algorithmic_mb": nbytes / 1e6, "gbs": gbs,
-            "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"],
-                         "peak_source": peaks["source"], "traffic": None},
+    by_k = {}
+    for k in (12, 24, 36):
+        _, reps = synth.batch_partitions(w.B, w.H, k, "uneven", 0, 4, 0)
+        reps = torch.as_tensor(reps, device=device)
+        k_rep = [torch.empty((w.B, k, w.T, w.D), device=device, dtype=torch.bfloat16) for _ in range(sets)]
+        nbytes = 2 * k * w.B * w.T * w.D * 2
+        ms = timed(k, reps, k_rep, None)
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        by_k[f"k{k}"] = {"us": ms * 1e3, "algorithmic_mb": nbytes / 1e6, "gbs": gbs, "frac": gbs / peaks["hbm"]}
+        if k == 24:
+            ms_dirty = timed(k, reps, k_rep, torch.empty(256 << 20, device=device, dtype=torch.uint8))
+            dirty = {"us": ms_dirty * 1e3, "gbs": nbytes / (ms_dirty * 1e-3) / 1e9,
+                     "note": "L2 full of the flush's dirty lines, which the call evicts"}
+        del k_rep
+    mid = by_k["k24"]
+    return {"workload": "config4 one layer (B 4, H 72, T 2048, D 128), k = 12 / 24 / 36", "by_k": by_k,
+            "us": mid["us"], "algorithmic_mb": mid["algorithmic_mb"], "gbs": mid["gbs"],
+            "roofline": {"bound": "hbm", "achieved": mid["gbs"], "peak": peaks["hbm"], "unit": "GB/s", "frac": mid["frac"],
+                         "peak_source": peaks["source"], "traffic": None, "workload": "k = 24"},
             "l2": "six layers' caches in rotation (1.2 GB): every call reads and writes memory that is not in L2",
-            "after_a_256MB_write": {"us": ms_dirty * 1e3, "gbs": nbytes / (ms_dirty * 1e-3) / 1e9,
-                                    "note": "L2 full of the flush's dirty lines, which the call evicts"}}
+            "after_a_256MB_write": dirty}
 
 
 def bench_serving(device, peaks, iters=20, warmup=3):
@@ -592,6 +682,34 @@ def bench_fp8(device, peaks, iters=20, warmup=3):
     return res
 
 
+def bench_decode_workload(cfg_id, device, peaks, steps=10, warmup=3):
+    """The decode step of another workload, timed like the headline: the step's layer calls captured once in a CUDA
+    graph and replayed `steps` times back to back (every layer has its own caches: tens of GB per step)."""
+    wl = DecodeWorkload(cfg_id, device)
+    for _ in range(warmup):
+        wl.step()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        wl.step()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(warmup):
+        graph.replay()
+    ms = time_region(graph.replay, steps, torch.cuda.synchronize) / steps
+    ms_eager = time_region(wl.step, steps, torch.cuda.synchronize) / steps
+    gbs = wl.bytes_per_step / 1e9 / (ms * 1e-3)
+    w = wl.w
+    res = {"workload": w.name, "layers": w.layers, "B": w.B, "H": w.H, "T": w.T, "steps": steps,
+           "algorithmic_gb_per_step": wl.bytes_per_step / 1e9, "us_per_step": ms * 1e3, "us_per_layer": ms * 1e3 / w.layers,
+           "achieved": gbs, "peak": peaks["hbm"], "unit": "GB/s", "frac": gbs / peaks["hbm"],
+           "eager_us_per_step": ms_eager * 1e3, "launch": "one CUDA graph of the step's layer calls, replayed"}
+    del wl, graph
+    torch.cuda.empty_cache()
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -602,9 +720,14 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers (not a bench result)")
     ap.add_argument("--skip-extras", action="store_true", help="only the decode step (no prefill/compaction/CPU legs)")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a replayed CUDA graph")
-    ap.add_argument("--only", default="", choices=["", "prefill", "compaction", "serving", "fp8", "config1"],
+    ap.add_argument("--only", default="", choices=["", "prefill", "compaction", "serving", "fp8", "config1", "workload3", "workload4"],
                     help="profiling aid: run just this leg and print its object (not the bench line)")
+    ap.add_argument("--record-traffic", default="", metavar="NCU_CSV",
+                    help="no GPU work: parse an ncu CSV of `--workload W --layers N --skip-extras` into the tracked DRAM-traffic record")
     args = ap.parse_args()
+    if args.record_traffic:
+        record_traffic(args.record_traffic, args.layers or synth.WORKLOADS[args.workload].layers, args.workload)
+        return
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
 
@@ -630,7 +753,8 @@ def main():
     peaks = load_peaks()
     if args.only:
         leg = {"prefill": bench_prefill, "compaction": bench_compaction, "serving": bench_serving, "fp8": bench_fp8,
-               "config1": lambda d, p: bench_config1(d)}[args.only]
+               "config1": lambda d, p: bench_config1(d), "workload3": lambda d, p: bench_decode_workload(3, d, p),
+               "workload4": lambda d, p: bench_decode_workload(4, d, p)}[args.only]
         print(json.dumps({"leg": args.only, "result": leg(device, peaks)}))
         ranks.close()
         return
@@ -694,6 +818,7 @@ def main():
     e2e_value = replicas.whole_job_throughput(ranks, wl.bytes_per_step / 1e9, ms_e2e / args.steps * 1e-3)["value"]
 
     if rank == 0:
+        traffic_ratio, traffic_rec = load_traffic_ratio()
         # average launch duration over the timed region itself (K steps x layers launches, gaps included)
         per_launch_ms = ms_step / w.layers
         achieved = float(np.mean(wl.bytes_per_layer)) / (per_launch_ms * 1e-3) / 1e9
@@ -720,9 +845,15 @@ def main():
             "roofline": {"bound": "hbm", "kernel": "decode_persistent_kernel (one launch per layer call)",
                          "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s", "frac": achieved / peaks["hbm"],
                          "peak_source": peaks["source"],
-                         # DRAM read+write bytes per launch: ncu measured 1.02 x the algorithmic bytes on full-size
-                         # layers (profiles/decode_persistent_kernel_workload2.md), scaled to the mean launch here
-                         "traffic": 1.02 * float(np.mean(wl.bytes_per_layer)), "traffic_unit": "bytes per launch",
+                         # DRAM read+write bytes per launch: the ratio to the algorithmic bytes that an ncu capture of
+                         # this kernel measured (the tracked record names the capture), applied to the mean launch
+                         # here; null when there is no record
+                         "traffic": (traffic_ratio * float(np.mean(wl.bytes_per_layer)) if traffic_ratio else None),
+                         "traffic_unit": "bytes per launch",
+                         "traffic_source": (None if traffic_rec is None else
+                                            {"ratio_to_algorithmic": traffic_ratio, "measured_on": traffic_rec["workload"],
+                                             "launches": traffic_rec["launches_captured"],
+                                             "note": "ncu dram__bytes_read.sum + dram__bytes_write.sum per launch, scaled by the units processed"}),
                          "us_per_layer_by_k": {str(k): statistics.median(v) for k, v in sorted(by_k.items())},
                          "us_per_layer_by_k_note": "eager launches with an event after every layer call",
                          "frac_of_nominal_8TBs": achieved / 8000.0},
@@ -751,7 +882,29 @@ def main():
             line["serving"] = bench_serving(device, peaks)
             line["fp8_decode"] = bench_fp8(device, peaks)
             line["config1"] = bench_config1(device)
+            others = {f"workload{c}": bench_decode_workload(c, device, peaks) for c in (3, 4) if c != args.workload}
+            line["decode_other_workloads"] = others
+            # Compact summaries of the other legs inside the roofline object, so that this one object carries the
+            # whole metric: decode at every model-shaped workload, prefill, compaction, the serving and fp8 steps.
+            rl = line["roofline"]
+            rl[f"workload{args.workload}"] = {"us_per_step": ms_step * 1e3, "achieved": achieved, "frac": achieved / peaks["hbm"]}
+            for name, o in others.items():
+                rl[name] = {k2: o[k2] for k2 in ("us_per_step", "us_per_layer", "achieved", "frac", "algorithmic_gb_per_step")}
+            pf = line["prefill"]
+            rl["prefill"] = {"workload": pf["workload"], "us": pf["ms_attention"] * 1e3, "achieved": pf["tflops"],
+                             "peak": peaks["tf_burst"], "unit": "TFLOP/s", "frac": pf["roofline"]["frac"], "peak_kind": "burst",
+                             "algorithmic_gflop": pf["algorithmic_gflop"], "bound": "tensor",
+                             "sustained_frac": pf["sustained"]["frac"],
+                             "longer_prompts_frac": {k2: v2["frac_of_burst_peak"] for k2, v2 in pf["longer_prompts"].items()}}
+            rl["compaction"] = {k2: {"us": v2["us"], "achieved": v2["gbs"], "frac": v2["frac"]}
+                                for k2, v2 in line["compaction"]["by_k"].items()}
+            sv = line["serving"]
+            rl["ragged_decode"] = {"us": sv["ragged_decode"]["us"], "achieved": sv["ragged_decode"]["gbs"],
+                                   "frac": sv["ragged_decode"]["roofline"]["frac"]}
+            rl["fp8_decode"] = {k2: {"us_per_layer": line["fp8_decode"][k2]["us_per_layer"], "achieved": line["fp8_decode"][k2]["gbs"],
+                                     "frac": line["fp8_decode"][k2]["roofline"]["frac"]} for k2 in ("k8", "k32")}
             line["cpu_baseline"] = cpu_baseline_decode(args.workload, 0)
+            line["cpu_baseline"]["prefill"] = cpu_baseline_prefill()
         print(json.dumps(line))
     ranks.close()
 
