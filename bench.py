@@ -528,6 +528,37 @@ def bench_serving(device, peaks, iters=20, warmup=3):
     ms_f = timed(lambda: chai.chai_decode_attention_ragged(c["q"], cache, c["v"], c["membership"], c["reps"], full, c["scale"],
                                                            T_max=T_cap, out=out, workspace=ws))
     bytes_f = (k + H) * B * T_cap * D * es + (k + H) * B * D * es
+    # the same two calls timed like the headline: back to back over four cache sets (2 GB: every call streams its
+    # own caches from DRAM), launch latency hidden behind the previous call
+    sets = [(cache, c["v"])] + [(torch.randn_like(cache), torch.randn_like(c["v"])) for _ in range(3)]
+
+    def back_to_back(lens_t):
+        def run():
+            for kc_, vc_ in sets:
+                chai.chai_decode_attention_ragged(c["q"], kc_, vc_, c["membership"], c["reps"], lens_t, c["scale"],
+                                                  T_max=T_cap, out=out, workspace=ws)
+        for _ in range(warmup):
+            run()
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()          # as in the headline: the calls captured once and replayed
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(5):
+                run()
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(iters // 5):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / ((iters // 5) * 5 * len(sets))
+
+    ms_d_b2b, ms_f_b2b = back_to_back(seq), back_to_back(full)
+    del sets
     # append (no advance, so every run writes the same rows)
     k_new = torch.randn((B, H, D), device=device).to(torch.bfloat16)
     v_new = torch.randn((B, H, D), device=device).to(torch.bfloat16)
@@ -554,7 +585,13 @@ def bench_serving(device, peaks, iters=20, warmup=3):
             "full_length_same_timing": {"us": ms_f * 1e3, "algorithmic_mb": bytes_f / 1e6, "gbs": bytes_f / (ms_f * 1e-3) / 1e9},
             "ragged_decode": {"us": ms_d * 1e3, "algorithmic_mb": bytes_d / 1e6, "gbs": gbs_d,
                               "roofline": {"bound": "hbm", "achieved": gbs_d, "peak": peaks["hbm"], "unit": "GB/s",
-                                           "frac": gbs_d / peaks["hbm"], "peak_source": peaks["source"], "traffic": None}},
+                                           "frac": gbs_d / peaks["hbm"], "peak_source": peaks["source"], "traffic": None},
+                              "back_to_back": {"us": ms_d_b2b * 1e3, "gbs": bytes_d / (ms_d_b2b * 1e-3) / 1e9,
+                                               "frac": bytes_d / (ms_d_b2b * 1e-3) / 1e9 / peaks["hbm"],
+                                               "full_length_us": ms_f_b2b * 1e3,
+                                               "full_length_gbs": bytes_f / (ms_f_b2b * 1e-3) / 1e9,
+                                               "us_over_full_length_us_times_byte_ratio": ms_d_b2b / (ms_f_b2b * bytes_d / bytes_f),
+                                               "note": "four cache sets in rotation, the calls captured in a CUDA graph and replayed"}},
             "compact_inplace": {"us": ms_c * 1e3, "planes_moved": moved, "algorithmic_mb": bytes_c / 1e6, "gbs": gbs_c,
                                 "roofline": {"bound": "hbm", "achieved": gbs_c, "peak": peaks["hbm"], "unit": "GB/s",
                                              "frac": gbs_c / peaks["hbm"], "peak_source": peaks["source"], "traffic": None}},
@@ -899,8 +936,10 @@ def main():
             rl["compaction"] = {k2: {"us": v2["us"], "achieved": v2["gbs"], "frac": v2["frac"]}
                                 for k2, v2 in line["compaction"]["by_k"].items()}
             sv = line["serving"]
-            rl["ragged_decode"] = {"us": sv["ragged_decode"]["us"], "achieved": sv["ragged_decode"]["gbs"],
-                                   "frac": sv["ragged_decode"]["roofline"]["frac"]}
+            rl["ragged_decode"] = {"us": sv["ragged_decode"]["back_to_back"]["us"], "achieved": sv["ragged_decode"]["back_to_back"]["gbs"],
+                                   "frac": sv["ragged_decode"]["back_to_back"]["frac"], "timing": "back to back over four cache sets, graph replay",
+                                   "single_cold_call": {"us": sv["ragged_decode"]["us"], "frac": sv["ragged_decode"]["roofline"]["frac"]},
+                                   "us_over_full_length_us_times_byte_ratio": sv["ragged_decode"]["back_to_back"]["us_over_full_length_us_times_byte_ratio"]}
             rl["fp8_decode"] = {k2: {"us_per_layer": line["fp8_decode"][k2]["us_per_layer"], "achieved": line["fp8_decode"][k2]["gbs"],
                                      "frac": line["fp8_decode"][k2]["roofline"]["frac"]} for k2 in ("k8", "k32")}
             line["cpu_baseline"] = cpu_baseline_decode(args.workload, 0)

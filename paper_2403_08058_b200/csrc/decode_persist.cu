@@ -53,6 +53,7 @@ struct Cfg<Fp8E4M3> {
 constexpr int MAX_IV = 4;                  // tiles per value item
 constexpr int ITEM_SLOTS = 8;              // value items whose tile partials may be open in one CTA
 constexpr int TABLE_CAP = 2048;            // heads whose cluster id is cached in shared memory
+constexpr int RAG_CAP = 1024;              // requests whose tile and item counts are kept in shared memory (ragged batches)
 // groups a head's n items are first added in (1 = all at once)
 __host__ __device__ inline int combine_groups(int n) { return n > 4 * kCombineGroup ? (n + kCombineGroup - 1) / kCombineGroup : 1; }
 constexpr int LATE_ITEMS = 2;              // the last LATE_ITEMS items per CTA are claimed only when the producer is free
@@ -89,6 +90,8 @@ struct Smem {
     int item_free[ITEM_SLOTS];  // 1 when the slot may be given to a new item
     int table[TABLE_CAP];
     unsigned ready[TABLE_CAP / 32];  // bit p: every key tile of plane p is known to carry this launch's token
+    int tpre[RAG_CAP + 1];      // ragged batches: key tiles (per plane) of the requests before b, summed ...
+    int ipre[RAG_CAP + 1];      // ... and value items (per head): work is dealt over what really exists
     WaitCtl wait;
     int next_pos;               // next ring position a consumer warp may take
     unsigned epoch;             // launch count of this workspace, read once at start
@@ -376,7 +379,7 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
     const int tp = (T_len + G::TR - 1) / G::TR;          // tiles per cache plane
     const long long n_ktiles = (long long)B * k * tp;    // key tiles of the layer
     const int nkt = n_ktiles > cta ? (int)((n_ktiles - cta + ncta - 1) / ncta) : 0;  // this CTA's share
-    const int n_items = B * H * P.nVi;                   // value items of the layer
+    const int n_items_full = B * H * P.nVi;              // value items of the layer when every request has all T rows
     int* work_counter = &P.hdr->pad[0];
     int* launch_epoch = &P.hdr->pad[8];
 
@@ -407,6 +410,44 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
         for (int i = tid; i < B * H; i += THREADS) {
             int c, r;
             sm.table[i] = resolve_head(P.membership, P.reps, i / H, i % H, H, k, &c, &r) ? c : -1;
+        }
+    }
+    // A ragged batch is dealt by what it really holds: with the running sums of every request's key tiles and value
+    // items in shared memory, the producer walks (or claims) positions in the list of existing tiles and items, so
+    // that neither a ring position nor a claim is spent on a tile beyond a request's end and every CTA gets the
+    // same number of real key tiles.  (More than RAG_CAP requests: the positions are those of the full-length
+    // batch and the missing ones are skipped.)
+    const bool dealt_by_length = RAGGED && B <= RAG_CAP;
+    if (dealt_by_length) {
+        const int tr = G::TR;
+        for (int b = tid; b < B; b += THREADS) {
+            const int len = P.seq_lens ? min(max(__ldg(P.seq_lens + b), 0), T_len) : T_len;
+            const int t = max(1, (len + tr - 1) / tr);
+            sm.tpre[b + 1] = t;
+            sm.ipre[b + 1] = (t + P.IV - 1) / P.IV;
+        }
+        __syncthreads();
+        if (warp == 0) {  // inclusive scans, 32 requests at a time
+            int tc = 0, ic = 0;
+            for (int b0 = 0; b0 < B; b0 += 32) {
+                const int b = b0 + lane;
+                int tv = b < B ? sm.tpre[b + 1] : 0, iv = b < B ? sm.ipre[b + 1] : 0;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int tu = __shfl_up_sync(0xffffffffu, tv, o), iu = __shfl_up_sync(0xffffffffu, iv, o);
+                    if (lane >= o) {
+                        tv += tu;
+                        iv += iu;
+                    }
+                }
+                if (b < B) {
+                    sm.tpre[b + 1] = tc + tv;
+                    sm.ipre[b + 1] = ic + iv;
+                }
+                tc += __shfl_sync(0xffffffffu, tv, 31);
+                ic += __shfl_sync(0xffffffffu, iv, 31);
+            }
+            if (lane == 0) sm.tpre[0] = sm.ipre[0] = 0;
         }
     }
     __syncthreads();
@@ -472,7 +513,21 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 return true;
             };
             // ---- key tiles: global tile ids cta, cta + ncta, ... ----
-            {
+            if (dealt_by_length) {
+                // positions cta, cta + ncta, ... in the list of the key tiles that exist, ordered by (request,
+                // cluster, tile); positions only grow, so the request is found by walking forward
+                const long long total = (long long)k * sm.tpre[B];
+                int b = 0;
+                for (long long r = cta; r < total && ok; r += ncta) {
+                    while ((long long)k * sm.tpre[b + 1] <= r) ++b;
+                    const int tb = sm.tpre[b + 1] - sm.tpre[b];
+                    const int rem = (int)(r - (long long)k * sm.tpre[b]);
+                    const int c = rem / tb, tile = rem - c * tb;
+                    const TileMeta m{(int)(((long long)b * k + c) * tp + tile), -1, 0, 0};  // (the id consumers decode)
+                    ok = issue(kc + (size_t)b * P.k_batch_bytes + ((size_t)c * P.T_cap + (size_t)tile * G::TR) * G::ROW_BYTES,
+                               (uint32_t)tile_rows(b, tile) * G::ROW_BYTES, m);
+                }
+            } else {
                 int plane = cta / tp, tile = cta % tp;
                 const int dplane = ncta / tp, dtile = ncta % tp;
                 constexpr bool plain = !RAGGED;
@@ -499,14 +554,30 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             // (the work counter is reset by the owner of the layer's first key tile before that tile's flag)
             if (ok) ok = flag_wait_one(P.flags, token, abort_flag);
             int n_open = 0;  // items this CTA has opened (item slots are handed out round-robin)
+            // what is claimed: positions in the list of items -- of the items that exist, ordered by (request,
+            // head, chunk), when the batch is dealt by length; of the full-length batch's items otherwise
+            const int n_items = dealt_by_length ? H * sm.ipre[B] : n_items_full;
+            int b_walk = 0;  // (claims only grow: the request of a position is found by walking forward)
             int next = ok ? atomicAdd(work_counter, 1) : n_items;
             while (ok && next < n_items) {
-                const int item = next;
+                const int pos = next;
                 // The next claim is fetched while this item streams -- except near the end of the item list,
                 // where a claimed but unstarted item on a slow SM is work a faster one could have taken.
-                const bool ahead = item < n_items - LATE_ITEMS * ncta;
+                const bool ahead = pos < n_items - LATE_ITEMS * ncta;
                 if (ahead) next = atomicAdd(work_counter, 1);
-                const int head = item / P.nVi, chunk = item % P.nVi;
+                int head, chunk;
+                if (dealt_by_length) {
+                    while (H * sm.ipre[b_walk + 1] <= pos) ++b_walk;
+                    const int ib = sm.ipre[b_walk + 1] - sm.ipre[b_walk];
+                    const int rem = pos - H * sm.ipre[b_walk];
+                    const int h = rem / ib;
+                    head = b_walk * H + h;
+                    chunk = rem - h * ib;
+                } else {
+                    head = pos / P.nVi;
+                    chunk = pos % P.nVi;
+                }
+                const int item = head * P.nVi + chunk;  // the id consumers decode
                 const int tile0 = chunk * P.IV;
                 const int b_item = RAGGED ? head / H : 0;
                 const int ntiles = min(P.IV, tiles_of(b_item) - tile0);
@@ -780,7 +851,20 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
             if (ok && have_p) {
                 {
-                    const unsigned char* data = sm.ring[slot];
+                    unsigned char* data = sm.ring[slot];
+                    if (rows < G::TR) {
+                        // Ragged last tile: the copy brought `rows` rows, the rest of the slot holds whatever it held
+                        // before.  Those rows' probabilities are 0, but 0 x (bytes that decode to NaN or infinity) is
+                        // not, so the warp clears them in shared memory and then runs the one loop every tile runs
+                        // (a separate loop with a test per row, visited once per plane, cost several full tiles each
+                        // time: 61 us instead of 52 for lengths of 1407 instead of 1408).  The slot's next fill is
+                        // by the copy engine: its writes are ordered after these by the proxy fence.
+                        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                        uint4* v16 = reinterpret_cast<uint4*>(data);
+                        for (int idx = rows * (G::ROW_BYTES / 16) + lane; idx < G::TR * (G::ROW_BYTES / 16); idx += 32) v16[idx] = zero;
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
                     if constexpr (std::is_same<T, Fp8E4M3>::value) {
                         // fp8 values: the per-element conversions to fp32 are what bounds this path, so the
                         // products are formed and summed as fp16 pairs (every e4m3 value is an fp16 value; a
@@ -807,19 +891,17 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                                 const int r32 = i * G::RPW + sub;
                                 const float pr = __shfl_sync(0xffffffffu, pv[u], r32);
                                 const int row = u * 32 + r32;
-                                if (row < rows) {  // never touch stale bytes of a ragged last tile (its probabilities are 0 anyway)
-                                    const uint4 raw = *reinterpret_cast<const uint4*>(data + row * G::ROW_BYTES + part * 16);
-                                    __half2 vh[8];
-                                    Vec16<T>::unpack_h2(raw, vh);
-                                    const __half2 ph = __float2half2_rn(pr);
+                                const uint4 raw = *reinterpret_cast<const uint4*>(data + row * G::ROW_BYTES + part * 16);
+                                __half2 vh[8];
+                                Vec16<T>::unpack_h2(raw, vh);
+                                const __half2 ph = __float2half2_rn(pr);
 #pragma unroll
-                                    for (int j = 0; j < 8; ++j) hacc[j] = __hfma2(ph, vh[j], hacc[j]);
-                                }
+                                for (int j = 0; j < 8; ++j) hacc[j] = __hfma2(ph, vh[j], hacc[j]);
                                 if ((u * G::IT + i) % FLUSH == FLUSH - 1) flush();
                             }
                         }
                         if ((G::PV * G::IT) % FLUSH != 0) flush();
-                    } else if (rows == G::TR) {
+                    } else {
 #pragma unroll
                         for (int u = 0; u < G::PV; ++u) {
 #pragma unroll
@@ -831,23 +913,6 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                                 Vec16<T>::unpack(raw, vf);
 #pragma unroll
                                 for (int e = 0; e < G::EPV; ++e) acc[e] = fmaf(pr, vf[e], acc[e]);
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int u = 0; u < G::PV; ++u) {
-#pragma unroll 4
-                            for (int i = 0; i < G::IT; ++i) {
-                                const int r32 = i * G::RPW + sub;
-                                const float pr = __shfl_sync(0xffffffffu, pv[u], r32);
-                                const int row = u * 32 + r32;
-                                if (row < rows) {  // never touch stale bytes of a ragged last tile
-                                    const uint4 raw = *reinterpret_cast<const uint4*>(data + row * G::ROW_BYTES + part * 16);
-                                    float vf[G::EPV];
-                                    Vec16<T>::unpack(raw, vf);
-#pragma unroll
-                                    for (int e = 0; e < G::EPV; ++e) acc[e] = fmaf(pr, vf[e], acc[e]);
-                                }
                             }
                         }
                     }
