@@ -719,6 +719,107 @@ def bench_fp8(device, peaks, iters=20, warmup=3):
     return res
 
 
+def graph_time_us(run, calls_per_run, reps=4, warmup=3):
+    """Mean microseconds per call of `run` (which enqueues `calls_per_run` calls), captured five times into one CUDA
+    graph that is replayed `reps` times back to back."""
+    for _ in range(warmup):
+        run()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for _ in range(5):
+            run()
+    torch.cuda.current_stream().wait_stream(side)
+    graph.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / (reps * 5 * calls_per_run)
+
+
+def bench_variants(device, peaks):
+    """The method's variants and second shapes: CHAI-QKV decode (values of non-representative heads dropped too: 2k
+    cache planes per request) at workload 2's layer shape beside the main decode call timed the same way; CHAI-QKV
+    prefill and head_dim-64 prefill at workload 5's shape."""
+    w = synth.WORKLOADS[2]
+    B, H, T, D, es = w.B, w.H, w.T, w.D, 2
+    res = {}
+    for k in (8, 16):
+        sets = []
+        for i in range(8):
+            c = synth.decode_layer(2, i, 5, device=device, B=B, H=H, T=T, k=k)
+            v_rep = torch.stack([c["v"][b].index_select(0, c["reps"][b].long()) for b in range(B)])
+            sets.append((c["q"], c["k_rep"], c["v"], v_rep, c["membership"], c["reps"], c["scale"]))
+        ws = chai.new_workspace(max(int(chai.load().chai_decode_qkv_workspace_bytes(B, H, k, T, D, chai.CHAI_BF16)),
+                                    chai.chai_decode_workspace_bytes(B, H, k, T, D, chai.CHAI_BF16)), device)
+        out = torch.empty_like(sets[0][0])
+
+        def run_qkv():
+            for (q, kr, v, vr, mem, reps, scale) in sets:
+                chai.chai_decode_attention_qkv(q, kr, vr, mem, reps, scale, out=out, workspace=ws)
+
+        def run_main():
+            for (q, kr, v, vr, mem, reps, scale) in sets:
+                chai.chai_decode_attention(q, kr, v, mem, reps, scale, out=out, workspace=ws)
+
+        us_q, us_m = graph_time_us(run_qkv, len(sets)), graph_time_us(run_main, len(sets))
+        by_q = 2 * k * B * T * D * es + k * B * D * es + H * B * D * es + 4 * B * (H + k)
+        by_m = decode_bytes(B, H, k, T, D, es)
+        # the main call on as many bytes as the QKV call moves (a shorter context of the same caches): what the same
+        # kernel reaches when a launch has this little to stream
+        T_eq = max(128, int(round(T * by_q / by_m / 128.0)) * 128)
+
+        def run_main_eq():
+            for (q, kr, v, vr, mem, reps, scale) in sets:
+                chai.chai_decode_attention(q, kr, v, mem, reps, scale, T=T_eq, out=out, workspace=ws)
+
+        us_e = graph_time_us(run_main_eq, len(sets))
+        by_e = decode_bytes(B, H, k, T_eq, D, es)
+        res[f"decode_qkv_k{k}"] = {"us": us_q, "algorithmic_mb": by_q / 1e6, "gbs": by_q / us_q / 1e3,
+                                   "frac": by_q / us_q / 1e3 / peaks["hbm"],
+                                   "main_call_same_timing": {"us": us_m, "algorithmic_mb": by_m / 1e6, "gbs": by_m / us_m / 1e3,
+                                                             "frac": by_m / us_m / 1e3 / peaks["hbm"]},
+                                   "main_call_on_equal_bytes": {"T": T_eq, "us": us_e, "algorithmic_mb": by_e / 1e6,
+                                                                "gbs": by_e / us_e / 1e3, "frac": by_e / us_e / 1e3 / peaks["hbm"]}}
+        del sets
+        torch.cuda.empty_cache()
+    # prefill: CHAI-QKV (one plain head per cluster: k QK^T and k PV products) and head_dim 64 at workload 5's shape
+    case = synth.prefill_case(seed=0, device=device)
+    Bp, Hp, Tp, Dp, kp = case["B"], case["H"], case["T"], case["D"], case["k"]
+    k_rep = chai.chai_compact_k_cache(case["k_full"], case["reps"])
+    v_rep = torch.stack([case["v"][b].index_select(0, case["reps"][b].long()) for b in range(Bp)])
+    ws = chai.new_workspace(int(chai.load().chai_prefill_qkv_workspace_bytes(Bp, Hp, kp, Tp, Dp, chai.CHAI_BF16)), device)
+    out = torch.empty_like(case["q_full"])
+    us = graph_time_us(lambda: chai.chai_prefill_attention_qkv(case["q_full"], k_rep, v_rep, case["membership"], case["reps"],
+                                                                case["scale"], True, out=out, workspace=ws), 1)
+    fl = 2 * Dp * (Tp * (Tp + 1) // 2) * (2 * kp) * Bp
+    res["prefill_qkv"] = {"workload": "workload 5's shape, values of the k representatives only", "us": us,
+                          "algorithmic_gflop": fl / 1e9, "tflops": fl / us / 1e6, "frac": fl / us / 1e6 / peaks["tf_burst"],
+                          "output_mb": out.numel() * 2 / 1e6,
+                          "note": "2k contractions per request instead of k + H: the call is bound by writing the H output planes"}
+    del case, k_rep, v_rep, out, ws
+    g = torch.Generator(device=device).manual_seed(64)
+    D64 = 64
+    mem, reps = synth.batch_partitions(Bp, Hp, kp, "even", 0, 5, 0)
+    mem, reps = torch.as_tensor(mem, device=device), torch.as_tensor(reps, device=device)
+    q = (torch.randn((Bp, Hp, Tp, D64), device=device, generator=g) * 0.5).to(torch.bfloat16)
+    kr = (torch.randn((Bp, kp, Tp, D64), device=device, generator=g) * 0.5).to(torch.bfloat16)
+    v = (torch.randn((Bp, Hp, Tp, D64), device=device, generator=g) * 0.5).to(torch.bfloat16)
+    ws = chai.new_workspace(chai.chai_prefill_workspace_bytes(Bp, Hp, kp, Tp, D64, chai.CHAI_BF16), device)
+    out = torch.empty_like(q)
+    us = graph_time_us(lambda: chai.chai_prefill_attention(q, kr, v, mem, reps, 0.125, True, out=out, workspace=ws), 1)
+    fl = prefill_flops(Bp, Hp, kp, Tp, D64)
+    res["prefill_head_dim_64"] = {"workload": "B 4, T 2048, H 32, k 8, head_dim 64 (items of four members)", "us": us,
+                                  "algorithmic_gflop": fl / 1e9, "tflops": fl / us / 1e6, "frac": fl / us / 1e6 / peaks["tf_burst"]}
+    return res
+
+
 def bench_decode_workload(cfg_id, device, peaks, steps=10, warmup=3):
     """The decode step of another workload, timed like the headline: the step's layer calls captured once in a CUDA
     graph and replayed `steps` times back to back (every layer has its own caches: tens of GB per step)."""
@@ -757,7 +858,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: keep only the first N layers (not a bench result)")
     ap.add_argument("--skip-extras", action="store_true", help="only the decode step (no prefill/compaction/CPU legs)")
     ap.add_argument("--no-graph", action="store_true", help="time eager launches instead of a replayed CUDA graph")
-    ap.add_argument("--only", default="", choices=["", "prefill", "compaction", "serving", "fp8", "config1", "workload3", "workload4"],
+    ap.add_argument("--only", default="", choices=["", "prefill", "compaction", "serving", "fp8", "config1", "workload3", "workload4", "variants"],
                     help="profiling aid: run just this leg and print its object (not the bench line)")
     ap.add_argument("--record-traffic", default="", metavar="NCU_CSV",
                     help="no GPU work: parse an ncu CSV of `--workload W --layers N --skip-extras` into the tracked DRAM-traffic record")
@@ -790,7 +891,8 @@ def main():
     peaks = load_peaks()
     if args.only:
         leg = {"prefill": bench_prefill, "compaction": bench_compaction, "serving": bench_serving, "fp8": bench_fp8,
-               "config1": lambda d, p: bench_config1(d), "workload3": lambda d, p: bench_decode_workload(3, d, p),
+               "config1": lambda d, p: bench_config1(d), "variants": bench_variants,
+               "workload3": lambda d, p: bench_decode_workload(3, d, p),
                "workload4": lambda d, p: bench_decode_workload(4, d, p)}[args.only]
         print(json.dumps({"leg": args.only, "result": leg(device, peaks)}))
         ranks.close()
@@ -919,6 +1021,7 @@ def main():
             line["serving"] = bench_serving(device, peaks)
             line["fp8_decode"] = bench_fp8(device, peaks)
             line["config1"] = bench_config1(device)
+            line["variants"] = bench_variants(device, peaks)
             others = {f"workload{c}": bench_decode_workload(c, device, peaks) for c in (3, 4) if c != args.workload}
             line["decode_other_workloads"] = others
             # Compact summaries of the other legs inside the roofline object, so that this one object carries the
@@ -942,6 +1045,11 @@ def main():
                                    "us_over_full_length_us_times_byte_ratio": sv["ragged_decode"]["back_to_back"]["us_over_full_length_us_times_byte_ratio"]}
             rl["fp8_decode"] = {k2: {"us_per_layer": line["fp8_decode"][k2]["us_per_layer"], "achieved": line["fp8_decode"][k2]["gbs"],
                                      "frac": line["fp8_decode"][k2]["roofline"]["frac"]} for k2 in ("k8", "k32")}
+            vr = line["variants"]
+            rl["variants"] = {"decode_qkv_k8": {k2: vr["decode_qkv_k8"][k2] for k2 in ("us", "gbs", "frac")},
+                              "decode_qkv_k16": {k2: vr["decode_qkv_k16"][k2] for k2 in ("us", "gbs", "frac")},
+                              "prefill_qkv": {k2: vr["prefill_qkv"][k2] for k2 in ("us", "tflops", "frac")},
+                              "prefill_head_dim_64": {k2: vr["prefill_head_dim_64"][k2] for k2 in ("us", "tflops", "frac")}}
             line["cpu_baseline"] = cpu_baseline_decode(args.workload, 0)
             line["cpu_baseline"]["prefill"] = cpu_baseline_prefill()
         print(json.dumps(line))

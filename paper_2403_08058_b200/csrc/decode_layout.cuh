@@ -76,6 +76,9 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
                              const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T,
                              int T_cap, int D, size_t k_batch_stride, float scale, int dtype, char* ws,
                              const DecodeLayout& L, cudaStream_t s, const float* k_scale = nullptr,
-                             const float* v_scale = nullptr);  // scales: fp8 caches only (dtype CHAI_FP8_E4M3)
+                             const float* v_scale = nullptr,  // scales: fp8 caches only (dtype CHAI_FP8_E4M3)
+                             // CHAI-QKV: H = k heads (the clusters), reps names representatives among the Hq heads of
+                             // q / out, and out_membership [B,Hq] says which heads receive each cluster's row
+                             const int32_t* out_membership = nullptr, int Hq = 0);
 
 }  // namespace chai

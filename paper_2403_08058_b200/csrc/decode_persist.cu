@@ -125,6 +125,12 @@ struct Params {
     int IV, nVi;                 // tiles per value item, items per head
     float scale;
     long long wait_limit;        // cycles after which a device-side wait gives up
+    // CHAI-QKV (values of non-representative heads dropped too): the kernel's heads are the k clusters themselves
+    // (H = k, v = the representatives' value planes), `reps` still names each cluster's representative among the
+    // Hq heads that q and out have, and a cluster's output row is written to every head that out_membership [B,Hq]
+    // assigns to it.  Null: the ordinary case, Hq = H and every head writes its own row.
+    const int32_t* out_membership;
+    int Hq;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -406,11 +412,19 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 0) sm.epoch = *reinterpret_cast<volatile unsigned*>(&P.hdr->pad[8]);
-    if (use_table) {
-        for (int i = tid; i < B * H; i += THREADS) {
-            int c, r;
-            sm.table[i] = resolve_head(P.membership, P.reps, i / H, i % H, H, k, &c, &r) ? c : -1;
+    const bool qkv = P.out_membership != nullptr;
+    // head -> cluster, or -1.  CHAI-QKV: head c of request b is cluster c, usable when its representative is one
+    // of the Hq heads and belongs to it.
+    auto resolve_cluster = [&](int b, int h) -> int {
+        if (qkv) {
+            const int r = P.reps[(size_t)b * k + h];
+            return (r >= 0 && r < P.Hq && P.out_membership[(size_t)b * P.Hq + r] == h) ? h : -1;
         }
+        int c, r;
+        return resolve_head(P.membership, P.reps, b, h, H, k, &c, &r) ? c : -1;
+    };
+    if (use_table) {
+        for (int i = tid; i < B * H; i += THREADS) sm.table[i] = resolve_cluster(i / H, i % H);
     }
     // A ragged batch is dealt by what it really holds: with the running sums of every request's key tiles and value
     // items in shared memory, the producer walks (or claims) positions in the list of existing tiles and items, so
@@ -458,8 +472,25 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
     const unsigned long long token = ((unsigned long long)sm.epoch << 32) | (P.token & 0xffffffffull);
     auto cluster_of = [&](int b, int h) -> int {
         if (use_table) return sm.table[b * H + h];
-        int c, r;
-        return resolve_head(P.membership, P.reps, b, h, H, k, &c, &r) ? c : -1;
+        return resolve_cluster(b, h);
+    };
+    // A finished head's output row (lane l holds columns l * DPL ..).  CHAI-QKV: the row goes to every head of the
+    // cluster, found by walking the request's membership.
+    auto store_row = [&](int head, const float* vals) {
+        constexpr int DPL = D / 32;
+        TQ* outp = static_cast<TQ*>(P.out);
+        if (!qkv) {
+#pragma unroll
+            for (int e = 0; e < DPL; ++e) outp[(size_t)head * D + lane * DPL + e] = from_float<TQ>(vals[e]);
+            return;
+        }
+        const int b = head / H, c = head % H;
+        const int32_t* mem = P.out_membership + (size_t)b * P.Hq;
+        for (int h = 0; h < P.Hq; ++h)
+            if (__ldg(mem + h) == c) {
+#pragma unroll
+                for (int e = 0; e < DPL; ++e) outp[((size_t)b * P.Hq + h) * D + lane * DPL + e] = from_float<TQ>(vals[e]);
+            }
     };
     // rows of request b's tile: requests shorter than T leave whole tiles empty (they pass through the ring as
     // markers without data and contribute nothing)
@@ -649,13 +680,13 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             const int b = plane / k;
             const int rows = tile_rows(b, tile);
             const int rep = P.reps[plane];
-            const bool live = rep >= 0 && rep < H;  // unused cluster slot: the tile is drained, nothing computed
+            const bool live = rep >= 0 && rep < P.Hq;  // unused cluster slot: the tile is drained, nothing computed
             float qf[G::EPV];
 #pragma unroll
             for (int e = 0; e < G::EPV; ++e) qf[e] = 0.f;
             if (live) {
                 // the EPV query elements that face this lane's 16-byte slice of a key row
-                const TQ* qsrc = static_cast<const TQ*>(P.q) + ((size_t)b * H + rep) * D + part * G::EPV;
+                const TQ* qsrc = static_cast<const TQ*>(P.q) + ((size_t)b * P.Hq + rep) * D + part * G::EPV;
 #pragma unroll
                 for (int x = 0; x < G::EPV / Vec16<TQ>::N; ++x)
                     Vec16<TQ>::unpack(*reinterpret_cast<const uint4*>(qsrc + x * Vec16<TQ>::N), qf + x * Vec16<TQ>::N);
@@ -844,8 +875,23 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
             } else if (chunk == 0 && m.t == 0) {
                 // unresolved head: zero output, flagged after the status reset (ordered by the layer's first flag)
                 ok = flags_wait(P.flags, 1, token, lane, abort_flag);
-                if (ok && lane == 0) flag_bad_membership(P.hdr, b, h);
-                for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<TQ>(0.f);
+                if (!qkv) {
+                    if (ok && lane == 0) flag_bad_membership(P.hdr, b, h);
+                    for (int d = lane; d < D; d += 32) outp[(size_t)head * D + d] = from_float<TQ>(0.f);
+                }
+            }
+            if (qkv && ok && chunk == 0 && m.t == 0) {
+                // CHAI-QKV, once per (request, cluster): the heads that name an unusable cluster get zero rows and
+                // are reported; cluster 0's item also takes the heads whose cluster id is out of range.
+                if (!live || h == 0) ok = flags_wait(P.flags, 1, token, lane, abort_flag);  // after the status reset
+                const int32_t* mem = P.out_membership + (size_t)b * P.Hq;
+                for (int hh = 0; hh < P.Hq && ok; ++hh) {
+                    const int cc = __ldg(mem + hh);
+                    const bool mine = (!live && cc == h) || (h == 0 && (cc < 0 || cc >= k));
+                    if (!mine) continue;
+                    if (lane == 0) flag_bad_membership(P.hdr, b, hh);
+                    for (int d = lane; d < D; d += 32) outp[((size_t)b * P.Hq + hh) * D + d] = from_float<TQ>(0.f);
+                }
             }
             // now the tile's bytes
             if (ok) ok = __all_sync(0xffffffffu, mbar_wait(ring.full(slot), (n / STAGES) & 1, abort_flag));
@@ -969,9 +1015,10 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 const GroupedSum<D / 32> gs = combine_grouped<D>(P.opart, P.lpart, P.gcnt, P.counters, P.nVi, P.capG, head, chunk, n_chunks, lane);
                 if (gs.done) {
                     const float vscale = P.v_scale ? __ldg(P.v_scale + head) : 1.f;
+                    float fin[D / 32];
 #pragma unroll
-                    for (int e = 0; e < D / 32; ++e)
-                        outp[(size_t)head * D + lane * (D / 32) + e] = from_float<TQ>(gs.l > 0.f ? gs.o[e] / gs.l * vscale : 0.f);
+                    for (int e = 0; e < D / 32; ++e) fin[e] = gs.l > 0.f ? gs.o[e] / gs.l * vscale : 0.f;
+                    store_row(head, fin);
                 }
                 continue;
             }
@@ -1008,8 +1055,8 @@ __global__ void __launch_bounds__(Cfg<T>::W * 32 + 32, 1) decode_persistent_kern
                 }
                 const float vscale = P.v_scale ? __ldg(P.v_scale + head) : 1.f;  // fp8 values carry a scale per plane
 #pragma unroll
-                for (int e = 0; e < DPL; ++e)  // (an empty context has no probabilities: the output is zero)
-                    outp[(size_t)head * D + lane * DPL + e] = from_float<TQ>(ll > 0.f ? o[e] / ll * vscale : 0.f);
+                for (int e = 0; e < DPL; ++e) o[e] = ll > 0.f ? o[e] / ll * vscale : 0.f;  // (an empty context has no probabilities: the output is zero)
+                store_row(head, o);
             }
         }
     }
@@ -1090,7 +1137,8 @@ static int launch(const Params& P0, int ncta, int dev, cudaStream_t s) {
 int launch_decode_persistent(const void* q, const void* k_rep, const void* v, const int32_t* membership,
                              const int32_t* reps, const int32_t* seq_lens, void* out, int B, int H, int k, int T,
                              int T_cap, int D, size_t k_batch_stride, float scale, int dtype, char* ws,
-                             const DecodeLayout& L, cudaStream_t s, const float* k_scale, const float* v_scale) {
+                             const DecodeLayout& L, cudaStream_t s, const float* k_scale, const float* v_scale,
+                             const int32_t* out_membership, int Hq) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return kDecodeNotLaunched;
     pd::DeviceInfo info;
@@ -1128,6 +1176,8 @@ int launch_decode_persistent(const void* q, const void* k_rep, const void* v, co
     P.nVi = (tiles + P.IV - 1) / P.IV;
     P.scale = scale;
     P.wait_limit = decode_wait_limit_cycles();
+    P.out_membership = out_membership;
+    P.Hq = out_membership != nullptr ? Hq : H;
     if (tiles > L.capK || P.nVi > L.capV || (long long)B * H * P.nVi > 0x7fffffffll ||
         (long long)B * k * tiles > 0x7fffffffll)  // item and key-tile ids travel as ints
         return kDecodeNotLaunched;

@@ -7,7 +7,7 @@
 //       each cluster's output to all of its members.
 //   CHAI-static (Section 3.5): one membership, found offline, is used for every request: the per-request
 //       arrays the other entry points expect are then B copies of it (chai_broadcast_membership).
-#include "chai_common.cuh"
+#include "decode_layout.cuh"
 
 namespace chai {
 
@@ -118,6 +118,17 @@ int chai_decode_attention_qkv(const void* q, const void* k_rep, const void* v_re
                  workspace_bytes, L.total);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
+    // One launch of the streaming decode kernel with the k clusters as its heads: it reads each representative's
+    // query row where it lies among the H heads and writes a cluster's row to all of its member heads itself.
+    CHAI_REQUIRE(T <= T_cap, CHAI_ERR_INVALID_ARG, "%s: T=%d exceeds T_cap=%d", fn, T, T_cap);
+    CHAI_REQUIRE(aligned16(k_rep) && aligned16(v_rep), CHAI_ERR_INVALID_ARG, "%s: pointers must be 16-byte aligned", fn);
+    DecodeLayout DL;
+    if (decode_layout(B, k, k, T, D, dtype, &DL) && DL.total <= inner) {
+        const int rc = launch_decode_persistent(q, k_rep, v_rep, membership, reps, seq_lens, out, B, k, k, T, T_cap, D,
+                                                (size_t)k * T_cap * D, scale, dtype, ws, DL, s, nullptr, nullptr, membership, H);
+        if (rc != kDecodeNotLaunched) return rc;
+    }
+    // (devices without cooperative launch: gather the query rows, run the k-head problem, copy to the members)
     int32_t* ident = reinterpret_cast<int32_t*>(ws + L.off_ident);
     const size_t vecs = (size_t)D * elem_size(dtype) / 16;
     CHAI_LAUNCH_DEPENDENT("gather_rep_rows_kernel launch", gather_rep_rows_kernel, dim3(1, k, B), dim3(32), 0, s,
