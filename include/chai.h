@@ -32,6 +32,8 @@
  *     the kernels record CHAI_ERR_BAD_MEMBERSHIP in the status word at the head of
  *     the workspace, give the affected heads an all-zero output and never form an
  *     out-of-range address.  Read the word with chai_device_status.
+ *   - Logging: with CHAI_LOG=1 in the environment (read once per process) the main entry points
+ *     write one line per call to stderr: their name, the shapes, and what they launch.
  *   - dtype: CHAI_F32 or CHAI_BF16 for Q, K, V and the output; accumulation is
  *     always fp32.  Head dimension D must be 64 or 128.
  *   - T counts cached positions INCLUDING the current token; T_cap (>= T) is the

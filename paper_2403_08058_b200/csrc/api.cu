@@ -1,5 +1,6 @@
 // Status plumbing of libchai: error text, status strings, the blocking status-word read.
 #include <stdarg.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "chai_common.cuh"
@@ -18,6 +19,23 @@ void set_last_error(const char* fmt, ...) {
 // Cycle limit of the decode kernel's device-side waits (see chai_set_decode_wait_limit_cycles).
 static std::atomic<long long> g_decode_wait_limit{kDefaultWaitLimitCycles};
 long long decode_wait_limit_cycles() { return g_decode_wait_limit.load(std::memory_order_relaxed); }
+
+// CHAI_LOG=1 in the environment: one line per call on stderr (entry point, shapes, what was launched).
+bool log_enabled() {
+    static const bool on = [] {
+        const char* e = getenv("CHAI_LOG");
+        return e != nullptr && e[0] != '\0' && e[0] != '0';
+    }();
+    return on;
+}
+void log_line(const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    fprintf(stderr, "[chai] %s\n", buf);
+}
 
 int cuda_fail(cudaError_t e, const char* what) {
     set_last_error("%s: %s", what, cudaGetErrorString(e));

@@ -36,6 +36,12 @@ constexpr long long kDefaultWaitLimitCycles = 2000000000ll;
 long long decode_wait_limit_cycles();  // current limit of the decode kernel's waits (api.cu)
 
 void set_last_error(const char* fmt, ...);
+bool log_enabled();                      // CHAI_LOG set in the environment (read once)
+void log_line(const char* fmt, ...);     // one line on stderr
+#define CHAI_LOG_CALL(...)                                   \
+    do {                                                     \
+        if (::chai::log_enabled()) ::chai::log_line(__VA_ARGS__); \
+    } while (0)
 int cuda_fail(cudaError_t e, const char* what);  // records the text, returns CHAI_ERR_CUDA
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -390,6 +390,8 @@ int chai_cluster_heads(const float* features, int B, int H, int F, int k, int ma
     CHAI_REQUIRE(H <= 1024 && smem <= 200 * 1024, CHAI_ERR_UNSUPPORTED,
                  "chai_cluster_heads: problem needs %zu bytes of shared memory (limit 204800)", smem);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CHAI_LOG_CALL("chai_cluster_heads: B=%d H=%d F=%d k=%d max_iter=%d seed=%llu, %d CTAs x 256 threads, %zu bytes of shared memory",
+                  B, H, F, k, max_iter, (unsigned long long)seed, B, smem);
     cudaError_t e = cudaFuncSetAttribute(kmeans_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return cuda_fail(e, "kmeans_kernel shared-memory opt-in");
     CHAI_LAUNCH_DEPENDENT("kmeans_kernel launch", kmeans_kernel, dim3(B), dim3(256), smem, s, features, H, F, k, max_iter,

@@ -57,6 +57,8 @@ extern "C" int chai_compact_k_cache(const void* k_full, void* k_rep, const int32
     dim3 grid((unsigned)((copy_vec + per_cta - 1) / per_cta), k, B);
     // an ordinary launch: as a programmatic dependent of the clustering kernel this grid of hundreds of CTAs made
     // the prefill flow 4 us slower (measured)
+    CHAI_LOG_CALL("chai_compact_k_cache: B=%d H=%d k=%d T=%d T_cap=%d D=%d dtype=%d, %zu bytes gathered", B, H, k, T, T_cap, D, dtype,
+                  (size_t)B * k * T * D * elem_size(dtype));
     compact_k_kernel<<<grid, kCompactThreads, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint4*>(k_full), static_cast<uint4*>(k_rep), reps, H, k, plane_cap_vec, copy_vec);
     CHAI_LAUNCH_CHECK("compact_k_kernel launch");

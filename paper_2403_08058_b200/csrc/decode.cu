@@ -278,6 +278,9 @@ int decode_impl(const char* fn, const void* q, const void* k_rep, const void* v,
         const char* e = getenv("CHAI_DECODE_IMPL");
         return e != nullptr && strcmp(e, "split") == 0;
     }();
+    CHAI_LOG_CALL("%s: B=%d H=%d k=%d T=%d T_cap=%d D=%d dtype=%d %s%s workspace=%zu of %zu bytes, kernel=%s", fn, B, H, k, T, T_cap,
+                  D, dtype, seq_lens ? "ragged " : "", k_batch_stride != dense ? "strided-K " : "", L.total, workspace_bytes,
+                  force_split ? "split (CHAI_DECODE_IMPL)" : "persistent, one CTA per SM");
     if (!force_split) {
         const int rc = launch_decode_persistent(q, k_rep, v, membership, reps, seq_lens, out, B, H, k, T, T_cap, D,
                                                 k_batch_stride, scale, dtype, ws, L, s);

@@ -164,6 +164,8 @@ int chai_decode_attention_fp8(const void* q, const void* k_rep, const void* v, c
     decode_layout(B, H, k, T, D, CHAI_FP8_E4M3, &L);
     CHAI_REQUIRE(workspace_bytes >= L.total, CHAI_ERR_WORKSPACE, "%s: workspace has %zu bytes, %zu needed", fn,
                  workspace_bytes, L.total);
+    CHAI_LOG_CALL("chai_decode_attention_fp8: B=%d H=%d k=%d T=%d T_cap=%d D=%d %se4m3 caches, persistent kernel, one CTA per SM", B, H, k,
+                  T, T_cap, D, seq_lens ? "ragged " : "");
     const int rc = launch_decode_persistent(q, k_rep, v, membership, reps, seq_lens, out, B, H, k, T, T_cap, D,
                                             k_batch_stride, scale, CHAI_FP8_E4M3, static_cast<char*>(workspace), L,
                                             static_cast<cudaStream_t>(stream), k_scale, v_scale);

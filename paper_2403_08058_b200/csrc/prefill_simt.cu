@@ -217,6 +217,8 @@ int chai_prefill_attention_simt_from(const void* q, const void* k_rep, const voi
                  q_start, T);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
+    CHAI_LOG_CALL("%s: B=%d H=%d k=%d T=%d q_start=%d D=%d causal=%d dtype=%d CUDA-core kernel, grid (%d, %d, %d)", fn, B, H, k, T,
+                  q_start, D, causal, dtype, (T + kSimtBQ - 1) / kSimtBQ - q_start / kSimtBQ, H, B);
     rc = prefill_run_plan(membership, reps, B, H, k, kSimtG, ws, s);
     if (rc != CHAI_OK) return rc;
     const PrefillLayout L = prefill_layout(B, H);

@@ -733,6 +733,9 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
     if (rc != CHAI_OK) return rc;
     const int n_sms = sms_of_device[dev];
     const int n_qtiles = (T + tc::BM - 1) / tc::BM;
+    CHAI_LOG_CALL("chai_prefill_attention: B=%d H=%d k=%d T=%d q_start=%d D=%d causal=%d tensor-core kernel, %d CTAs x %d threads, "
+                  "%d query tiles, %d launch(es), members per item <= %d", B, H, k, T, q_start, D, causal, n_sms, tc::THREADS,
+                  n_qtiles - q_start / tc::BM, (B + tc::MAX_B - 1) / tc::MAX_B, D == 128 ? 2 : 4);
     // one persistent CTA per SM; requests are processed in chunks of MAX_B (the per-request group counts of
     // a chunk are kept in shared memory), each chunk with its own work counter in the workspace header
     for (int b0 = 0, chunk = 0; b0 < B; b0 += tc::MAX_B, ++chunk) {

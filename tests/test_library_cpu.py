@@ -135,3 +135,19 @@ def test_binding_signatures_match_the_header(lib):
                 assert ct is ctypes.c_float, where
             else:
                 assert ct is ctypes.c_int, where
+
+
+def test_chai_log_prints_one_line_per_call():
+    """CHAI_LOG=1: an entry point writes a line with its shapes and launch plan to stderr before it launches (here
+    the launch itself cannot happen without a device; the pointers are never dereferenced on the host)."""
+    import subprocess
+    import sys
+    code = (
+        "import sys; sys.path.insert(0, %r)\n"
+        "from paper_2403_08058_b200 import chai\n"
+        "lib = chai.load()\n"
+        "lib.chai_cluster_heads(256, 2, 32, 64, 8, 20, 7, 256, 256, 256, None, None)\n" % ROOT)
+    for flag, expect in (("1", True), ("0", False)):
+        r = subprocess.run([sys.executable, "-c", code], env=dict(os.environ, CHAI_LOG=flag), capture_output=True, text=True)
+        assert r.returncode == 0, r.stderr
+        assert ("[chai] chai_cluster_heads: B=2 H=32 F=64 k=8 max_iter=20 seed=7" in r.stderr) == expect, r.stderr
