@@ -21,6 +21,10 @@
 // N = 64 x members serves them all.
 // Every mbarrier wait is bounded: on expiry the CTA records CHAI_ERR_TIMEOUT in the workspace
 // status word, skips the rest of its work, frees its tensor memory and returns.
+// CHAI-QKV (Table 4: the values of non-representative heads are dropped too) is a third instantiation: the work
+// items are the clusters themselves (one accumulator: the representative's Q, K and V), the representative's
+// query tile is read where it lies among the H heads, and the epilogue writes a finished row to every head that
+// the membership assigns to the cluster.
 #include <cuda.h>
 #include <stdlib.h>
 #include <string.h>
@@ -121,13 +125,16 @@ static_assert(sizeof(ItemT<2>) == 32 && sizeof(ItemT<4>) == 48, "item descriptor
 // by an atomic counter in descending order of cost.  While the softmax warps finish one item, the
 // producer is already fetching the next item's Q, K and V tiles and the tensor core computes its
 // first scores, so the pipeline fill of an item hides behind the drain of the previous one.
-template <int HD>
+template <int HD, bool QKV>
 __global__ void __launch_bounds__(THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const int* __restrict__ n_groups,
                   const GroupEntry* __restrict__ groups, __nv_bfloat16* __restrict__ out, WsHeader* __restrict__ hdr,
                   const int* __restrict__ bad, int B_total, int b_begin, int B, int H, int k, int T_len, int q_start,
-                  float scale_log2, int causal, int n_qtiles, int counter_slot) {
+                  float scale_log2, int causal, int n_qtiles, int counter_slot, const int32_t* __restrict__ qkv_membership,
+                  int Hq, int group_stride) {
+    // QKV: H is the number of clusters (the heads of K_rep and V_rep), Hq the number of heads of q and out, and
+    // qkv_membership [B_total, Hq] says which of those heads receive a cluster's rows.
     static_assert(HD == 128 || HD == 64, "head_dim 128 or 64");
     constexpr int LOAD_BYTES = BN * HD * 2;  // bytes one tile copy brings
     // stride between the 64-column blocks an MN-major V operand walks: the two halves of a 128-wide tile, or
@@ -216,7 +223,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (prefix[mid] <= pair) lo = mid; else hi = mid;
                 }
                 c.b = b_begin + lo;
-                c.e = groups[(size_t)c.b * H + (pair - prefix[lo])];
+                c.e = groups[(size_t)c.b * group_stride + (pair - prefix[lo])];
             };
             Claim cur, nxt;
             cur.id = atomicAdd(&hdr->pad[counter_slot], 1);  // (the counter was cleared by the planning kernel)
@@ -237,7 +244,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const int n_members = min(e.n, GM);
                 item.q0 = qt * BM;
                 item.n_members = n_members;
-                for (int g = 0; g < GM; ++g) item.o_plane[g] = b * H + e.heads[g < n_members ? g : 0];
+                // (CHAI-QKV: a zero-fill item names heads of the output, a computing item its cluster)
+                for (int g = 0; g < GM; ++g) item.o_plane[g] = b * ((QKV && e.cluster < 0) ? Hq : H) + e.heads[g < n_members ? g : 0];
                 if (e.cluster < 0) {                       // unresolved heads: zero rows, nothing to load
                     item.n_kv = 0;
                     item.q_plane = item.k_plane = 0;
@@ -249,7 +257,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 }
                 const int n_kv = causal ? min(qt + 1, (T_len + BN - 1) / BN) : (T_len + BN - 1) / BN;
                 item.n_kv = n_kv;
-                item.q_plane = b * H + e.rep;
+                item.q_plane = b * (QKV ? Hq : H) + e.rep;
                 item.k_plane = b * k + e.cluster;
                 mbar_arrive(bar.item_full(is));
                 const int q_plane = item.q_plane, k_plane = item.k_plane, q0 = item.q0;
@@ -617,7 +625,32 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                             for (int x = ep.n_members; x < GM; ++x) mbar_arrive(bar.o_free(x));
                     }
                 }
-                if (row_abs >= q_start && row_abs < T_len) {  // rows before q_start belong to the caller
+                if constexpr (QKV) {
+                    // the cluster's row goes to every head of the cluster: the warp finds them 32 heads at a time
+                    uint32_t w[16];
+#pragma unroll
+                    for (int x = 0; x < 16; ++x) {
+                        float y0, y1;
+                        unpack2(mul2(pack2(__uint_as_float(cur[2 * x]), __uint_as_float(cur[2 * x + 1])), inv2), y0, y1);
+                        __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+                        w[x] = *reinterpret_cast<uint32_t*>(&pk);
+                    }
+                    const int bq = ep.o_plane[0] / H, cq = ep.o_plane[0] % H;
+                    const bool row_live = row_abs >= q_start && row_abs < T_len;
+                    for (int h0 = 0; h0 < Hq; h0 += 32) {
+                        const int hh = h0 + lane;
+                        unsigned members = __ballot_sync(0xffffffffu, hh < Hq && __ldg(qkv_membership + (size_t)bq * Hq + hh) == cq);
+                        while (members) {
+                            const int h = h0 + __ffs(members) - 1;
+                            members &= members - 1;
+                            if (row_live) {
+                                __nv_bfloat16* orow = out + (((size_t)bq * Hq + h) * T_len + row_abs) * HD + sc * 32;
+                                st_global_32B(orow, w);
+                                st_global_32B(orow + 16, w + 8);
+                            }
+                        }
+                    }
+                } else if (row_abs >= q_start && row_abs < T_len) {  // rows before q_start belong to the caller
                     __nv_bfloat16* orow = out + ((size_t)ep.o_plane[g] * T_len + row_abs) * HD + sc * 32;
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
@@ -689,43 +722,86 @@ extern "C" int chai_prefill_attention_simt_from(const void* q, const void* k_rep
                                                 int D, float scale, int causal, int dtype, void* workspace,
                                                 size_t workspace_bytes, void* stream);
 
-extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, const void* v, const int32_t* membership,
-                                           const int32_t* reps, void* out, int B, int H, int k, int T, int q_start, int D,
-                                           float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
-                                           void* stream) {
-    using namespace chai;
-    // The tensor-core kernel takes a row's largest raw score and scales it afterwards, which is the largest scaled
-    // score only for a positive, finite scale; anything else goes to the CUDA-core kernel, which scales first.
-    if (dtype != CHAI_BF16 || (D != 128 && D != 64) || B > 60 * tc::MAX_B || !(scale > 0.f) || !(scale <= 3.0e38f))
-        return chai_prefill_attention_simt_from(q, k_rep, v, membership, reps, out, B, H, k, T, q_start, D, scale, causal,
-                                                dtype, workspace, workspace_bytes, stream);
-    int rc = prefill_check_args("chai_prefill_attention", q, k_rep, v, membership, reps, out, B, H, k, T, D, dtype,
-                                workspace, workspace_bytes);
-    if (rc != CHAI_OK) return rc;
-    CHAI_REQUIRE(q_start >= 0 && q_start < T, CHAI_ERR_INVALID_ARG,
-                 "chai_prefill_attention: need 0 <= q_start < T (q_start=%d, T=%d)", q_start, T);
+namespace chai {
+
+// Plan of CHAI-QKV prefill: one group per usable cluster (cluster c, its representative among the Hq heads, one
+// "member": the cluster itself), then zero-fill groups of up to gmax heads for the heads that name no usable cluster.
+// grid B, block 128, k ints of shared memory.
+static __global__ void __launch_bounds__(128)
+prefill_plan_qkv_kernel(const int32_t* __restrict__ membership, const int32_t* __restrict__ reps, WsHeader* __restrict__ hdr,
+                        int* __restrict__ n_groups, int* __restrict__ bad_out, GroupEntry* __restrict__ groups, int Hq, int k,
+                        int gmax, int group_stride) {
+    extern __shared__ __align__(16) int s_live[];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    dependent_grid_sync();
+    if (b == 0)
+        for (int i = tid; i < 60; i += blockDim.x) hdr->pad[i] = 0;
+    const int32_t* mem = membership + (size_t)b * Hq;
+    for (int c = tid; c < k; c += blockDim.x) {
+        const int r = reps[(size_t)b * k + c];
+        s_live[c] = (r >= 0 && r < Hq && mem[r] == c) ? r : -1;
+    }
+    __syncthreads();
+    if (tid != 0) return;
+    GroupEntry* out = groups + (size_t)b * group_stride;
+    int ng = 0;
+    for (int c = 0; c < k; ++c)
+        if (s_live[c] >= 0) {
+            int4* dst = reinterpret_cast<int4*>(out + ng++);
+            dst[0] = make_int4(c, s_live[c], 1, 0);
+            dst[1] = make_int4(c, c, c, c);
+        }
+    int cnt = 0, first_bad = -1, hd[kGroupMax] = {0, 0, 0, 0};
+    for (int h = 0; h < Hq; ++h) {
+        const int c = mem[h];
+        if (c >= 0 && c < k && s_live[c] >= 0) continue;
+        if (first_bad < 0) first_bad = h;
+        if (cnt == 0)
+            for (int x = 0; x < kGroupMax; ++x) hd[x] = h;
+        for (int x = 0; x < kGroupMax; ++x)
+            if (x == cnt) hd[x] = h;
+        if (++cnt == gmax) {
+            int4* dst = reinterpret_cast<int4*>(out + ng++);
+            dst[0] = make_int4(-1, -1, cnt, 0);
+            dst[1] = make_int4(hd[0], hd[1], hd[2], hd[3]);
+            cnt = 0;
+        }
+    }
+    if (cnt > 0) {
+        int4* dst = reinterpret_cast<int4*>(out + ng++);
+        dst[0] = make_int4(-1, -1, cnt, 0);
+        dst[1] = make_int4(hd[0], hd[1], hd[2], hd[3]);
+    }
+    n_groups[b] = ng;
+    bad_out[b] = first_bad + 1;
+}
+
+// Launches the tensor-core kernel on a plan that lies in `ws` (layout L).  H: heads per request that the items'
+// value and output planes count (the clusters, for CHAI-QKV); qkv_membership / Hq: see the kernel.
+static int prefill_tc_launch(const char* fn, const void* q, int q_planes, const void* k_rep, const void* v, int v_planes,
+                             void* out, int B, int H, int k, int T, int q_start, int D, float scale, int causal, char* ws,
+                             const PrefillLayout& L, int group_stride, const int32_t* qkv_membership, int Hq, cudaStream_t s) {
     CUtensorMap mq, mk, mv;
-    CHAI_REQUIRE(tc::make_map(&mq, q, B * H, T, D) && tc::make_map(&mk, k_rep, B * k, T, D) && tc::make_map(&mv, v, B * H, T, D),
-                 CHAI_ERR_CUDA, "chai_prefill_attention: cuTensorMapEncodeTiled failed");
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    char* ws = static_cast<char*>(workspace);
-    rc = prefill_run_plan(membership, reps, B, H, k, D == 128 ? 2 : 4, ws, s);
-    if (rc != CHAI_OK) return rc;
-    const PrefillLayout L = prefill_layout(B, H);
+    CHAI_REQUIRE(tc::make_map(&mq, q, q_planes, T, D) && tc::make_map(&mk, k_rep, B * k, T, D) && tc::make_map(&mv, v, v_planes, T, D),
+                 CHAI_ERR_CUDA, "%s: cuTensorMapEncodeTiled failed", fn);
     // per device, once: SM count, and the kernels' opt-in to their shared-memory size
     static PerDeviceOnce once;
     static int sms_of_device[kMaxDevices] = {};
     int dev = 0;
     cudaError_t de = cudaGetDevice(&dev);
     if (de != cudaSuccess) return cuda_fail(de, "prefill_tc_kernel set-up");
-    CHAI_REQUIRE(dev >= 0 && dev < kMaxDevices, CHAI_ERR_UNSUPPORTED, "chai_prefill_attention: device index %d out of range", dev);
-    rc = once.run(dev, [&]() -> int {
+    CHAI_REQUIRE(dev >= 0 && dev < kMaxDevices, CHAI_ERR_UNSUPPORTED, "%s: device index %d out of range", fn, dev);
+    int rc = once.run(dev, [&]() -> int {
         int count = 0;
         cudaError_t e = cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc::prefill_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+            e = cudaFuncSetAttribute(tc::prefill_tc_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(tc::prefill_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+            e = cudaFuncSetAttribute(tc::prefill_tc_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc::prefill_tc_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(tc::prefill_tc_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
         if (e != cudaSuccess) return cuda_fail(e, "prefill_tc_kernel set-up");
         sms_of_device[dev] = count;
         return CHAI_OK;
@@ -733,9 +809,11 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
     if (rc != CHAI_OK) return rc;
     const int n_sms = sms_of_device[dev];
     const int n_qtiles = (T + tc::BM - 1) / tc::BM;
-    CHAI_LOG_CALL("chai_prefill_attention: B=%d H=%d k=%d T=%d q_start=%d D=%d causal=%d tensor-core kernel, %d CTAs x %d threads, "
-                  "%d query tiles, %d launch(es), members per item <= %d", B, H, k, T, q_start, D, causal, n_sms, tc::THREADS,
-                  n_qtiles - q_start / tc::BM, (B + tc::MAX_B - 1) / tc::MAX_B, D == 128 ? 2 : 4);
+    const bool qkv = qkv_membership != nullptr;
+    CHAI_LOG_CALL("%s: B=%d H=%d k=%d T=%d q_start=%d D=%d causal=%d tensor-core kernel%s, %d CTAs x %d threads, "
+                  "%d query tiles, %d launch(es), members per item <= %d", fn, B, qkv ? Hq : H, k, T, q_start, D, causal,
+                  qkv ? " (one item per cluster, rows written to all members)" : "", n_sms, tc::THREADS,
+                  n_qtiles - q_start / tc::BM, (B + tc::MAX_B - 1) / tc::MAX_B, qkv ? 1 : (D == 128 ? 2 : 4));
     // one persistent CTA per SM; requests are processed in chunks of MAX_B (the per-request group counts of
     // a chunk are kept in shared memory), each chunk with its own work counter in the workspace header
     for (int b0 = 0, chunk = 0; b0 < B; b0 += tc::MAX_B, ++chunk) {
@@ -758,15 +836,56 @@ extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, con
         WsHeader* hdr = reinterpret_cast<WsHeader*>(ws);
         const int* bad = reinterpret_cast<const int*>(ws + L.off_bad);
         const float scale_log2 = scale * 1.4426950408889634f;
-        cudaError_t le =
-            D == 128 ? cudaLaunchKernelEx(&cfg, tc::prefill_tc_kernel<128>, mq, mk, mv, ng, gr, o, hdr, bad, B, b0, nb, H, k, T,
-                                          q_start, scale_log2, causal, n_qtiles, chunk)
-                     : cudaLaunchKernelEx(&cfg, tc::prefill_tc_kernel<64>, mq, mk, mv, ng, gr, o, hdr, bad, B, b0, nb, H, k, T,
-                                          q_start, scale_log2, causal, n_qtiles, chunk);
+        auto kernel = D == 128 ? (qkv ? tc::prefill_tc_kernel<128, true> : tc::prefill_tc_kernel<128, false>)
+                               : (qkv ? tc::prefill_tc_kernel<64, true> : tc::prefill_tc_kernel<64, false>);
+        cudaError_t le = cudaLaunchKernelEx(&cfg, kernel, mq, mk, mv, ng, gr, o, hdr, bad, B, b0, nb, H, k, T, q_start, scale_log2,
+                                            causal, n_qtiles, chunk, qkv_membership, Hq, group_stride);
         if (le != cudaSuccess) return cuda_fail(le, "prefill_tc_kernel launch");
         CHAI_LAUNCH_CHECK("prefill_tc_kernel launch");
     }
     return CHAI_OK;
+}
+
+// CHAI-QKV prefill on the tensor-core kernel (bf16, head_dim 64 or 128, at most 60 * 64 requests, positive finite
+// scale); kDecodeNotLaunched-style -1 when the call is outside that range and the caller should take the general path.
+int prefill_qkv_tc(const void* q, const void* k_rep, const void* v_rep, const int32_t* membership, const int32_t* reps,
+                   void* out, int B, int H, int k, int T, int q_start, int D, float scale, int causal, int dtype, void* workspace,
+                   size_t workspace_bytes, cudaStream_t s) {
+    if (dtype != CHAI_BF16 || (D != 128 && D != 64) || B > 60 * tc::MAX_B || !(scale > 0.f) || !(scale <= 3.0e38f)) return -1;
+    const PrefillLayout L = prefill_layout(B, H + k);
+    if (workspace_bytes < L.total || (size_t)k * sizeof(int) > 48 * 1024) return -1;
+    char* ws = static_cast<char*>(workspace);
+    CHAI_LAUNCH_DEPENDENT("prefill_plan_qkv_kernel launch", prefill_plan_qkv_kernel, dim3(B), dim3(128), sizeof(int) * (size_t)k, s,
+                          membership, reps, reinterpret_cast<WsHeader*>(ws), reinterpret_cast<int*>(ws + L.off_ngroups),
+                          reinterpret_cast<int*>(ws + L.off_bad), reinterpret_cast<GroupEntry*>(ws + L.off_groups), H, k,
+                          D == 128 ? 2 : 4, H + k);
+    return prefill_tc_launch("chai_prefill_attention_qkv", q, B * H, k_rep, v_rep, B * k, out, B, k, k, T, q_start, D, scale, causal,
+                             ws, L, H + k, membership, H, s);
+}
+
+}  // namespace chai
+
+extern "C" int chai_prefill_attention_from(const void* q, const void* k_rep, const void* v, const int32_t* membership,
+                                           const int32_t* reps, void* out, int B, int H, int k, int T, int q_start, int D,
+                                           float scale, int causal, int dtype, void* workspace, size_t workspace_bytes,
+                                           void* stream) {
+    using namespace chai;
+    // The tensor-core kernel takes a row's largest raw score and scales it afterwards, which is the largest scaled
+    // score only for a positive, finite scale; anything else goes to the CUDA-core kernel, which scales first.
+    if (dtype != CHAI_BF16 || (D != 128 && D != 64) || B > 60 * tc::MAX_B || !(scale > 0.f) || !(scale <= 3.0e38f))
+        return chai_prefill_attention_simt_from(q, k_rep, v, membership, reps, out, B, H, k, T, q_start, D, scale, causal,
+                                                dtype, workspace, workspace_bytes, stream);
+    int rc = prefill_check_args("chai_prefill_attention", q, k_rep, v, membership, reps, out, B, H, k, T, D, dtype,
+                                workspace, workspace_bytes);
+    if (rc != CHAI_OK) return rc;
+    CHAI_REQUIRE(q_start >= 0 && q_start < T, CHAI_ERR_INVALID_ARG,
+                 "chai_prefill_attention: need 0 <= q_start < T (q_start=%d, T=%d)", q_start, T);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    rc = prefill_run_plan(membership, reps, B, H, k, D == 128 ? 2 : 4, ws, s);
+    if (rc != CHAI_OK) return rc;
+    return prefill_tc_launch("chai_prefill_attention", q, B * H, k_rep, v, B * H, out, B, H, k, T, q_start, D, scale, causal, ws,
+                             prefill_layout(B, H), H, nullptr, H, s);
 }
 
 extern "C" int chai_prefill_attention(const void* q, const void* k_rep, const void* v, const int32_t* membership,

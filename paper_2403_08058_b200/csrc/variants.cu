@@ -2,14 +2,22 @@
 //
 //   CHAI-QKV (Table 4): besides the queries and keys, the VALUES of non-representative heads are dropped
 //       too, so a member head's output IS its representative's output.  Per cluster this is one plain
-//       attention head (the representative's Q, K, V); the entry points below gather the representatives'
-//       query rows, run the library's own attention kernels on the k heads with identity maps, and copy
-//       each cluster's output to all of its members.
+//       attention head (the representative's Q, K, V).  The streaming decode kernel and the tensor-core prefill
+//       kernel take the clusters as their heads / work items, read each representative's query rows where they lie
+//       among the H heads and write a cluster's rows to all of its members (one launch each); where those
+//       kernels do not apply (fp32 prefill, devices without cooperative launch) the entry points gather the
+//       query rows, run the k-head problem with identity maps, and copy each cluster's output to its members.
 //   CHAI-static (Section 3.5): one membership, found offline, is used for every request: the per-request
 //       arrays the other entry points expect are then B copies of it (chai_broadcast_membership).
 #include "decode_layout.cuh"
+#include "prefill_plan.cuh"
 
 namespace chai {
+
+// CHAI-QKV prefill on the tensor-core kernel (prefill_tc.cu); -1 when the call is outside its range.
+int prefill_qkv_tc(const void* q, const void* k_rep, const void* v_rep, const int32_t* membership, const int32_t* reps,
+                   void* out, int B, int H, int k, int T, int q_start, int D, float scale, int causal, int dtype, void* workspace,
+                   size_t workspace_bytes, cudaStream_t s);
 
 // rows of `rows_per_head` * vec_per_row 16-byte vectors per head.
 // gather:  dst[b][c] = src[b][reps[b][c]]   (zero for an unused slot); also writes the identity maps of the
@@ -152,7 +160,9 @@ size_t chai_prefill_qkv_workspace_bytes(int B, int H, int k, int T, int D, int d
     (void)H;
     const size_t inner = chai_prefill_workspace_bytes(B, k, k, T, D, dtype);
     if (inner == 0 || T <= 0 || D <= 0) return 0;
-    return chai::qkv_layout(inner, B, k, (size_t)T * D, dtype).total;
+    const size_t general = chai::qkv_layout(inner, B, k, (size_t)T * D, dtype).total;  // copies of Q rows and outputs
+    const size_t fused = chai::prefill_layout(B, H + k).total;                           // the plan alone
+    return general > fused ? general : fused;
 }
 
 int chai_prefill_attention_qkv(const void* q, const void* k_rep, const void* v_rep, const int32_t* membership,
@@ -176,6 +186,15 @@ int chai_prefill_attention_qkv(const void* q, const void* k_rep, const void* v_r
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     char* ws = static_cast<char*>(workspace);
     int32_t* ident = reinterpret_cast<int32_t*>(ws + L.off_ident);
+    // bf16: one launch of the tensor-core kernel with the clusters as its work items (it reads the representatives'
+    // query tiles in place and writes every member's rows itself)
+    CHAI_REQUIRE(aligned16(k_rep) && aligned16(v_rep), CHAI_ERR_INVALID_ARG, "%s: pointers must be 16-byte aligned", fn);
+    {
+        const int rc = prefill_qkv_tc(q, k_rep, v_rep, membership, reps, out, B, H, k, T, q_start, D, scale, causal, dtype,
+                                      workspace, workspace_bytes, s);
+        if (rc != -1) return rc;
+    }
+    // otherwise: gather the query rows, run the k-head problem, copy each cluster's rows to its members
     const size_t row_vecs = (size_t)D * elem_size(dtype) / 16;
     const size_t vecs = (size_t)T * row_vecs;
     gather_rep_rows_kernel<<<dim3(blocks_for(vecs), k, B), 256, 0, s>>>(

@@ -209,6 +209,58 @@ def test_prefill_qkv(T, q_start, dtype):
     assert_parity(got[:, :, q_start:], ref[:, :, q_start:], dtype, f"QKV prefill T {T} q_start {q_start} {dtype}")
 
 
+@pytest.mark.parametrize("B,H,k,T,D,causal", [(2, 72, 9, 450, 128, True),    # more than 32 heads: members found word by word
+                                               (3, 40, 8, 300, 64, True), (1, 12, 12, 260, 128, True),
+                                               (2, 33, 2, 200, 128, False)])
+def test_prefill_qkv_shapes(B, H, k, T, D, causal, guard):
+    """CHAI-QKV prefill on the tensor-core kernel: clusters of many members, singletons, head_dim 64, not causal."""
+    r = synth.batch_partitions(B, H, k, "uneven", T, 81, H)
+    g = torch.Generator().manual_seed(T + H)
+    q = (torch.randn(B, H, T, D, generator=g) * 2.0).to(torch.bfloat16)
+    kr = (torch.randn(B, k, T, D, generator=g) * 0.5).to(torch.bfloat16)
+    vr = (torch.randn(B, k, T, D, generator=g) * 0.5).to(torch.bfloat16)
+    mem, reps = torch.as_tensor(r[0]), torch.as_tensor(r[1])
+    scale = 1.0 / np.sqrt(D)
+    out = guard.empty((B, H, T, D), torch.bfloat16)
+    chai.chai_prefill_attention_qkv(q.to(DEV), kr.to(DEV), vr.to(DEV), mem.to(DEV), reps.to(DEV), scale, causal, 0, out=out)
+    got = out.float().cpu().numpy()
+    ref = orc.cha_attention_qkv(q, kr, vr, mem, reps, scale, causal)
+    assert_parity(got, ref, "bf16", f"QKV prefill B {B} H {H} k {k} T {T} D {D} causal {causal}")
+    for b in range(B):
+        for h in range(H):
+            assert np.array_equal(got[b, h], got[b, int(reps[b, int(mem[b, h])])])   # a member's rows ARE its representative's
+
+
+def test_prefill_qkv_bad_membership_is_reported():
+    """Heads that name no cluster, a cluster without a usable representative: zero rows and the status word; the
+    other heads are untouched by it."""
+    B, H, k, T, D = 2, 10, 3, 200, 128
+    r = synth.batch_partitions(B, H, k, "uneven", 3, 82, T)
+    g = torch.Generator().manual_seed(9)
+    q = (torch.randn(B, H, T, D, generator=g) * 2.0).to(torch.bfloat16)
+    kr = (torch.randn(B, k, T, D, generator=g) * 0.5).to(torch.bfloat16)
+    vr = (torch.randn(B, k, T, D, generator=g) * 0.5).to(torch.bfloat16)
+    mem, reps = torch.as_tensor(r[0]).clone(), torch.as_tensor(r[1]).clone()
+    ref = orc.cha_attention_qkv(q, kr, vr, mem, reps, 1.0 / np.sqrt(D), True)
+    non_reps = [h for h in range(H) if h not in reps[0].tolist()]
+    mem[0, non_reps[0]] = 77                     # no such cluster
+    lost = [h for h in range(H) if int(mem[1, h]) == 1]
+    reps[1, 1] = -1                              # cluster 1 of request 1 has no representative
+    ws = chai.new_workspace(int(chai.load().chai_prefill_qkv_workspace_bytes(B, H, k, T, D, chai.CHAI_BF16)), DEV)
+    out = torch.full((B, H, T, D), 7.0, dtype=torch.bfloat16, device=DEV)
+    chai.chai_prefill_attention_qkv(q.to(DEV), kr.to(DEV), vr.to(DEV), mem.to(DEV), reps.to(DEV), 1.0 / np.sqrt(D), True, 0,
+                                    out=out, workspace=ws)
+    assert chai.chai_device_status(ws) == chai.CHAI_ERR_BAD_MEMBERSHIP
+    got = out.float().cpu().numpy()
+    bad = {(0, non_reps[0])} | {(1, h) for h in lost}
+    for b in range(B):
+        for h in range(H):
+            if (b, h) in bad:
+                assert not got[b, h].any()
+            else:
+                assert_parity(got[b, h], ref[b, h], "bf16", f"head ({b},{h}) beside unresolved ones")
+
+
 def test_qkv_bad_membership_is_reported():
     B, H, k, T = 1, 6, 2, 64
     case = ragged_case(2, 5, B, H, k, T)
