@@ -558,6 +558,11 @@ def bench_serving(device, peaks, iters=20, warmup=3):
         return e0.elapsed_time(e1) / ((iters // 5) * 5 * len(sets))
 
     ms_d_b2b, ms_f_b2b = back_to_back(seq), back_to_back(full)
+    # equal lengths that end exactly on a 128-row tile, one row short of it and one row past it: a ragged last tile
+    # must cost what its bytes cost (it once cost several full tiles)
+    tail_check = {}
+    for n in (T_cap - 641, T_cap - 640, T_cap - 639):
+        tail_check[str(n)] = back_to_back(torch.full((B,), n, dtype=torch.int32, device=device)) * 1e3
     del sets
     # append (no advance, so every run writes the same rows)
     k_new = torch.randn((B, H, D), device=device).to(torch.bfloat16)
@@ -591,6 +596,7 @@ def bench_serving(device, peaks, iters=20, warmup=3):
                                                "full_length_us": ms_f_b2b * 1e3,
                                                "full_length_gbs": bytes_f / (ms_f_b2b * 1e-3) / 1e9,
                                                "us_over_full_length_us_times_byte_ratio": ms_d_b2b / (ms_f_b2b * bytes_d / bytes_f),
+                                               "equal_lengths_us": tail_check,
                                                "note": "four cache sets in rotation, the calls captured in a CUDA graph and replayed"}},
             "compact_inplace": {"us": ms_c * 1e3, "planes_moved": moved, "algorithmic_mb": bytes_c / 1e6, "gbs": gbs_c,
                                 "roofline": {"bound": "hbm", "achieved": gbs_c, "peak": peaks["hbm"], "unit": "GB/s",
