@@ -72,3 +72,20 @@ def test_decode_fp8_from_a_cache_compacted_in_place():
     ref = orc.decode_attention_fp8(c["q"], k8_full[:, :k].cpu().numpy(), v8.cpu().numpy(), ks.cpu().numpy(),
                                    vs.cpu().numpy(), c["membership"], c["reps"], [T_cap] * B, c["scale"])
     assert_parity(out.float().cpu().numpy(), ref, "bf16", "fp8 decode, strided K cache")
+
+
+@pytest.mark.parametrize("k", [8, 32])
+def test_decode_fp8_at_workload_2_layer_shape(k):
+    """The shape and launch configuration the fp8 bench leg times (B 16, H 32, T 2048, D 128): every output element
+    against the oracle on the numbers the bytes stand for."""
+    w = synth.WORKLOADS[2]
+    c = synth.decode_layer(2, 3, 2, B=w.B, H=w.H, T=w.T, k=k)
+    k8, ks = chai.chai_quantize_cache_fp8(c["k_rep"].to(DEV))
+    v8, vs = chai.chai_quantize_cache_fp8(c["v"].to(DEV))
+    out = chai.chai_decode_attention_fp8(c["q"].to(DEV), k8, v8, ks, vs, c["membership"].to(DEV), c["reps"].to(DEV),
+                                         c["scale"])
+    got = out.float().cpu().numpy()
+    ref = orc.decode_attention_fp8(c["q"], k8.cpu().numpy(), v8.cpu().numpy(), ks.cpu().numpy(), vs.cpu().numpy(),
+                                   c["membership"], c["reps"], [w.T] * w.B, c["scale"])
+    assert np.isfinite(got).all()
+    assert_parity(got, ref, "bf16", f"fp8 decode, workload 2 layer shape, k {k}")
