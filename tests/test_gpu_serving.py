@@ -325,3 +325,41 @@ def test_cluster_sweep_on_unstructured_features():
     ref_curve, ref_knee = orc.cluster_sweep(feats, 24, 20, 3)
     assert np.allclose(curve.cpu().numpy(), ref_curve, rtol=1e-12, atol=1e-18)
     assert knee.cpu().tolist() == ref_knee.tolist()
+
+
+@pytest.mark.parametrize("k", [8, 16])
+def test_decode_qkv_at_workload_2_layer_shape(k):
+    """CHAI-QKV decode at the shape and launch configuration its bench leg times (B 16, H 32, T 2048, D 128; one launch
+    with the clusters as heads): every output element against the oracle."""
+    w = synth.WORKLOADS[2]
+    c = synth.decode_layer(2, 4, 5, B=w.B, H=w.H, T=w.T, k=k)
+    reps = c["reps"]
+    v_rep = torch.stack([c["v"][b].index_select(0, reps[b].long()) for b in range(w.B)]).contiguous()
+    out = chai.chai_decode_attention_qkv(c["q"].to(DEV), c["k_rep"].to(DEV), v_rep.to(DEV), c["membership"].to(DEV),
+                                         reps.to(DEV), c["scale"])
+    got = out.float().cpu().numpy()
+    ref = orc.cha_attention_qkv(c["q"], c["k_rep"], v_rep, c["membership"], reps, c["scale"], False)
+    assert_parity(got, ref, "bf16", f"QKV decode, workload 2 layer shape, k {k}")
+
+
+def test_prefill_qkv_at_workload_5_shape_sampled_rows():
+    """CHAI-QKV prefill at workload 5's shape (B 4, T 2048, H 32, k 8; one launch, a work item per cluster): run-to-run
+    bitwise identical; first rows, rows across a query-tile boundary and last rows against the oracle."""
+    case = synth.prefill_case(seed=3, device=DEV)
+    B, H, k, T = case["B"], case["H"], case["k"], case["T"]
+    k_rep = chai.chai_compact_k_cache(case["k_full"], case["reps"])
+    v_rep = torch.stack([case["v"][b].index_select(0, case["reps"][b].long()) for b in range(B)]).contiguous()
+    run = lambda: chai.chai_prefill_attention_qkv(case["q_full"], k_rep, v_rep, case["membership"], case["reps"],
+                                                  case["scale"], True, 0)
+    out, out2 = run(), run()
+    torch.cuda.synchronize()
+    assert torch.equal(out, out2)
+    q, kr, vr = case["q_full"].cpu(), k_rep.cpu(), v_rep.cpu()
+    mem, reps = case["membership"].cpu(), case["reps"].cpu()
+    head = orc.cha_attention_qkv(q[:, :, :192], kr[:, :, :192], vr[:, :, :192], mem, reps, case["scale"], True)
+    assert_parity(out[:, :, :192].float().cpu().numpy(), head, "bf16", "QKV prefill first rows")
+    lo, hi = 992, 1056
+    mid = orc.cha_attention_qkv(q[:, :, :hi], kr[:, :, :hi], vr[:, :, :hi], mem, reps, case["scale"], True)
+    assert_parity(out[:, :, lo:hi].float().cpu().numpy(), mid[:, :, lo:hi], "bf16", "QKV prefill middle rows")
+    tail = orc.cha_attention_qkv(q[:, :, T - 64:], kr, vr, mem, reps, case["scale"], True)
+    assert_parity(out[:, :, T - 64:].float().cpu().numpy(), tail, "bf16", "QKV prefill last rows")
