@@ -363,3 +363,25 @@ def test_prefill_qkv_at_workload_5_shape_sampled_rows():
     assert_parity(out[:, :, lo:hi].float().cpu().numpy(), mid[:, :, lo:hi], "bf16", "QKV prefill middle rows")
     tail = orc.cha_attention_qkv(q[:, :, T - 64:], kr, vr, mem, reps, case["scale"], True)
     assert_parity(out[:, :, T - 64:].float().cpu().numpy(), tail, "bf16", "QKV prefill last rows")
+
+
+def test_ragged_decode_at_the_serving_bench_shape(guard):
+    """The ragged decode call its bench leg times: workload 2's layer shape (B 16, H 32, k 8, D 128, capacity 2048),
+    lengths spread over 1/4..1 of the capacity, keys read from a cache compacted in place (strided planes).  Every
+    output element against the oracle."""
+    w = synth.WORKLOADS[2]
+    k, B, H, T_cap = 8, w.B, w.H, w.T
+    c = synth.decode_layer(2, 0, 1, B=B, H=H, T=T_cap, k=k, with_k_full=True)
+    rng = np.random.default_rng(7)
+    lens = rng.integers(T_cap // 4, T_cap, size=B).astype(np.int32)
+    lens[0] = T_cap - 1
+    cache = c["k_full"].to(DEV).clone()
+    chai.chai_compact_k_cache_inplace(cache, c["reps"].to(DEV), T=T_cap)
+    q = c["q"].to(DEV)
+    out = chai.chai_decode_attention_ragged(q, cache, c["v"].to(DEV), c["membership"].to(DEV), c["reps"].to(DEV),
+                                            torch.as_tensor(lens, device=DEV), c["scale"], T_max=T_cap, k_planes=k,
+                                            out=guard.empty_like(q))
+    torch.cuda.synchronize()
+    ref = orc.decode_attention_ragged(c["q"], c["k_rep"], c["v"], c["membership"], c["reps"], [int(n) for n in lens],
+                                      c["scale"])
+    assert_parity(out.float().cpu().numpy(), ref, "bf16", "ragged decode at the serving bench shape")
