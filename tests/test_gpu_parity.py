@@ -298,6 +298,24 @@ def test_compaction_bit_exact():
         assert not got[2, 3, :T].any()
 
 
+@pytest.mark.parametrize("k", [12, 24, 36])
+def test_compaction_bit_exact_at_workload_4_layer_shape(k):
+    """The compaction calls the bench leg times (B 4, H 72, T 2048, D 128, k = 12 / 24 / 36), out of place and in place,
+    bit for bit against the oracle's gather."""
+    w = synth.WORKLOADS[4]
+    B, H, T, D = w.B, w.H, w.T, w.D
+    g = torch.Generator().manual_seed(k)
+    kf = torch.randn(B, H, T, D, generator=g).to(torch.bfloat16)
+    _, reps = synth.batch_partitions(B, H, k, "uneven", k, 4)
+    reps_t = torch.as_tensor(reps, device=DEV)
+    want, _ = orc.compact_k_cache(kf.view(torch.int16).numpy(), reps)
+    got = chai.chai_compact_k_cache(kf.to(DEV), reps_t)
+    assert np.array_equal(got.cpu().view(torch.int16).numpy(), want)
+    cache = kf.to(DEV).clone()
+    chai.chai_compact_k_cache_inplace(cache, reps_t)
+    assert np.array_equal(cache[:, :k].cpu().view(torch.int16).numpy(), want)
+
+
 # ---- prefill --------------------------------------------------------------------------------------------
 
 def prefill_inputs(seed, B, H, T, k, dtype="bf16", kind="uneven", peaked=1.0, D=128):
